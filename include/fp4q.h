@@ -1,0 +1,187 @@
+/*
+ * fp4q -- transposition-invariant 2D-block FP4 quantization and the block-scaled
+ * GEMMs it feeds, for NVIDIA B200 (sm_100a).  C ABI of libfp4q.so.
+ *
+ * Method: "Stable FP4 Training via Transposition-Invariant Block Quantization".
+ *   Section 3      2D square blocks (32x32) share one scale; S(B_ij) = S(B_ij^T).
+ *   Section 3.1    truncation-free scale S = 2^ceil(log2(2M/(Qp-Qn))); stochastic rounding
+ *                  with E[roundS(x)] = x for the backward pass.
+ *   Section 3.2    MXFP8 for the query and key projections.
+ *   Section 3, "Application to linear layers":  Y = X W^T,  dX = dY W,  dW = dY^T X.
+ *
+ * Conventions common to every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the descriptor structs
+ *     themselves (fp4q_tensor, fp4q_groups) are read on the HOST during the call.
+ *   - The library allocates no device memory, never synchronises the device, and only
+ *     enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     The first call in a process creates per-process state (module load, driver entry
+ *     point lookup) and should be made outside stream capture.
+ *   - Every function returns an fp4q_status; nothing throws, traps or aborts.  Argument
+ *     errors are reported before any work is enqueued.  Device-side anomalies (a bounded
+ *     wait that ran out) are recorded in the workspace status word and read back with
+ *     fp4q_workspace_status(); the kernel then skips its remaining work and exits normally.
+ *   - Matrices are row-major with an explicit leading dimension.
+ */
+#ifndef FP4Q_H
+#define FP4Q_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FP4Q_OK = 0,
+    FP4Q_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+    FP4Q_ERR_SHAPE = 2,       /* negative size, mismatched operand shapes, leading dim too small */
+    FP4Q_ERR_ALIGN = 3,       /* pointer or leading dimension violates an alignment rule      */
+    FP4Q_ERR_UNSUPPORTED = 4, /* valid request this build does not implement                  */
+    FP4Q_ERR_WORKSPACE = 5,   /* workspace missing or smaller than fp4q_workspace_bytes()     */
+    FP4Q_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, tensor map)       */
+    FP4Q_ERR_TIMEOUT = 7      /* device status word: a bounded wait expired inside a kernel   */
+} fp4q_status;
+
+typedef enum {
+    FP4Q_ROUND_NEAREST = 0,    /* round to nearest, ties to even code (forward pass)           */
+    FP4Q_ROUND_STOCHASTIC = 1  /* stochastic rounding (gradient tensors in the backward pass) */
+} fp4q_round;
+
+typedef enum { FP4Q_OUT_BF16 = 0, FP4Q_OUT_F32 = 1 } fp4q_out;
+
+/* fp4q_quantize2d flag: key the stochastic-rounding stream on the element's index in the
+ * TRANSPOSED tensor (j*rows + i instead of i*cols + j), so that quantize(A^T) with this flag
+ * reproduces quantize(A) transposed bit for bit. */
+#define FP4Q_INDEX_TRANSPOSED 1u
+
+/*
+ * A 2D-block-quantized tensor with logical source shape [rows, cols] (Section 3; appendix
+ * "2D Block Scaling and Transposition Consistency").  One UE8M0 scale byte (code = e + 127,
+ * S = 2^e) per 32x32 block serves both payload layouts:
+ *   q_rm  [rows, ld_rm] bytes: element (i,j) is nibble (j&1) of q_rm[i*ld_rm + j/2]
+ *   q_t   [cols, ld_t ] bytes: element (i,j) is nibble (i&1) of q_t [j*ld_t  + i/2]   (may be NULL)
+ *   scale [ceil(rows/32), ld_s] bytes: block (I,J) at scale[I*ld_s + J]
+ * The low nibble holds the even index.  Element codes are E2M1: bit 3 sign, bits 2..0
+ * magnitude code for {0, 0.5, 1, 1.5, 2, 3, 4, 6}.
+ * Alignment: q_rm and q_t 16-byte aligned; ld_rm and ld_t multiples of 16 bytes with
+ * ld_rm >= ceil32(cols)/2 and ld_t >= ceil32(rows)/2 (ceil32 = round up to 32);
+ * ld_s >= ceil(cols/32).  The quantizer writes every payload byte of every block it
+ * touches (codes beyond the logical extent are 0); bytes beyond ceil32(.)/2 are left alone.
+ */
+typedef struct {
+    int64_t rows, cols;
+    uint8_t *q_rm;
+    int64_t ld_rm;
+    uint8_t *q_t;
+    int64_t ld_t;
+    uint8_t *scale;
+    int64_t ld_s;
+} fp4q_tensor;
+
+/*
+ * Token groups of a grouped (mixture-of-experts) product: group g owns rows
+ * row_offsets[g] .. row_offsets[g+1]-1 of the token matrices.  row_offsets is a DEVICE array
+ * of n_groups+1 non-decreasing int64 values, each a multiple of 128, with row_offsets[0] = 0
+ * and row_offsets[n_groups] = the token matrices' row count; padding rows inside a group must
+ * hold zeros (the boundary-block rule of the appendix then makes them inert).  Groups may be
+ * empty.
+ */
+typedef struct {
+    int32_t n_groups;
+    const int64_t *row_offsets;
+} fp4q_groups;
+
+/*
+ * fp4q_quantize2d -- Sections 3 and 3.1; appendix "2D Block Scaling ..." and "Rounding ...".
+ * Cuts x (BF16, [rows, cols], leading dimension ld_x in ELEMENTS, any 2-byte-aligned pointer;
+ * fastest when 16-byte aligned with ld_x a multiple of 8) into 32x32 blocks; per block takes the
+ * maximum magnitude M over the valid entries, the truncation-free scale S = 2^e with e the
+ * smallest integer such that 6*2^e >= M (clamped to [-127, 127]; M = 0 gives e = -127), and
+ * rounds every x/S to E2M1: to nearest (ties to even) or stochastically.  In stochastic mode
+ * an element between neighbours lo <= v < hi goes up iff floor(256*(v-lo)/(hi-lo)) + r8 >= 256
+ * where r8 is byte (idx & 15) of Philox4x32-10(counter = (idx>>4 low, idx>>4 high, tensor_id, 0),
+ * key = (seed low, seed high)) and idx = i*cols + j.  The same code is written to out->q_rm and
+ * (unless NULL) out->q_t, and the scale byte to out->scale.  Inputs are expected finite; for
+ * completeness M ignores non-finite entries, +-Inf becomes +-6 and NaN becomes +0.
+ * out->rows/cols must equal rows/cols.  rows == 0 or cols == 0 is a no-op.
+ */
+fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                            const fp4q_tensor *out, fp4q_round mode, uint64_t seed,
+                            uint32_t tensor_id, uint32_t flags, void *stream);
+
+/* GEMM workspace: fp4q_workspace_bytes() bytes of device memory, 256-byte aligned, zeroed once by
+ * the caller before first use (the kernels restore what they use).  Holds the device status word.
+ * Calls that share a workspace must not overlap on the GPU. */
+size_t fp4q_workspace_bytes(void);
+
+/* Reads the status word of a workspace (synchronous 4-byte device-to-host copy on `stream`
+ * followed by a stream synchronise) and clears it.  FP4Q_OK, FP4Q_ERR_TIMEOUT or FP4Q_ERR_CUDA. */
+fp4q_status fp4q_workspace_status(void *ws, void *stream);
+
+/*
+ * fp4q_gemm_fwd -- Y[T,N] = X^[T,K] W^[N,K]^T  (Section 3, first product), FP32 accumulation.
+ * Reads X.q_rm and W.q_rm (both contraction-contiguous) with scales X.scale[t/32, k/32] and
+ * W.scale[n/32, k/32].  Y is BF16 or FP32 (dt), leading dimension ldy in elements; Y must be
+ * 16-byte aligned and ldy*sizeof(element) a multiple of 16.  T, N arbitrary; K = X.cols = W.cols.
+ * Grouped form (g != NULL): X is the permuted token matrix, W the expert stack [n_groups*N, K];
+ * row t of group g is multiplied by rows g*N .. g*N+N-1 of the stack.
+ */
+fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy,
+                          fp4q_out dt, const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * fp4q_gemm_dgrad -- dX[T,K] = dY^[T,N] W^[N,K]  (Section 3, second product).
+ * Reads dY.q_rm and W.q_t; the scale of W for output column k and contraction block nb is
+ * W.scale[nb, k/32] -- the same bytes the forward product used, read transposed.
+ * Grouped form: W is the stack [n_groups*N, K]; rows of group g contract over stack rows g*N...
+ */
+fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx,
+                            fp4q_out dt, const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * fp4q_gemm_wgrad -- dW[N,K] = dY^[T,N]^T X^[T,K]  (Section 3, third product).
+ * Reads dY.q_t and X.q_t (both token-contiguous) with scales dY.scale[t/32, n/32] and
+ * X.scale[t/32, k/32].  accumulate != 0 adds to the existing dW (FP32 output only).
+ * Grouped form: dW is the stack [n_groups*N, K]; block g contracts over the rows of group g
+ * only; an empty group yields zeros (or leaves dW unchanged when accumulating).
+ */
+fp4q_status fp4q_gemm_wgrad(const fp4q_tensor *dY, const fp4q_tensor *X, void *dW, int64_t ldw,
+                            fp4q_out dt, int accumulate, const fp4q_groups *g, void *ws,
+                            size_t ws_bytes, void *stream);
+
+/*
+ * fp4q_mxfp8_quantize1d -- Section 3.2 operand format: x (BF16 [rows, cols], ld_x elements) to
+ * E4M3 payload q[rows, ld_q] (bytes; ld_q multiple of 16, q 16-byte aligned) with one UE8M0 scale
+ * per 32 consecutive elements of a row, scale[rows, ld_s], ld_s >= ceil(cols/32).  The block scale
+ * is the smallest power of two with 448*S >= M (clamped as above); rounding to nearest even;
+ * +-Inf -> +-448, NaN -> 0.  Payload bytes from cols to ceil32(cols) are written as 0.
+ */
+fp4q_status fp4q_mxfp8_quantize1d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                  uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s,
+                                  void *stream);
+
+/*
+ * fp4q_mxfp8_qk -- the query and key projections in MXFP8 (Section 3.2):
+ *   Q[T,N] = X^ Wq^^T,  K[T,N] = X^ Wk^^T,  FP32 accumulation,
+ * on operands produced by fp4q_mxfp8_quantize1d: xq [T, ld_xq] / xs [T, ld_xs];
+ * wq_q, wk_q [N, ld_wq] / wq_s, wk_s [N, ld_ws]; contraction length Kdim.
+ * Q_out and K_out are BF16 or FP32 with leading dimension ldo (elements).  Either weight may be
+ * NULL to skip that projection.
+ */
+fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, int64_t ld_xs,
+                          int64_t T, int64_t Kdim,
+                          const uint8_t *wq_q, const uint8_t *wq_s,
+                          const uint8_t *wk_q, const uint8_t *wk_s, int64_t ld_wq, int64_t ld_ws,
+                          int64_t N, void *Q_out, void *K_out, int64_t ldo, fp4q_out dt,
+                          void *ws, size_t ws_bytes, void *stream);
+
+const char *fp4q_status_string(fp4q_status s);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int fp4q_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP4Q_H */

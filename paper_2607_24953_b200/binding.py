@@ -1,0 +1,254 @@
+"""Thin Python binding of libfp4q.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/fp4q.h) and does nothing
+but turn torch tensors into device pointers, sizes and leading dimensions.  All arithmetic runs in
+the CUDA kernels of the library.  There is no CPU fallback: if the library is missing or the
+tensors are not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfp4q.so")
+
+ROUND_NEAREST = 0
+ROUND_STOCHASTIC = 1
+OUT_BF16 = 0
+OUT_F32 = 1
+INDEX_TRANSPOSED = 1
+
+EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgrad",
+           "fp4q_mxfp8_quantize1d", "fp4q_mxfp8_qk", "fp4q_workspace_bytes", "fp4q_workspace_status",
+           "fp4q_status_string", "fp4q_version"]
+
+
+class Fp4qError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: status %d (%s)" % (where, status, status_string(status)))
+
+
+class _CTensor(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("q_rm", ctypes.c_void_p), ("ld_rm", ctypes.c_int64),
+                ("q_t", ctypes.c_void_p), ("ld_t", ctypes.c_int64),
+                ("scale", ctypes.c_void_p), ("ld_s", ctypes.c_int64)]
+
+
+class _CGroups(ctypes.Structure):
+    _fields_ = [("n_groups", ctypes.c_int32), ("row_offsets", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libfp4q.so (built in-tree by paper_2607_24953_b200.build). Fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libfp4q.so is not built: run `python -m paper_2607_24953_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        i64, u64, u32, vp, ci = ctypes.c_int64, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_int
+        L.fp4q_quantize2d.restype = ci
+        L.fp4q_quantize2d.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_CTensor), ci, u64, u32, u32, vp]
+        L.fp4q_mxfp8_quantize1d.restype = ci
+        L.fp4q_mxfp8_quantize1d.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
+        L.fp4q_workspace_bytes.restype = ctypes.c_size_t
+        L.fp4q_workspace_bytes.argtypes = []
+        L.fp4q_workspace_status.restype = ci
+        L.fp4q_workspace_status.argtypes = [vp, vp]
+        L.fp4q_status_string.restype = ctypes.c_char_p
+        L.fp4q_status_string.argtypes = [ci]
+        L.fp4q_version.restype = ci
+        L.fp4q_version.argtypes = []
+        gemm_args = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64, ci, ctypes.POINTER(_CGroups),
+                     vp, ctypes.c_size_t, vp]
+        if hasattr(L, "fp4q_gemm_fwd"):
+            L.fp4q_gemm_fwd.restype = ci
+            L.fp4q_gemm_fwd.argtypes = gemm_args
+            L.fp4q_gemm_dgrad.restype = ci
+            L.fp4q_gemm_dgrad.argtypes = gemm_args
+            L.fp4q_gemm_wgrad.restype = ci
+            L.fp4q_gemm_wgrad.argtypes = gemm_args[:5] + [ci] + gemm_args[5:]
+        if hasattr(L, "fp4q_mxfp8_qk"):
+            L.fp4q_mxfp8_qk.restype = ci
+            L.fp4q_mxfp8_qk.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, i64, i64, i64, vp, vp, i64,
+                                        ci, vp, ctypes.c_size_t, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().fp4q_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise Fp4qError(status, where)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError("%s must live on a CUDA device (there is no CPU path)" % name)
+    return t
+
+
+@dataclass
+class QTensor:
+    """Device buffers of a 2D-block-quantized tensor (fp4q_tensor of include/fp4q.h)."""
+    rows: int
+    cols: int
+    q_rm: torch.Tensor               # uint8 [rows, ld_rm]
+    q_t: Optional[torch.Tensor]      # uint8 [cols, ld_t] or None
+    scale: torch.Tensor              # uint8 [ceil(rows/32), ld_s]
+
+    def c_struct(self) -> _CTensor:
+        return _CTensor(self.rows, self.cols,
+                        self.q_rm.data_ptr(), self.q_rm.stride(0),
+                        self.q_t.data_ptr() if self.q_t is not None else None,
+                        self.q_t.stride(0) if self.q_t is not None else 0,
+                        self.scale.data_ptr(), self.scale.stride(0))
+
+
+def _pad16(n: int) -> int:
+    return (n + 15) // 16 * 16
+
+
+def alloc_qtensor(rows: int, cols: int, device, want_t: bool = True) -> QTensor:
+    """Allocate the output buffers of fp4q_quantize2d with the leading dimensions the ABI asks for."""
+    ld_rm = max(_pad16((cols + 31) // 32 * 16), 16)
+    ld_t = max(_pad16((rows + 31) // 32 * 16), 16)
+    q_rm = torch.empty((rows, ld_rm), dtype=torch.uint8, device=device)
+    q_t = torch.empty((cols, ld_t), dtype=torch.uint8, device=device) if want_t else None
+    scale = torch.empty(((rows + 31) // 32, max((cols + 31) // 32, 1)), dtype=torch.uint8, device=device)
+    return QTensor(rows, cols, q_rm, q_t, scale)
+
+
+def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = ROUND_NEAREST, seed: int = 0,
+                    tensor_id: int = 0, flags: int = 0, want_t: bool = True, stream=None) -> QTensor:
+    """x: BF16 [rows, cols] on the GPU, unit stride along columns. Returns (and fills) a QTensor."""
+    _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+        raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
+    rows, cols = x.shape
+    if out is None:
+        out = alloc_qtensor(rows, cols, x.device, want_t)
+    cs = out.c_struct()
+    st = lib().fp4q_quantize2d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, ctypes.byref(cs),
+                               mode, seed, tensor_id, flags, _stream(stream))
+    _check(st, "fp4q_quantize2d")
+    return out
+
+
+def fp4q_mxfp8_quantize1d(x: torch.Tensor, stream=None):
+    """x: BF16 [rows, cols]. Returns (q uint8 [rows, ld_q], scale uint8 [rows, ceil(cols/32)])."""
+    _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+        raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
+    rows, cols = x.shape
+    ld_q = max((cols + 31) // 32 * 32, 32)
+    q = torch.empty((rows, ld_q), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((rows, max((cols + 31) // 32, 1)), dtype=torch.uint8, device=x.device)
+    st = lib().fp4q_mxfp8_quantize1d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, q.data_ptr(), ld_q,
+                                     scale.data_ptr(), scale.stride(0), _stream(stream))
+    _check(st, "fp4q_mxfp8_quantize1d")
+    return q, scale
+
+
+def fp4q_workspace_bytes() -> int:
+    return int(lib().fp4q_workspace_bytes())
+
+
+def alloc_workspace(device) -> torch.Tensor:
+    return torch.zeros(fp4q_workspace_bytes(), dtype=torch.uint8, device=device)
+
+
+def fp4q_workspace_status(ws: torch.Tensor, stream=None) -> int:
+    return int(lib().fp4q_workspace_status(ws.data_ptr(), _stream(stream)))
+
+
+def _groups(row_offsets: Optional[torch.Tensor]):
+    if row_offsets is None:
+        return None, None
+    _dev(row_offsets, "row_offsets")
+    if row_offsets.dtype != torch.int64 or not row_offsets.is_contiguous():
+        raise ValueError("row_offsets must be a contiguous int64 device tensor")
+    g = _CGroups(row_offsets.numel() - 1, row_offsets.data_ptr())
+    return g, ctypes.byref(g)
+
+
+def _out_dtype(dt: int):
+    return torch.bfloat16 if dt == OUT_BF16 else torch.float32
+
+
+def _gemm(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, row_offsets, ws, stream, accumulate=None):
+    dev = a.q_rm.device
+    if out is None:
+        # the ABI wants the leading dimension to be a multiple of 16 bytes: pad it and return a view
+        per16 = 8 if dt == OUT_BF16 else 4
+        ld = max((out_cols + per16 - 1) // per16 * per16, per16)
+        out = torch.empty((out_rows, ld), dtype=_out_dtype(dt), device=dev)[:, :out_cols]
+    if ws is None:
+        ws = alloc_workspace(dev)
+    ca, cb = a.c_struct(), b.c_struct()
+    g, gref = _groups(row_offsets)
+    fn = getattr(lib(), fn_name)
+    args = [ctypes.byref(ca), ctypes.byref(cb), out.data_ptr(), out.stride(0) if out.numel() else out_cols, dt]
+    if accumulate is not None:
+        args.append(int(accumulate))
+    args += [gref, ws.data_ptr(), ws.numel(), _stream(stream)]
+    _check(fn(*args), fn_name)
+    return out
+
+
+def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None):
+    """Y[T,N] = X^ W^^T. Grouped when row_offsets is given (W is then the expert stack [E*N, K])."""
+    n = W.rows if row_offsets is None else W.rows // (row_offsets.numel() - 1)
+    return _gemm("fp4q_gemm_fwd", X, W, X.rows, n, out, dt, row_offsets, ws, stream)
+
+
+def fp4q_gemm_dgrad(dY: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None):
+    """dX[T,K] = dY^ W^."""
+    return _gemm("fp4q_gemm_dgrad", dY, W, dY.rows, W.cols, out, dt, row_offsets, ws, stream)
+
+
+def fp4q_gemm_wgrad(dY: QTensor, X: QTensor, out=None, dt: int = OUT_F32, accumulate: bool = False,
+                    row_offsets=None, ws=None, stream=None):
+    """dW[N,K] = dY^^T X^ (stack [E*N, K] when grouped)."""
+    e = 1 if row_offsets is None else row_offsets.numel() - 1
+    return _gemm("fp4q_gemm_wgrad", dY, X, dY.cols * e, X.cols, out, dt, row_offsets, ws, stream,
+                 accumulate=accumulate)
+
+
+def fp4q_mxfp8_qk(xq, xs, wq_q, wq_s, wk_q, wk_s, T: int, K: int, N: int, dt: int = OUT_BF16, ws=None,
+                  stream=None):
+    """Q = X^ Wq^^T and K = X^ Wk^^T on MXFP8 operands from fp4q_mxfp8_quantize1d."""
+    dev = xq.device
+    per16 = 8 if dt == OUT_BF16 else 4
+    ldo = max((N + per16 - 1) // per16 * per16, per16)
+    q_out = torch.empty((T, ldo), dtype=_out_dtype(dt), device=dev)[:, :N] if wq_q is not None else None
+    k_out = torch.empty((T, ldo), dtype=_out_dtype(dt), device=dev)[:, :N] if wk_q is not None else None
+    if ws is None:
+        ws = alloc_workspace(dev)
+    wref = wq_q if wq_q is not None else wk_q
+    sref = wq_s if wq_s is not None else wk_s
+    p = lambda t: t.data_ptr() if t is not None else None
+    st = lib().fp4q_mxfp8_qk(xq.data_ptr(), xq.stride(0), xs.data_ptr(), xs.stride(0), T, K,
+                             p(wq_q), p(wq_s), p(wk_q), p(wk_s), wref.stride(0), sref.stride(0), N,
+                             p(q_out), p(k_out), ldo, dt, ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "fp4q_mxfp8_qk")
+    return q_out, k_out

@@ -1,0 +1,745 @@
+// Block-scaled tcgen05 GEMMs for sm_100a: C[M,N] = A[M,K] * B[N,K]^T with both operands
+// contraction-contiguous ("K-major"), FP32 accumulation in tensor memory.
+//
+//   kind::mxf4      E2M1 payload, 2 codes per byte, one UE8M0 scale per 32x32 block of the source tensor
+//                   (the 2D-block format): the hardware's per-row, per-32-element scale for row r and
+//                   contraction block kb is scale[r/32][kb] or, for a transposed view, scale[kb][r/32].
+//   kind::mxf8f6f4  E4M3 payload, one UE8M0 scale per row and 32 contraction elements (MXFP8).
+//
+// One persistent CTA per SM, 128x256 output tile, 12 warps:
+//   warp 0      TMA producer: A tile (128 rows x 128 B) and B tile (256 rows x 128 B) per stage, 128B swizzle
+//   warp 1      MMA issuer: tcgen05.cp of the stage's scale image smem -> TMEM, then 4 tcgen05.mma per stage
+//   warp 2      scale loader: compact scale bytes -> the 32-lane x 16-byte image tcgen05.cp expects
+//   warps 4-11  epilogue: tcgen05.ld of the 128x256 FP32 accumulator (each warp 32 lanes x 128 columns),
+//               release of the accumulator as soon as it sits in registers, then convert and store
+// Four smem stages (48 KB of operands + 3 KB of scale image each) form a ring guarded by mbarriers; the
+// scale columns in TMEM form a ring of the same depth.  Every wait is bounded: when a limit is hit the
+// CTA records FP4Q_ERR_TIMEOUT in the workspace, stops issuing work and leaves through the normal exit
+// (TMEM is freed).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace fp4q {
+
+constexpr int BM = 128, BN = 256;
+constexpr int kStages = 4;
+constexpr int kAStageBytes = BM * 128;
+constexpr int kBStageBytes = BN * 128;
+constexpr int kSfStageBytes = 3072;          // SFA 2 x 512 B, SFB 2 x 1024 B
+constexpr int kSfaOff = 0, kSfbOff = 1024;
+constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
+constexpr int kSmemSf = kStages * kSfStageBytes;
+constexpr int kSmemTail = 256;               // barriers, TMEM base, abort flag, scale scratch
+constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemTail;
+constexpr int kThreads = 384;
+constexpr int kTmemCols = 512;
+constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
+constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint8_t kScalePad = 127;           // UE8M0 code of 1.0 for scale slots beyond the tensor (their payload is 0)
+
+enum { KIND_MXF4 = 0, KIND_MXF8 = 1 };
+enum { MODE_DENSE = 0, MODE_GROUPED_ROWS = 1, MODE_GROUPED_K = 2 };
+
+struct ScaleView {
+    const uint8_t *ptr;
+    int64_t stride_row;   // mxf4: bytes between consecutive 32-row tiles; mxf8: bytes between consecutive rows
+    int64_t stride_kb;    // bytes between consecutive contraction blocks of 32
+    int32_t n_row;        // mxf4: number of row tiles; mxf8: number of rows
+    int32_t n_kb;         // number of contraction blocks
+};
+
+struct GemmParams {
+    ScaleView sfa, sfb;
+    void *C;
+    int64_t ldc;
+    int32_t M, N, K;                 // per-problem output rows, output columns, contraction length (elements)
+    int32_t m_tiles, n_tiles, n_tile_total;
+    int32_t out_f32, accumulate;
+    int32_t mode, n_groups;
+    const int64_t *row_offsets;
+    int32_t b_rows_per_group;        // grouped rows: B row offset per group (forward)
+    int32_t b_k_per_group;           // grouped rows: B contraction offset per group (dgrad)
+    uint32_t *status;
+};
+
+struct Tile {
+    int32_t a_row0, b_row0, a_k0, b_k0, k_len, c_row0, c_col0, m_valid, n_valid;
+};
+
+// ---------------------------------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when the limit ran out (the timeout is then recorded) or when another
+// role of this CTA has already given up.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                       uint32_t where)
+{
+    for (uint32_t it = 0; it < kWaitLimit; it++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    if (atomicCAS(status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) status[1] = where;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+
+template <int KIND>
+__device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                         uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
+{
+    if (KIND == KIND_MXF4) {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
+    } else {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
+    }
+}
+
+// Shared-memory matrix descriptor, K-major operand tile stored as rows of 128 B with the 128-byte swizzle
+// (8-row groups 1024 B apart).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Descriptor of a scale image: 32 rows of 16 B, contiguous (no swizzle; 8-row groups 128 B apart).
+__device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | (1ull << 46);
+}
+
+// Instruction descriptor of the block-scaled MMA: formats, K-major operands, N, UE8M0 scales, M, scale byte ids.
+template <int KIND>
+__device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_id)
+{
+    const uint32_t fmt = KIND == KIND_MXF4 ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
+    return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) |
+           ((uint32_t)(BM >> 4) << 24) | (a_sf_id << 29);
+}
+
+#define FP4Q_TMEM_LD_X32(taddr, v)                                                                              \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                      \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                      \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                     \
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), \
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),      \
+                   "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),    \
+                   "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),    \
+                   "=r"(v[29]), "=r"(v[30]), "=r"(v[31])                                                         \
+                 : "r"(taddr))
+
+// ---------------------------------------------------------------------------------------- tile decoding
+
+__device__ __forceinline__ int find_group(const int64_t *offs, int n_groups, int64_t row)
+{
+    int lo = 0, hi = n_groups;      // largest g with offs[g] <= row
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(offs + mid) <= row) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, Tile &t)
+{
+    const int per_problem = p.m_tiles * p.n_tiles;
+    const int g = p.mode == MODE_GROUPED_K ? tile / per_problem : 0;
+    const int local = tile - g * per_problem;
+    const int m_blk = local % p.m_tiles, n_blk = local / p.m_tiles;
+    t.a_row0 = m_blk * BM;
+    t.b_row0 = n_blk * BN;
+    t.a_k0 = t.b_k0 = 0;
+    t.k_len = p.K;
+    t.c_row0 = t.a_row0;
+    t.c_col0 = t.b_row0;
+    t.m_valid = min(BM, p.M - t.a_row0);
+    t.n_valid = min(BN, p.N - t.b_row0);
+    if (p.mode == MODE_GROUPED_ROWS) {
+        const int grp = find_group(p.row_offsets, p.n_groups, (int64_t)t.a_row0);
+        t.b_row0 += grp * p.b_rows_per_group;
+        t.b_k0 = grp * p.b_k_per_group;
+    } else if (p.mode == MODE_GROUPED_K) {
+        const int64_t k0 = __ldg(p.row_offsets + g), k1 = __ldg(p.row_offsets + g + 1);
+        t.a_k0 = t.b_k0 = (int32_t)k0;
+        t.k_len = (int32_t)(k1 - k0);
+        t.c_row0 = g * p.M + t.a_row0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------- scale images
+
+__device__ __forceinline__ uint8_t load_scale(const ScaleView &v, int row, int kb)
+{
+    return (row < v.n_row && kb < v.n_kb) ? __ldg(v.ptr + (int64_t)row * v.stride_row + (int64_t)kb * v.stride_kb) : kScalePad;
+}
+
+// mxf4 / 2D blocks: a stage covers 8 contraction blocks (two chunks of 4).  For 128 operand rows and one chunk
+// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3].
+__device__ __forceinline__ void build_scale_images_2d(const GemmParams &p, const Tile &t, int it, uint8_t *sf_stage,
+                                                      uint8_t *scratch, int lane)
+{
+    {   // A: 2 chunks x 4 row tiles x 4 blocks = 32 bytes, one per lane
+        const int c = lane >> 4, rt = (lane >> 2) & 3, kb = lane & 3;
+        scratch[lane] = load_scale(p.sfa, (t.a_row0 >> 5) + rt, (t.a_k0 >> 5) + it * 8 + c * 4 + kb);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; h++) {   // B: 2 chunks x 8 row tiles x 4 blocks = 64 bytes, two per lane
+        const int idx = lane + 32 * h, c = idx >> 5, rt = (idx >> 2) & 7, kb = idx & 3;
+        scratch[32 + idx] = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + c * 4 + kb);
+    }
+    __syncwarp();
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(scratch);
+    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
+    img[(kSfaOff >> 4) + lane] = s4[0];             // SFA chunk 0
+    img[(kSfaOff >> 4) + 32 + lane] = s4[1];        // SFA chunk 1
+    img[(kSfbOff >> 4) + lane] = s4[2];             // SFB chunk 0, rows 0..127
+    img[(kSfbOff >> 4) + 32 + lane] = s4[3];        // SFB chunk 0, rows 128..255
+    img[(kSfbOff >> 4) + 64 + lane] = s4[4];        // SFB chunk 1, rows 0..127
+    img[(kSfbOff >> 4) + 96 + lane] = s4[5];        // SFB chunk 1, rows 128..255
+    __syncwarp();
+}
+
+// mxf8 / 1D blocks: a stage covers 4 contraction blocks (one chunk); image row l holds rows l, l+32, l+64, l+96.
+__device__ __forceinline__ void build_scale_images_1d(const GemmParams &p, const Tile &t, int it, uint8_t *sf_stage, int lane)
+{
+    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
+#pragma unroll
+    for (int blk = 0; blk < 3; blk++) {   // 0: A rows 0..127; 1, 2: B rows 0..127, 128..255
+        const ScaleView &v = blk == 0 ? p.sfa : p.sfb;
+        const int row0 = blk == 0 ? t.a_row0 : t.b_row0 + (blk - 1) * 128;
+        const int kb0 = ((blk == 0 ? t.a_k0 : t.b_k0) >> 5) + it * 4;
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const int row = row0 + lane + 32 * j;
+            uint32_t word = 0;
+#pragma unroll
+            for (int kb = 0; kb < 4; kb++) word |= (uint32_t)load_scale(v, row, kb0 + kb) << (8 * kb);
+            w[j] = word;
+        }
+        const int off = blk == 0 ? (kSfaOff >> 4) : (kSfbOff >> 4) + (blk - 1) * 32;
+        img[off + lane] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __syncwarp();
+}
+
+// ---------------------------------------------------------------------------------------- epilogue store
+
+__device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row, int col0, int n_cols_valid,
+                                                const uint32_t v[32])
+{
+    // 32 consecutive accumulator columns of one output row, starting at column col0
+    if (n_cols_valid <= 0) return;
+    if (p.out_f32) {
+        float *dst = static_cast<float *>(p.C) + row * p.ldc + col0;
+        if (n_cols_valid >= 32) {
+#pragma unroll
+            for (int q = 0; q < 8; q++) {
+                float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                       __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                if (p.accumulate) {
+                    const float4 old = *reinterpret_cast<const float4 *>(dst + 4 * q);
+                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                *reinterpret_cast<float4 *>(dst + 4 * q) = o;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 32; q++)
+                if (q < n_cols_valid) dst[q] = __uint_as_float(v[q]) + (p.accumulate ? dst[q] : 0.0f);
+        }
+    } else {
+        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.C) + row * p.ldc + col0;
+        if (n_cols_valid >= 32) {
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[8 * q + 2 * e]),
+                                                                   __uint_as_float(v[8 * q + 2 * e + 1]));
+                    w[e] = *reinterpret_cast<const uint32_t *>(&b);
+                }
+                *reinterpret_cast<uint4 *>(dst + 8 * q) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 32; q++)
+                if (q < n_cols_valid) dst[q] = __float2bfloat16_rn(__uint_as_float(v[q]));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------- kernel
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ GemmParams p)
+{
+    constexpr int kStageElems = KIND == KIND_MXF4 ? 256 : 128;   // contraction elements per stage (128 B per row)
+    constexpr int kMmaK = KIND == KIND_MXF4 ? 64 : 32;           // contraction elements per MMA (32 B per row)
+    constexpr int kElemsPerByte = KIND == KIND_MXF4 ? 2 : 1;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *smem_a = smem;
+    uint8_t *smem_b = smem + kStages * kAStageBytes;
+    uint8_t *smem_sf = smem + kSmemOperands;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kSmemOperands + kSmemSf);
+    // bars[0..3] full, bars[4..7] empty, bars[8] accumulator full, bars[9] accumulator empty
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 10);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 10) + 1;
+    uint8_t *scale_scratch = reinterpret_cast<uint8_t *>(bars + 12);    // 96 bytes, 16-byte aligned
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
+    const uint32_t bar_acc_full = smem_u32(bars + 8), bar_acc_empty = smem_u32(bars + 9);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; s++) {
+            mbar_init(bar_full + 8 * s, 2);     // producer's expect_tx arrival + scale loader's arrival
+            mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 8);            // one arrival per epilogue warp
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_slot)),
+                     "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+                Tile t;
+                decode_tile(p, tile, t);
+                const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
+                for (int it = 0; it < n_it; it++) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage))) break;
+                    mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
+                    tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA,
+                                (t.a_k0 + it * kStageElems) / kElemsPerByte, t.a_row0, bar_full + 8 * stage);
+                    tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB,
+                                (t.b_k0 + it * kStageElems) / kElemsPerByte, t.b_row0, bar_full + 8 * stage);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {   // give copies already in flight time to land before the CTA's shared memory is released
+                for (int i = 0; i < 200; i++) __nanosleep(1000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        uint32_t stage = 0, phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            Tile t;
+            decode_tile(p, tile, t);
+            const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
+            if (n_it == 0) continue;
+            if (lane == 0) ok = mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
+            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            if (!ok) break;
+            acc_phase ^= 1u;
+            tcgen05_fence_after();
+            for (int it = 0; it < n_it; it++) {
+                if (lane == 0) ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x210u + stage);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                if (lane == 0) {
+                    tcgen05_fence_after();
+                    const uint32_t sf_smem = smem_u32(smem_sf + stage * kSfStageBytes);
+                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
+                    constexpr int kChunks = KIND == KIND_MXF4 ? 2 : 1;
+#pragma unroll
+                    for (int c = 0; c < kChunks; c++) {
+                        tcgen05_cp_32x128b_warpx4(sf_tmem + 4 * c, smem_desc_scale_image(sf_smem + kSfaOff + 512 * c));
+                        tcgen05_cp_32x128b_warpx4(sf_tmem + 8 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c));
+                        tcgen05_cp_32x128b_warpx4(sf_tmem + 12 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c + 512));
+                    }
+                    const uint64_t adesc = smem_desc_sw128(smem_u32(smem_a + stage * kAStageBytes));
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(smem_b + stage * kBStageBytes));
+                    const int k_left = t.k_len - it * kStageElems;
+                    const int n_mma = min(4, (k_left + kMmaK - 1) / kMmaK);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        if (i < n_mma) {
+                            const int chunk = KIND == KIND_MXF4 ? (i >> 1) : 0;
+                            const uint32_t sf_id = KIND == KIND_MXF4 ? 2u * (i & 1) : (uint32_t)i;
+                            tcgen05_mma_block_scaled<KIND>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
+                                                           instr_desc<KIND>(sf_id, sf_id), sf_tmem + 4 * chunk,
+                                                           sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
+                        }
+                    }
+                    tcgen05_commit(bar_empty + 8 * stage);
+                    if (it == n_it - 1) tcgen05_commit(bar_acc_full);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ scale loader
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            Tile t;
+            decode_tile(p, tile, t);
+            const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
+            for (int it = 0; it < n_it; it++) {
+                if (lane == 0) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                uint8_t *sf_stage = smem_sf + stage * kSfStageBytes;
+                if (KIND == KIND_MXF4) build_scale_images_2d(p, t, it, sf_stage, scale_scratch, lane);
+                else build_scale_images_1d(p, t, it, sf_stage, lane);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_full + 8 * stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 (hardware: warp id mod 4)
+        const int half = (warp - 4) >> 2;        // accumulator columns 128*half .. +127
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            Tile t;
+            decode_tile(p, tile, t);
+            const int row_in_tile = 32 * quarter + lane;
+            const int64_t row = (int64_t)t.c_row0 + row_in_tile;
+            const bool row_ok = row_in_tile < t.m_valid;
+            uint32_t v[4][32];
+            if (t.k_len > 0) {
+                if (lane == 0) ok = mbar_wait(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                acc_phase ^= 1u;
+                tcgen05_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(32 * quarter) << 16) + 128u * half;
+                FP4Q_TMEM_LD_X32(taddr, v[0]);
+                FP4Q_TMEM_LD_X32(taddr + 32, v[1]);
+                FP4Q_TMEM_LD_X32(taddr + 64, v[2]);
+                FP4Q_TMEM_LD_X32(taddr + 96, v[3]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty);     // the accumulator now lives in registers
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; j++)
+#pragma unroll
+                    for (int q = 0; q < 32; q++) v[j][q] = 0u;
+            }
+            if (row_ok) {
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const int col_in_tile = 128 * half + 32 * j;
+                    store_row_chunk(p, row, t.c_col0 + col_in_tile, t.n_valid - col_in_tile, v[j]);
+                }
+            }
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Operand tile map: a [rows, row_bytes] byte matrix with pitch ld_bytes, box = 128 B x box_rows, 128B swizzle.
+static bool make_operand_map(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes, int64_t ld_bytes,
+                             int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld_bytes};
+    const cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Operand {
+    const uint8_t *payload;
+    int64_t rows, row_bytes, ld_bytes;
+    ScaleView sf;
+};
+
+static int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int KIND>
+static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!ws || ws_bytes < sizeof(Workspace)) return FP4Q_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return FP4Q_ERR_ALIGN;
+    if (!aligned(A.payload, 16) || !aligned(B.payload, 16) || A.ld_bytes % 16 || B.ld_bytes % 16) return FP4Q_ERR_ALIGN;
+    const size_t esize = p.out_f32 ? 4 : 2;
+    if (!aligned(p.C, 16) || (p.ldc * esize) % 16) return FP4Q_ERR_ALIGN;
+    if (p.n_tile_total <= 0) return FP4Q_OK;
+
+    CUtensorMap tmA, tmB;
+    if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, BN)) return FP4Q_ERR_CUDA;
+    p.sfa = A.sf;
+    p.sfb = B.sf;
+    p.status = reinterpret_cast<uint32_t *>(ws);
+
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[KIND]) {
+        if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
+            return FP4Q_ERR_CUDA;
+        attr_set[KIND] = true;
+    }
+    const int grid = p.n_tile_total < sm_count() ? p.n_tile_total : sm_count();
+    gemm_block_scaled_kernel<KIND><<<grid, kThreads, kSmemBytes, static_cast<cudaStream_t>(stream)>>>(tmA, tmB, p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
+
+static bool tensor_ok(const fp4q_tensor *t) { return t && t->rows >= 0 && t->cols >= 0; }
+
+static fp4q_status check_groups(const fp4q_groups *g)
+{
+    if (!g) return FP4Q_OK;
+    if (g->n_groups <= 0) return FP4Q_ERR_SHAPE;
+    if (!g->row_offsets) return FP4Q_ERR_NULL;
+    return FP4Q_OK;
+}
+
+// Row-major payload of a tensor [rows, cols] as an operand whose rows are the tensor's rows.
+static Operand operand_rm(const fp4q_tensor *t)
+{
+    Operand o;
+    o.payload = t->q_rm;
+    o.rows = t->rows;
+    o.row_bytes = round_up(t->cols, 32) / 2;
+    o.ld_bytes = t->ld_rm;
+    o.sf = ScaleView{t->scale, t->ld_s, 1, (int32_t)ceil_div(t->rows, 32), (int32_t)ceil_div(t->cols, 32)};
+    return o;
+}
+// Transposed payload: operand rows are the tensor's columns, contraction runs over the tensor's rows.
+static Operand operand_t(const fp4q_tensor *t)
+{
+    Operand o;
+    o.payload = t->q_t;
+    o.rows = t->cols;
+    o.row_bytes = round_up(t->rows, 32) / 2;
+    o.ld_bytes = t->ld_t;
+    o.sf = ScaleView{t->scale, 1, t->ld_s, (int32_t)ceil_div(t->cols, 32), (int32_t)ceil_div(t->rows, 32)};
+    return o;
+}
+
+static void dense_tiles(GemmParams &p)
+{
+    p.m_tiles = (int32_t)ceil_div(p.M, BM);
+    p.n_tiles = (int32_t)ceil_div(p.N, BN);
+    p.n_tile_total = p.m_tiles * p.n_tiles;
+}
+
+}  // namespace fp4q
+
+using namespace fp4q;
+
+static const int64_t kMaxDim = 0x7FFFFFFF - 4096;
+
+extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt,
+                                     const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(X) || !tensor_ok(W)) return X && W ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (fp4q_status s = check_groups(g)) return s;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (X->cols != W->cols) return FP4Q_ERR_SHAPE;
+    const int64_t T = X->rows, K = X->cols;
+    const int64_t N = g ? W->rows / g->n_groups : W->rows;
+    if (g && (W->rows % g->n_groups || N % 32)) return FP4Q_ERR_SHAPE;   // expert blocks must start on a 32-row tile
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim || W->rows > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (T == 0 || N == 0) return FP4Q_OK;
+    if (!Y || !X->q_rm || !W->q_rm || !X->scale || !W->scale) return FP4Q_ERR_NULL;
+    if (ldy < N) return FP4Q_ERR_SHAPE;
+    GemmParams p = {};
+    p.C = Y; p.ldc = ldy; p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)K;
+    p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = 0;
+    dense_tiles(p);
+    if (g) {
+        p.mode = MODE_GROUPED_ROWS; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.b_rows_per_group = (int32_t)N; p.b_k_per_group = 0;
+    }
+    return launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt,
+                                       const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(dY) || !tensor_ok(W)) return dY && W ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (fp4q_status s = check_groups(g)) return s;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    const int64_t T = dY->rows, N = dY->cols, K = W->cols;
+    if (g ? (W->rows != N * g->n_groups) : (W->rows != N)) return FP4Q_ERR_SHAPE;
+    if (g && N % 64) return FP4Q_ERR_UNSUPPORTED;   // a group's contraction range must end on an MMA boundary
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim || W->rows > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (T == 0 || K == 0) return FP4Q_OK;
+    if (!dX || !dY->q_rm || !W->q_t || !dY->scale || !W->scale) return FP4Q_ERR_NULL;
+    if (ldx < K) return FP4Q_ERR_SHAPE;
+    GemmParams p = {};
+    p.C = dX; p.ldc = ldx; p.M = (int32_t)T; p.N = (int32_t)K; p.K = (int32_t)N;
+    p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = 0;
+    dense_tiles(p);
+    if (g) {
+        p.mode = MODE_GROUPED_ROWS; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.b_rows_per_group = 0; p.b_k_per_group = (int32_t)N;
+    }
+    return launch_gemm<KIND_MXF4>(operand_rm(dY), operand_t(W), p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_wgrad(const fp4q_tensor *dY, const fp4q_tensor *X, void *dW, int64_t ldw, fp4q_out dt,
+                                       int accumulate, const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(dY) || !tensor_ok(X)) return dY && X ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (fp4q_status s = check_groups(g)) return s;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (accumulate && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (dY->rows != X->rows) return FP4Q_ERR_SHAPE;
+    const int64_t T = dY->rows, N = dY->cols, K = X->cols;
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (g && N * g->n_groups > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (N == 0 || K == 0) return FP4Q_OK;
+    if (!dW || !dY->q_t || !X->q_t || !dY->scale || !X->scale) return FP4Q_ERR_NULL;
+    if (ldw < K) return FP4Q_ERR_SHAPE;
+    GemmParams p = {};
+    p.C = dW; p.ldc = ldw; p.M = (int32_t)N; p.N = (int32_t)K; p.K = (int32_t)T;
+    p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = accumulate ? 1 : 0;
+    dense_tiles(p);
+    if (g) {
+        p.mode = MODE_GROUPED_K; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.n_tile_total *= g->n_groups;
+    }
+    return launch_gemm<KIND_MXF4>(operand_t(dY), operand_t(X), p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, int64_t ld_xs, int64_t T,
+                                     int64_t Kdim, const uint8_t *wq_q, const uint8_t *wq_s, const uint8_t *wk_q,
+                                     const uint8_t *wk_s, int64_t ld_wq, int64_t ld_ws, int64_t N, void *Q_out,
+                                     void *K_out, int64_t ldo, fp4q_out dt, void *ws, size_t ws_bytes, void *stream)
+{
+    if (T < 0 || N < 0 || Kdim < 0) return FP4Q_ERR_SHAPE;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (T > kMaxDim || N > kMaxDim || Kdim > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (T == 0 || N == 0) return FP4Q_OK;
+    if (!xq || !xs) return FP4Q_ERR_NULL;
+    if ((wq_q && (!wq_s || !Q_out)) || (wk_q && (!wk_s || !K_out))) return FP4Q_ERR_NULL;
+    const int64_t kpad = round_up(Kdim, 32), nkb = ceil_div(Kdim, 32);
+    if (ld_xq < kpad || ld_wq < kpad || ld_xs < nkb || ld_ws < nkb || ldo < N) return FP4Q_ERR_SHAPE;
+    Operand A;
+    A.payload = xq; A.rows = T; A.row_bytes = kpad; A.ld_bytes = ld_xq;
+    A.sf = ScaleView{xs, ld_xs, 1, (int32_t)T, (int32_t)nkb};
+    const uint8_t *wq[2] = {wq_q, wk_q};
+    const uint8_t *wsf[2] = {wq_s, wk_s};
+    void *out[2] = {Q_out, K_out};
+    for (int i = 0; i < 2; i++) {
+        if (!wq[i]) continue;
+        Operand B;
+        B.payload = wq[i]; B.rows = N; B.row_bytes = kpad; B.ld_bytes = ld_wq;
+        B.sf = ScaleView{wsf[i], ld_ws, 1, (int32_t)N, (int32_t)nkb};
+        GemmParams p = {};
+        p.C = out[i]; p.ldc = ldo; p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)Kdim;
+        p.out_f32 = dt == FP4Q_OUT_F32;
+        dense_tiles(p);
+        if (fp4q_status s = launch_gemm<KIND_MXF8>(A, B, p, ws, ws_bytes, stream)) return s;
+    }
+    return FP4Q_OK;
+}

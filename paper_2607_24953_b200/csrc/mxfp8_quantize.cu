@@ -1,0 +1,120 @@
+// fp4q_mxfp8_quantize1d: BF16 -> MXFP8 operand (E4M3 payload, one UE8M0 scale per 32 consecutive
+// elements of a row), the operand format of the query/key projections.  Streaming kernel: each
+// thread owns 16 consecutive elements (two 128-bit loads, one 128-bit store); two neighbouring
+// lanes own one 32-element block and exchange their maxima with one shuffle.
+#include "common.cuh"
+
+namespace fp4q {
+
+struct Mxfp8QuantParams {
+    const uint16_t *x;
+    int64_t rows, cols, ld_x;
+    uint8_t *q;
+    int64_t ld_q;
+    uint8_t *scale;
+    int64_t ld_s;
+    int64_t segs_per_row;   // 16-element segments per row, even
+    int x_vec_ok;
+};
+
+// {hi, lo} -> two E4M3 bytes (hi in bits 15..8), round to nearest even, saturating to +-448.
+__device__ __forceinline__ uint32_t cvt_rn_e4m3x2(float hi, float lo)
+{
+    uint16_t d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+__global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_constant__ Mxfp8QuantParams p)
+{
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = p.rows * p.segs_per_row;
+    // whole warps stay in the shuffle below: total is a multiple of 2 and lanes pair as (even, odd)
+    const bool active = gid < total;
+    const int64_t i = active ? gid / p.segs_per_row : 0;
+    const int64_t seg = active ? gid % p.segs_per_row : 0;
+    const int64_t j0 = seg * 16;
+
+    uint32_t raw[8];
+#pragma unroll
+    for (int k = 0; k < 8; k++) raw[k] = 0u;
+    if (active && j0 < p.cols) {
+        const uint16_t *src = p.x + i * p.ld_x + j0;
+        if (p.x_vec_ok && j0 + 16 <= p.cols) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
+            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
+            raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
+            raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
+                const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
+                raw[k] = lo | (hi << 16);
+            }
+        }
+    }
+
+    // block maximum over finite magnitudes (BF16 magnitudes order like unsigned integers)
+    uint32_t fm = 0;
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
+        if (lo < 0x7F80u && lo > fm) fm = lo;
+        if (hi < 0x7F80u && hi > fm) fm = hi;
+    }
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, 1);
+    fm = other > fm ? other : fm;
+
+    // smallest e with 448*2^e >= M: code = be - 8 + (m7 > 0x60), clamped at 0
+    const int be = (int)(fm >> 7), m7 = (int)(fm & 0x7F);
+    int code = be == 0 ? 0 : be - 8 + (m7 > 0x60 ? 1 : 0);
+    code = code < 0 ? 0 : code;
+    const float inv = __uint_as_float((uint32_t)(254 - code) << 23);   // 2^(127-code) = 2^-e
+
+    if (!active) return;
+    if ((seg & 1) == 0) p.scale[i * p.ld_s + (seg >> 1)] = (uint8_t)code;
+
+    uint32_t out[4];
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        float v[4];
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            const uint32_t word = raw[2 * w + h];
+            const uint32_t lo = word << 16, hi = word & 0xFFFF0000u;
+            // NaN -> +0; +-Inf saturates to +-448 in the conversion
+            v[2 * h] = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv;
+            v[2 * h + 1] = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv;
+        }
+        out[w] = cvt_rn_e4m3x2(v[1], v[0]) | (cvt_rn_e4m3x2(v[3], v[2]) << 16);
+    }
+    *reinterpret_cast<uint4 *>(p.q + i * p.ld_q + j0) = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+}  // namespace fp4q
+
+using namespace fp4q;
+
+extern "C" fp4q_status fp4q_mxfp8_quantize1d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                             uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s,
+                                             void *stream)
+{
+    if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return FP4Q_OK;
+    if (!x_bf16 || !q || !scale) return FP4Q_ERR_NULL;
+    if (ld_x < cols || ld_q < round_up(cols, 32) || ld_s < ceil_div(cols, 32)) return FP4Q_ERR_SHAPE;
+    if (!aligned(x_bf16, 2) || !aligned(q, 16) || ld_q % 16 != 0) return FP4Q_ERR_ALIGN;
+
+    Mxfp8QuantParams p;
+    p.x = static_cast<const uint16_t *>(x_bf16);
+    p.rows = rows; p.cols = cols; p.ld_x = ld_x;
+    p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
+    p.segs_per_row = round_up(cols, 32) / 16;
+    p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
+    const int64_t total = rows * p.segs_per_row;
+    const int64_t n_cta = ceil_div(total, 256);
+    if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
+    mxfp8_quantize1d_kernel<<<(unsigned)n_cta, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}

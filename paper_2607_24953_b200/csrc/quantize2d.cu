@@ -1,0 +1,385 @@
+// fp4q_quantize2d: 2D-block (32x32) FP4 quantization with dual-layout pack, sm_100a.
+//
+// One pass over HBM: 2 B/element read, 0.5 + 0.5 B/element written, 1 B per 1024 elements of scale.
+// A CTA of 4 warps owns a 128x128 element block; a warp owns 32 rows x 128 columns (four 32x32
+// blocks side by side); 8 lanes own one 32x32 block, each lane 8 rows x 16 consecutive columns
+// (two 128-bit loads per row).  The block maximum is reduced with warp shuffles over those
+// 8 lanes, the E2M1 codes of a row segment are produced 2 at a time on packed fp16 lanes, the
+// row-major payload goes straight to global memory (8 B per lane and row, 64 B contiguous per
+// row and warp) and the transposed payload is built with an in-register 8x8 nibble transpose,
+// staged through 8 KB of shared memory and written as 64 B contiguous segments.
+//
+// Rounding works on the BF16 value scaled by 2^(-e-14) and converted (toward zero) to fp16: the
+// fp16 bit pattern of |x| 2^(-e-14) has the E2M1 magnitude code in bits 11..9 and the position
+// between the two neighbouring codes in bits 8..0, uniformly over normal and subnormal codes.
+// Adding 2*r8 (stochastic) or 0xFF + lsb (nearest-even) and taking bits 11..9 is the rounding.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace fp4q {
+
+struct PhiloxRoundKeys {
+    uint32_t k0[10], k1[10];   // key after r Weyl increments, r = 0..9
+};
+
+struct Quant2dParams {
+    const uint16_t *x;
+    int64_t rows, cols, ld_x;
+    uint8_t *q_rm;
+    int64_t ld_rm;
+    uint8_t *q_t;
+    int64_t ld_t;
+    uint8_t *scale;
+    int64_t ld_s;
+    int64_t grid_x;           // CTAs along the column direction
+    uint32_t tensor_id;
+    uint32_t flags;
+    int x_vec_ok;             // x 16-byte aligned and ld_x % 8 == 0: 128-bit loads are legal
+    int rng_aligned;          // cols % 16 == 0 and index not transposed: one Philox block per 16-element segment
+    PhiloxRoundKeys keys;
+};
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              const PhiloxRoundKeys &k, uint32_t out[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; r++) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__device__ __noinline__ uint32_t philox_byte(const Quant2dParams &p, uint64_t idx)
+{
+    uint32_t o[4];
+    const uint64_t blk = idx >> 4;
+    philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, o);
+    const uint32_t w = (idx >> 2) & 3;
+    const uint32_t word = w == 0 ? o[0] : w == 1 ? o[1] : w == 2 ? o[2] : o[3];
+    return (word >> (8 * (idx & 3))) & 0xFFu;
+}
+
+// {hi, lo} -> packed fp16x2, rounded toward zero (subnormal results are produced, not flushed).
+__device__ __forceinline__ uint32_t cvt_rz_f16x2(float hi, float lo)
+{
+    uint32_t d;
+    asm("cvt.rz.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// UE8M0 code of the truncation-free scale from the BF16 magnitude bits of the block maximum:
+// smallest e with 6*2^e >= M, code = e + 127, clamped below at 0.
+__device__ __forceinline__ int scale_code_from_max(uint32_t mbits)
+{
+    const int be = (int)(mbits >> 7), m7 = (int)(mbits & 0x7F);
+    if (be == 0) return 0;
+    const int c = be - 2 + (m7 > 0x40 ? 1 : 0);
+    return c < 0 ? 0 : c;
+}
+
+// 2^(-e-14) = 2^(113-code) as an FP32 (subnormal for code >= 240).
+__device__ __forceinline__ float inv_scale_f16_aligned(int code)
+{
+    const int e = 240 - code;
+    return __uint_as_float(e > 0 ? (uint32_t)e << 23 : 1u << (22 + e));
+}
+
+// One element, scalar: used for blocks that contain non-finite values.
+template <int MODE>
+__device__ __forceinline__ uint32_t quantize_scalar(uint32_t bits16, float inv, uint32_t r8)
+{
+    const uint32_t sign = (bits16 >> 15) & 1u, mag = bits16 & 0x7FFFu;
+    if (mag > 0x7F80u) return 0u;                 // NaN -> +0
+    if (mag == 0x7F80u) return (sign << 3) | 7u;  // +-Inf -> +-6
+    const float v = __uint_as_float(mag << 16) * inv;
+    const uint32_t h = cvt_rz_f16x2(0.0f, v) & 0xFFFFu;
+    const uint32_t b = MODE == FP4Q_ROUND_STOCHASTIC ? h + (r8 << 1) : h + 0xFFu + ((h >> 9) & 1u);
+    return (sign << 3) | (b >> 9);
+}
+
+// 16 consecutive elements of a row (raw[0..7], two BF16 per word) -> two words of 8 nibbles.
+// R[0..3]: the 16 random bytes of the segment, byte k for element k (unused for nearest).
+template <int MODE>
+__device__ __forceinline__ void round_segment(const uint32_t raw[8], float inv, const uint32_t R[4], uint32_t W[2])
+{
+#pragma unroll
+    for (int g = 0; g < 2; g++) {
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+            const uint32_t w = raw[4 * g + q];
+            v[2 * q] = __uint_as_float(w << 16) * inv;
+            v[2 * q + 1] = __uint_as_float(w & 0xFFFF0000u) * inv;
+        }
+        uint32_t acc = 0;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            // fp16 lanes: low = element 8g+j, high = element 8g+j+4 (nibbles j and j+4 are 16 bits apart)
+            const uint32_t h2 = cvt_rz_f16x2(v[j + 4], v[j]);
+            uint32_t b2;
+            if (MODE == FP4Q_ROUND_STOCHASTIC) {
+                const uint32_t sel = (uint32_t)j | ((uint32_t)j << 4) | ((uint32_t)(4 + j) << 8) | ((uint32_t)j << 12);
+                const uint32_t rm = __byte_perm(R[2 * g], R[2 * g + 1], sel) & 0x00FF00FFu;
+                b2 = h2 + (rm << 1);
+            } else {
+                b2 = h2 + 0x00FF00FFu + ((h2 >> 9) & 0x00010001u);
+            }
+            const uint32_t t = b2 | (b2 >> 3);   // sign (bit 15) next to the magnitude code (bits 11..9)
+            const uint32_t nib = (j < 3 ? t >> (9 - 4 * j) : t << 3) & (0x000F000Fu << (4 * j));
+            acc |= nib;
+        }
+        W[g] = acc;
+    }
+}
+
+// In-register transpose of an 8x8 matrix of nibbles: a[r] holds row r (nibble c = column c);
+// on return a[c] holds column c (nibble r = row r).
+__device__ __forceinline__ void transpose8x8_nibbles(uint32_t a[8])
+{
+#pragma unroll
+    for (int r = 0; r < 4; r++) {   // swap 4x4 quadrants (16-bit halves between rows r and r+4)
+        const uint32_t lo = __byte_perm(a[r], a[r + 4], 0x5410), hi = __byte_perm(a[r], a[r + 4], 0x7632);
+        a[r] = lo; a[r + 4] = hi;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; q++) {   // swap 2x2 blocks (bytes between rows r and r+2)
+        const int r = (q & 1) + 4 * (q >> 1);
+        const uint32_t lo = __byte_perm(a[r], a[r + 2], 0x6240), hi = __byte_perm(a[r], a[r + 2], 0x7351);
+        a[r] = lo; a[r + 2] = hi;
+    }
+#pragma unroll
+    for (int r = 0; r < 8; r += 2) {  // swap single nibbles between rows r and r+1
+        const uint32_t lo = (a[r] & 0x0F0F0F0Fu) | ((a[r + 1] & 0x0F0F0F0Fu) << 4);
+        const uint32_t hi = ((a[r] >> 4) & 0x0F0F0F0Fu) | (a[r + 1] & 0xF0F0F0F0u);
+        a[r] = lo; a[r + 1] = hi;
+    }
+}
+
+__device__ __forceinline__ void load_segment(const Quant2dParams &p, int64_t i, int64_t j0, uint32_t out[8])
+{
+    if (i >= p.rows || j0 >= p.cols) {
+#pragma unroll
+        for (int k = 0; k < 8; k++) out[k] = 0u;
+        return;
+    }
+    const uint16_t *src = p.x + i * p.ld_x + j0;
+    if (p.x_vec_ok && j0 + 16 <= p.cols) {
+        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
+        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
+            const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
+            out[k] = lo | (hi << 16);
+        }
+    }
+}
+
+// The 16 random bytes of the row segment starting at element (i, j0).
+__device__ __forceinline__ void segment_random_bytes(const Quant2dParams &p, int64_t i, int64_t j0, uint32_t R[4])
+{
+    if (p.rng_aligned) {
+        const uint64_t blk = ((uint64_t)i * (uint64_t)p.cols + (uint64_t)j0) >> 4;
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, R);
+        return;
+    }
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        uint32_t word = 0;
+#pragma unroll 1
+        for (int b = 0; b < 4; b++) {
+            const int64_t j = j0 + 4 * w + b;
+            if (j < p.cols) {
+                const uint64_t idx = (p.flags & FP4Q_INDEX_TRANSPOSED)
+                                         ? (uint64_t)j * (uint64_t)p.rows + (uint64_t)i
+                                         : (uint64_t)i * (uint64_t)p.cols + (uint64_t)j;
+                word |= philox_byte(p, idx) << (8 * b);
+            }
+        }
+        R[w] = word;
+    }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(128) quantize2d_kernel(const __grid_constant__ Quant2dParams p)
+{
+    __shared__ uint4 qt_stage[128 * 4];   // 128 transposed rows x 64 B (four 16-byte chunks, XOR-swizzled)
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = lane >> 3;          // which of the warp's four 32x32 blocks
+    const int rg = (lane >> 1) & 3;   // group of 8 rows inside the block
+    const int ch = lane & 1;          // 16-column half of the block
+    const int64_t bx = (int64_t)blockIdx.x % p.grid_x, by = (int64_t)blockIdx.x / p.grid_x;
+    const int64_t tile_row0 = by * 128 + warp * 32, tile_col0 = bx * 128 + t * 32;
+    const int64_t row0 = tile_row0 + rg * 8, col0 = tile_col0 + ch * 16;
+    const bool tile_exists = tile_row0 < p.rows && tile_col0 < p.cols;
+
+    uint32_t raw[8][8];
+#pragma unroll
+    for (int r = 0; r < 8; r++) load_segment(p, row0 + r, col0, raw[r]);
+
+    // block maximum: packed BF16 |.| max with NaN propagation, so that any non-finite entry shows
+    // up in the result and routes the block to the scalar path
+    __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
+#pragma unroll
+    for (int r = 0; r < 8; r++)
+#pragma unroll
+        for (int k = 0; k < 8; k++)
+            m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r][k])));
+#pragma unroll
+    for (int s = 1; s <= 4; s <<= 1) {
+        uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), s);
+        m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
+    }
+    const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
+    uint32_t mbits = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
+
+    const bool nonfinite = mbits >= 0x7F80u;
+    if (__any_sync(0xFFFFFFFFu, nonfinite)) {
+        // maximum over the finite entries only
+        uint32_t fm = 0;
+#pragma unroll
+        for (int r = 0; r < 8; r++)
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint32_t lo = raw[r][k] & 0x7FFFu, hi = (raw[r][k] >> 16) & 0x7FFFu;
+                if (lo < 0x7F80u && lo > fm) fm = lo;
+                if (hi < 0x7F80u && hi > fm) fm = hi;
+            }
+#pragma unroll
+        for (int s = 1; s <= 4; s <<= 1) {
+            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, s);
+            fm = other > fm ? other : fm;
+        }
+        if (nonfinite) mbits = fm;
+    }
+
+    const int code = scale_code_from_max(mbits);
+    const float inv = inv_scale_f16_aligned(code);
+    if (tile_exists && (lane & 7) == 0)
+        p.scale[(tile_row0 >> 5) * p.ld_s + (tile_col0 >> 5)] = (uint8_t)code;
+
+    uint32_t W[8][2];
+#pragma unroll
+    for (int r = 0; r < 8; r++) {
+        const int64_t i = row0 + r;
+        if (!tile_exists || i >= p.rows) {
+            W[r][0] = W[r][1] = 0u;
+            continue;
+        }
+        uint32_t R[4] = {0u, 0u, 0u, 0u};
+        if (MODE == FP4Q_ROUND_STOCHASTIC) segment_random_bytes(p, i, col0, R);
+        if (!nonfinite) {
+            round_segment<MODE>(raw[r], inv, R, W[r]);
+        } else {
+#pragma unroll
+            for (int g = 0; g < 2; g++) {
+                uint32_t acc = 0;
+#pragma unroll
+                for (int e = 0; e < 8; e++) {
+                    const int k = 8 * g + e;
+                    const uint32_t bits = (raw[r][k >> 1] >> (16 * (k & 1))) & 0xFFFFu;
+                    const uint32_t r8 = (R[k >> 2] >> (8 * (k & 3))) & 0xFFu;
+                    acc |= quantize_scalar<MODE>(bits, inv, r8) << (4 * e);
+                }
+                W[r][g] = acc;
+            }
+        }
+        *reinterpret_cast<uint2 *>(p.q_rm + i * p.ld_rm + (col0 >> 1)) = make_uint2(W[r][0], W[r][1]);
+    }
+
+    if (p.q_t == nullptr) return;
+
+    // transposed payload: per lane two 8x8 nibble blocks -> 16 words (one per column, 8 rows each)
+    uint32_t *stage = reinterpret_cast<uint32_t *>(qt_stage);
+#pragma unroll
+    for (int g = 0; g < 2; g++) {
+        uint32_t a[8];
+#pragma unroll
+        for (int r = 0; r < 8; r++) a[r] = W[r][g];
+        transpose8x8_nibbles(a);
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+            const int col_local = 32 * t + 16 * ch + 8 * g + c;
+            // word index inside the 64-byte row: 4*(source warp) + rg, with the 16-byte chunk index
+            // XORed by the column's block index so that a warp's stores spread over the banks
+            stage[col_local * 16 + (((warp ^ t) << 2) | rg)] = a[c];
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const int row_local = (threadIdx.x >> 2) + 32 * k;   // transposed row = source column; its block index is k
+        const int chunk = threadIdx.x & 3;                    // 32 source rows = one source warp
+        const int64_t col = bx * 128 + row_local;
+        if (col < p.cols && by * 128 + chunk * 32 < p.rows) {
+            const uint4 v = qt_stage[row_local * 4 + (chunk ^ k)];
+            *reinterpret_cast<uint4 *>(p.q_t + col * p.ld_t + by * 64 + chunk * 16) = v;
+        }
+    }
+}
+
+static void philox_round_keys(uint64_t seed, PhiloxRoundKeys &k)
+{
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; r++) {
+        k.k0[r] = k0;
+        k.k1[r] = k1;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+}
+
+}  // namespace fp4q
+
+using namespace fp4q;
+
+extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                       const fp4q_tensor *out, fp4q_round mode, uint64_t seed,
+                                       uint32_t tensor_id, uint32_t flags, void *stream)
+{
+    if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
+    if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
+    if (flags & ~FP4Q_INDEX_TRANSPOSED) return FP4Q_ERR_UNSUPPORTED;
+    if (!out) return FP4Q_ERR_NULL;
+    if (out->rows != rows || out->cols != cols) return FP4Q_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return FP4Q_OK;
+    if (!x_bf16 || !out->q_rm || !out->scale) return FP4Q_ERR_NULL;
+    if (ld_x < cols || out->ld_rm < round_up(cols, 32) / 2 || out->ld_s < ceil_div(cols, 32)) return FP4Q_ERR_SHAPE;
+    if (out->q_t && out->ld_t < round_up(rows, 32) / 2) return FP4Q_ERR_SHAPE;
+    if (!aligned(x_bf16, 2) || !aligned(out->q_rm, 16) || out->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
+    if (out->q_t && (!aligned(out->q_t, 16) || out->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
+
+    Quant2dParams p;
+    p.x = static_cast<const uint16_t *>(x_bf16);
+    p.rows = rows; p.cols = cols; p.ld_x = ld_x;
+    p.q_rm = out->q_rm; p.ld_rm = out->ld_rm;
+    p.q_t = out->q_t; p.ld_t = out->ld_t;
+    p.scale = out->scale; p.ld_s = out->ld_s;
+    p.grid_x = ceil_div(cols, 128);
+    p.tensor_id = tensor_id;
+    p.flags = flags;
+    p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
+    p.rng_aligned = cols % 16 == 0 && !(flags & FP4Q_INDEX_TRANSPOSED);
+    philox_round_keys(seed, p.keys);
+
+    const int64_t n_cta = p.grid_x * ceil_div(rows, 128);
+    if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (mode == FP4Q_ROUND_STOCHASTIC)
+        quantize2d_kernel<FP4Q_ROUND_STOCHASTIC><<<(unsigned)n_cta, 128, 0, s>>>(p);
+    else
+        quantize2d_kernel<FP4Q_ROUND_NEAREST><<<(unsigned)n_cta, 128, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
