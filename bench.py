@@ -1,0 +1,507 @@
+#!/usr/bin/env python
+"""Benchmark of the fp4q hot path on B200.
+
+One step = one pass of the whole path over one batch of seeded synthetic tensors of the 7B-class dense
+layer configuration (hidden 4096, FFN 11008, 16384 tokens): the 2D-block FP4 quantize + dual-layout pack
+of every operand (7 weights, 4 distinct activations, 7 output gradients, stochastic rounding) followed by
+the forward, dgrad and wgrad block-scaled FP4 GEMMs of the 7 linear layers.  The headline value is the
+quantize+dual-pack throughput in GB/s (3.001 algorithmic bytes per element); the GEMM TFLOP/s per product
+are reported beside it, and the MXFP8 query/key projections and the grouped MoE expert layer are timed
+separately under "extras".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the CPU oracle is timed instead, on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+BYTES_PER_ELEMENT = 2.0 + 0.5 + 0.5 + 1.0 / 1024.0   # BF16 read, two packed layouts, one scale byte per 32x32 block
+METRIC = "2D-FP4 quantize+dual-pack GB/s; block-scaled FP4 GEMM TFLOPS (fwd/dgrad/wgrad)"
+FP4_OVER_BF16 = 4.0      # nominal dense tensor-core ratio (9 PFLOP/s FP4 : 2.25 PFLOP/s BF16)
+FP8_OVER_BF16 = 2.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (reads only)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: str):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="fp4q_clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    t = [x.strip() for x in line.split(",")]
+                    if len(t) < 8:
+                        continue
+                    try:
+                        sm.append(float(t[0]))
+                        smax.append(float(t[1]))
+                    except ValueError:
+                        continue
+                    for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), t[4:8]):
+                        if v.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ multi-rank
+
+def max_over_ranks(values, dist, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (replicas are timed by the slowest one)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.cpu().tolist()
+
+
+def aggregate_throughput(units_per_rank, world, ms):
+    """Whole-job throughput of `world` replicas that each processed units_per_rank in ms (max over ranks)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
+# ------------------------------------------------------------------------------------------ workload
+
+def build_dense_workload(cfg, device, torch, workloads):
+    """All BF16 operands of one dense layer set: per layer W [N,K], X [T,K] (shared between layers with the
+    same input), dY [T,N]."""
+    T = cfg.tokens
+    layers = cfg.layers()
+    x_of = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "gate": "mlp_in", "up": "mlp_in", "down": "down_in"}
+    xs, ops = {}, []
+    for i, (name, n, k) in enumerate(layers):
+        key = x_of[name]
+        if key not in xs:
+            xs[key] = workloads.activations_student_t(T, k, cfg.data_seed + 10 * i + 1, device, nu=cfg.nu)
+        ops.append({"name": name, "N": n, "K": k, "W": workloads.weights(n, k, cfg.data_seed + 10 * i, device),
+                    "X": xs[key], "x_key": key, "dY": workloads.gradients_rowscaled(T, n, cfg.data_seed + 10 * i + 2, device)})
+    return ops, xs
+
+
+def run_gpu(args):
+    import torch
+    from paper_2607_24953_b200 import binding, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    binding.lib()   # fail loudly if the CUDA library is missing
+
+    cfg = {"7b": workloads.CONFIG_7B, "1b": workloads.CONFIG_1B, "tiny": workloads.CONFIG_TINY}[args.workload]
+    T = cfg.tokens
+    ops, xs = build_dense_workload(cfg, dev, torch, workloads)
+    seed = cfg.philox_seed
+    SR = binding.ROUND_STOCHASTIC
+
+    # quantize targets: 7 W, the distinct X, 7 dY -- preallocated outputs
+    q_w = [binding.alloc_qtensor(o["N"], o["K"], dev) for o in ops]
+    q_x = {k: binding.alloc_qtensor(T, v.shape[1], dev) for k, v in xs.items()}
+    q_dy = [binding.alloc_qtensor(T, o["N"], dev) for o in ops]
+    quant_jobs = [(o["W"], q_w[i], 10 * i) for i, o in enumerate(ops)]
+    quant_jobs += [(xs[k], q_x[k], 100 + j) for j, k in enumerate(xs)]
+    quant_jobs += [(o["dY"], q_dy[i], 10 * i + 2) for i, o in enumerate(ops)]
+    quant_elems = sum(t.numel() for t, _, _ in quant_jobs)
+    quant_bytes = quant_elems * BYTES_PER_ELEMENT
+
+    max_n, max_k = max(o["N"] for o in ops), max(o["K"] for o in ops)
+    y_buf = torch.empty((T, max_n), dtype=torch.bfloat16, device=dev)
+    dx_buf = torch.empty((T, max_k), dtype=torch.bfloat16, device=dev)
+    dw_buf = torch.empty((max(o["N"] * o["K"] for o in ops),), dtype=torch.float32, device=dev)
+    ws = binding.alloc_workspace(dev)
+    gemm_flops = sum(2.0 * T * o["N"] * o["K"] for o in ops)
+
+    def outputs(o):
+        return (y_buf[:, :o["N"]], dx_buf[:, :o["K"]], dw_buf[:o["N"] * o["K"]].view(o["N"], o["K"]))
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        if marks: marks[0].record()
+        for x, q, tid in quant_jobs:
+            binding.fp4q_quantize2d(x, q, mode=SR, seed=seed, tensor_id=tid)
+        if marks: marks[1].record()
+        for i, o in enumerate(ops):
+            binding.fp4q_gemm_fwd(q_x[o["x_key"]], q_w[i], out=outputs(o)[0], dt=binding.OUT_BF16, ws=ws)
+        if marks: marks[2].record()
+        for i, o in enumerate(ops):
+            binding.fp4q_gemm_dgrad(q_dy[i], q_w[i], out=outputs(o)[1], dt=binding.OUT_BF16, ws=ws)
+        if marks: marks[3].record()
+        for i, o in enumerate(ops):
+            binding.fp4q_gemm_wgrad(q_dy[i], q_x[o["x_key"]], out=outputs(o)[2], dt=binding.OUT_F32, ws=ws)
+        if marks: marks[4].record()
+
+    launches_per_step = len(quant_jobs) + 3 * len(ops)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    if binding.fp4q_workspace_status(ws) != 0:
+        raise RuntimeError("a GEMM kernel reported a device-side timeout during warm-up")
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    sampler.start()
+    barrier()
+    t0, t1 = ev(), ev()
+    t0.record()
+    for s in range(args.steps):
+        step(marks[s])
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t0.elapsed_time(t1)
+    status = binding.fp4q_workspace_status(ws)
+    if status != 0:
+        raise RuntimeError("a GEMM kernel reported a device-side timeout: status %d" % status)
+
+    phase_ms = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(4)] for m in marks])   # quant, fwd, dgrad, wgrad
+    red = max_over_ranks([total_ms] + phase_ms.sum(0).tolist(), dist, dev)
+    total_ms, phase_tot = red[0], np.array(red[1:])
+    ms_per_step = total_ms / args.steps
+    q_ms, f_ms, d_ms, w_ms = (phase_tot / args.steps).tolist()
+    quant_gbs = aggregate_throughput(quant_bytes, world, q_ms) / 1e9
+    tf = lambda ms: aggregate_throughput(gemm_flops, world, ms) / 1e12
+    gemm_tflops = {"fwd": tf(f_ms), "dgrad": tf(d_ms), "wgrad": tf(w_ms),
+                   "all": aggregate_throughput(3 * gemm_flops, world, f_ms + d_ms + w_ms) / 1e12}
+
+    # ---- end to end: pinned host inputs -> device, quantize + GEMMs, results -> pinned host
+    e2e = None
+    if not args.no_e2e:
+        host_in = []
+        for x, _, _ in quant_jobs:
+            h = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+            h.copy_(x)
+            host_in.append(h)
+        host_out = [[torch.empty(b.shape, dtype=b.dtype, pin_memory=True) for b in outputs(o)] for o in ops]
+        h2d = sum(h.numel() * h.element_size() for h in host_in)
+        d2h = sum(b.numel() * b.element_size() for bs in host_out for b in bs)
+
+        def e2e_step():
+            for (x, q, tid), h in zip(quant_jobs, host_in):
+                x.copy_(h, non_blocking=True)
+                binding.fp4q_quantize2d(x, q, mode=SR, seed=seed, tensor_id=tid)
+            for i, o in enumerate(ops):
+                y, dx, dw = outputs(o)
+                binding.fp4q_gemm_fwd(q_x[o["x_key"]], q_w[i], out=y, dt=binding.OUT_BF16, ws=ws)
+                host_out[i][0].copy_(y, non_blocking=True)
+                binding.fp4q_gemm_dgrad(q_dy[i], q_w[i], out=dx, dt=binding.OUT_BF16, ws=ws)
+                host_out[i][1].copy_(dx, non_blocking=True)
+                binding.fp4q_gemm_wgrad(q_dy[i], q_x[o["x_key"]], out=dw, dt=binding.OUT_F32, ws=ws)
+                host_out[i][2].copy_(dw, non_blocking=True)
+
+        e2e_steps = max(1, min(args.steps, 3))
+        e2e_step()
+        barrier()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b) / e2e_steps
+        e_ms = max_over_ranks([e_ms], dist, dev)[0]
+        # same metric: quantize+dual-pack algorithmic bytes over the end-to-end step time
+        e2e = {"value": aggregate_throughput(quant_bytes, world, e_ms) / 1e9, "unit": "GB/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "note": "whole step (H2D of all BF16 operands, quantize sweep, 21 GEMMs, D2H of all outputs); "
+                       "PCIe-bound"}
+        del host_in, host_out
+
+    extras = {}
+    if not args.no_extras:
+        extras = run_extras(torch, binding, workloads, dev, ws)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    gemm_ms_per_launch = (f_ms + d_ms + w_ms) / (3 * len(ops))
+    achieved_tf = 3 * gemm_flops / ((f_ms + d_ms + w_ms) * 1e-3) / 1e12
+    roofline = {"kernel": "gemm_block_scaled_kernel<mxf4>", "bound": "tensor", "achieved": achieved_tf, "peak": fp4_peak,
+                "unit": "TFLOP/s", "frac": achieved_tf / fp4_peak, "traffic": None,
+                "peak_source": "%s bf16 sustained %.1f TFLOP/s x %.0f (nominal FP4:BF16 ratio)" %
+                               (peaks["source"], peaks["bf16_tflops_sustained"], FP4_OVER_BF16),
+                "flops_per_launch": 3 * gemm_flops / (3 * len(ops)), "ms_per_launch": gemm_ms_per_launch,
+                "time_share_of_step": (f_ms + d_ms + w_ms) / ms_per_step}
+    q_gbs_1 = quant_bytes / (q_ms * 1e-3) / 1e9
+    roofline_quantize = {"kernel": "quantize2d_kernel<stochastic>", "bound": "hbm", "achieved": q_gbs_1,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": q_gbs_1 / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": peaks["source"] + " copy bandwidth",
+                         "bytes_per_launch": quant_bytes / len(quant_jobs), "ms_per_launch": q_ms / len(quant_jobs),
+                         "time_share_of_step": q_ms / ms_per_step}
+    fill_traffic(roofline, roofline_quantize)
+
+    cpu = cpu_baseline_quantize(workloads, cfg, seconds=args.cpu_seconds)
+
+    line = {
+        "metric": METRIC, "value": quant_gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp4-e2m1 (bf16 in, fp32 accumulate)", "data": "synthetic",
+        "config": {"workload": cfg.name + ": hidden %d, FFN %d, %d tokens; quantize sweep over 7 W + %d X + 7 dY "
+                               "(stochastic rounding) then fwd/dgrad/wgrad FP4 GEMMs of 7 linear layers" %
+                               (cfg.hidden, cfg.ffn, cfg.tokens, len(xs)),
+                   "parallelism": "replicas only (x%d)" % world, "l2": "inputs larger than L2 (%.2f GB of BF16 operands per step)" %
+                   (quant_elems * 2 / 1e9), "quantize_bytes_per_step": quant_bytes, "gemm_flops_per_step": 3 * gemm_flops},
+        "gemm_tflops": gemm_tflops,
+        "phase_ms": {"quantize": q_ms, "fwd": f_ms, "dgrad": d_ms, "wgrad": w_ms},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "roofline_quantize": roofline_quantize, "cpu_baseline": cpu, "extras": extras,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def fill_traffic(roofline, roofline_quantize):
+    """DRAM traffic per launch from the committed ncu summaries (profiles/traffic.json), if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return
+    try:
+        with open(path) as f:
+            t = json.load(f)
+        # captured on a smaller case and scaled by the units processed (traffic grows in proportion)
+        if "gemm_bytes_per_flop" in t:
+            roofline["traffic"] = t["gemm_bytes_per_flop"] * roofline["flops_per_launch"]
+        if "quantize_dram_bytes_per_algorithmic_byte" in t:
+            roofline_quantize["traffic"] = t["quantize_dram_bytes_per_algorithmic_byte"] * roofline_quantize["bytes_per_launch"]
+    except Exception:
+        pass
+
+
+def run_extras(torch, binding, workloads, dev, ws):
+    """MXFP8 query/key projections at 7B shapes and the grouped MoE expert layer, timed on their own."""
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, iters=5):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters
+
+    # --- MXFP8 Q/K projections: X 16384x4096, Wq, Wk 4096x4096
+    cfg = workloads.CONFIG_ATTN_7B
+    T, H = cfg.tokens, cfg.hidden
+    X = workloads.activations_student_t(T, H, cfg.data_seed + 1, dev, nu=cfg.nu)
+    Wq, Wk = workloads.weights(H, H, cfg.data_seed, dev), workloads.weights(H, H, cfg.data_seed + 10, dev)
+    xq, xs = binding.fp4q_mxfp8_quantize1d(X)
+    wqq, wqs = binding.fp4q_mxfp8_quantize1d(Wq)
+    wkq, wks = binding.fp4q_mxfp8_quantize1d(Wk)
+    ms_q = timed(lambda: binding.fp4q_mxfp8_quantize1d(X))
+    ms_g = timed(lambda: binding.fp4q_mxfp8_qk(xq, xs, wqq, wqs, wkq, wks, T, H, H, ws=ws))
+    out["mxfp8_qk"] = {"workload": "Q and K projections, %d tokens, %dx%d each" % (T, H, H),
+                       "quantize_gbs": T * H * (3.0 + 1 / 32) / (ms_q * 1e-3) / 1e9,
+                       "gemm_tflops": 2 * 2.0 * T * H * H / (ms_g * 1e-3) / 1e12, "gemm_ms": ms_g}
+    del X, Wq, Wk, xq, xs, wqq, wqs, wkq, wks
+
+    # --- grouped MoE expert layer: 128 experts, hidden 2048, expert FFN 768, top-8 of 16384 tokens
+    moe = workloads.CONFIG_MOE
+    counts = workloads.moe_routing(moe)
+    offs = workloads.padded_row_offsets(counts, moe.pad)
+    Tp = int(offs[-1])
+    d_offs = torch.from_numpy(offs).to(dev)
+    E, H, F = moe.experts, moe.hidden, moe.expert_ffn
+    res = {"workload": "%d experts, hidden %d, expert FFN %d, %d routed rows padded to %d; loads max %d / median %d / min %d" %
+                       (E, H, F, int(counts.sum()), Tp, int(counts.max()), int(np.median(counts)), int(counts.min()))}
+    tot_ms, tot_flops = 0.0, 0.0
+    for name, n, k in moe.layers():
+        Xm = workloads.zero_padding_rows(workloads.activations_student_t(Tp, k, moe.data_seed + 1, dev), counts, offs)
+        dYm = workloads.zero_padding_rows(workloads.gradients_rowscaled(Tp, n, moe.data_seed + 2, dev), counts, offs)
+        Wm = workloads.weights(E * n, k, moe.data_seed, dev)
+        qx, qw, qdy = (binding.fp4q_quantize2d(t, mode=1, seed=moe.philox_seed, tensor_id=i) for i, t in enumerate((Xm, Wm, dYm)))
+        y = torch.empty((Tp, n), dtype=torch.bfloat16, device=dev)
+        dx = torch.empty((Tp, k), dtype=torch.bfloat16, device=dev)
+        dw = torch.empty((E * n, k), dtype=torch.float32, device=dev)
+        flops = 2.0 * float(counts.sum()) * n * k
+        ms = [timed(lambda: binding.fp4q_gemm_fwd(qx, qw, out=y, row_offsets=d_offs, ws=ws)),
+              timed(lambda: binding.fp4q_gemm_dgrad(qdy, qw, out=dx, row_offsets=d_offs, ws=ws)),
+              timed(lambda: binding.fp4q_gemm_wgrad(qdy, qx, out=dw, row_offsets=d_offs, ws=ws))]
+        res[name] = {"fwd_tflops": flops / (ms[0] * 1e-3) / 1e12, "dgrad_tflops": flops / (ms[1] * 1e-3) / 1e12,
+                     "wgrad_tflops": flops / (ms[2] * 1e-3) / 1e12, "ms": ms,
+                     "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9}
+        tot_ms += sum(ms)
+        tot_flops += 3 * flops
+        del Xm, dYm, Wm, qx, qw, qdy, y, dx, dw
+    res["all_tflops"] = tot_flops / (tot_ms * 1e-3) / 1e12
+    out["moe_grouped"] = res
+    if binding.fp4q_workspace_status(ws) != 0:
+        out["status"] = "device-side timeout reported"
+    return out
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+
+def cpu_baseline_quantize(workloads, cfg, seconds=12.0):
+    """The oracle quantizer, as it stands, timed on the host cores on a bounded row slab of the largest
+    activation (stochastic rounding, same seed)."""
+    import oracle
+    cols = cfg.ffn
+    probe_rows = 64
+    x = workloads.bf16_bits(workloads.activations_student_t(probe_rows, cols, cfg.data_seed + 61, "cpu", nu=cfg.nu))
+    t0 = time.perf_counter()
+    oracle.quantize2d(x, oracle.MODE_STOCHASTIC, seed=cfg.philox_seed, tensor_id=7)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    rows = int(min(cfg.tokens, max(probe_rows, (seconds / dt) * probe_rows // 32 * 32)))
+    x = workloads.bf16_bits(workloads.activations_student_t(rows, cols, cfg.data_seed + 61, "cpu", nu=cfg.nu))
+    t0 = time.perf_counter()
+    oracle.quantize2d(x, oracle.MODE_STOCHASTIC, seed=cfg.philox_seed, tensor_id=7)
+    dt = time.perf_counter() - t0
+    return {"value": rows * cols * BYTES_PER_ELEMENT / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": dt,
+            "sample": "quantize+dual-pack (stochastic) of a %dx%d row slab of the %dx%d down-projection activation" %
+                      (rows, cols, cfg.tokens, cols)}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores; each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2607_24953_b200 import workloads
+    cfg = {"7b": workloads.CONFIG_7B, "1b": workloads.CONFIG_1B, "tiny": workloads.CONFIG_TINY}[args.workload]
+    rows = 256
+    tensors = [workloads.bf16_bits(workloads.weights(rows, cfg.hidden, cfg.data_seed, "cpu")),
+               workloads.bf16_bits(workloads.activations_student_t(rows, cfg.ffn, cfg.data_seed + 61, "cpu", nu=cfg.nu)),
+               workloads.bf16_bits(workloads.gradients_rowscaled(rows, cfg.hidden, cfg.data_seed + 2, "cpu"))]
+    elems = sum(t.size for t in tensors)
+    n_tok, n_out, k = 32, 512, cfg.hidden
+
+    def step():
+        qs = [oracle.quantize2d(t, oracle.MODE_STOCHASTIC, seed=cfg.philox_seed, tensor_id=i) for i, t in enumerate(tensors)]
+        wd = oracle.dequantize2d(qs[0][0], qs[0][2], rows, cfg.hidden)
+        xd = oracle.dequantize2d(qs[2][0], qs[2][2], rows, cfg.hidden)
+        t0 = time.perf_counter()
+        oracle.gemm_fwd(xd[:n_tok], wd[:n_out])
+        oracle.gemm_dgrad(xd[:n_tok, :rows], wd)
+        oracle.gemm_wgrad(xd[:n_tok, :rows], xd[:n_tok])
+        return time.perf_counter() - t0
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    gemm_s = 0.0
+    for _ in range(args.steps):
+        gemm_s += step()
+    total = time.perf_counter() - t0
+    quant_s = total - gemm_s
+    value = args.steps * elems * BYTES_PER_ELEMENT / quant_s / 1e9
+    gemm_flops = 2.0 * n_tok * (n_out * k + rows * cfg.hidden + rows * cfg.hidden)
+    sample = ("per step: oracle quantize+dual-pack (stochastic) of %d-row slabs of a weight, the down-projection "
+              "activation and an output gradient (%d elements), then the three float64 products on %d sampled rows" %
+              (rows, elems, n_tok))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name + " (bounded sample)", "parallelism": "host cores"},
+            "gemm_tflops": {"all": args.steps * gemm_flops / max(gemm_s, 1e-9) / 1e12},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="fp4q", choices=["fp4q", "reference"])
+    ap.add_argument("--workload", default="7b", choices=["7b", "1b", "tiny"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

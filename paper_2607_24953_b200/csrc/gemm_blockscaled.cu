@@ -218,20 +218,53 @@ __device__ __forceinline__ uint8_t load_scale(const ScaleView &v, int row, int k
     return (row < v.n_row && kb < v.n_kb) ? __ldg(v.ptr + (int64_t)row * v.stride_row + (int64_t)kb * v.stride_kb) : kScalePad;
 }
 
+// The scale loader runs ahead of the ring: the compact scale bytes of a stage are fetched into registers
+// kStages iterations before its image is written, so that the global-memory latency is off the critical path.
+struct WorkIter {
+    int tile, it, n_it;
+    Tile t;
+    __device__ __forceinline__ void seek(const GemmParams &p, int stage_elems)
+    {
+        while (tile < p.n_tile_total) {
+            decode_tile(p, tile, t);
+            n_it = (t.k_len + stage_elems - 1) / stage_elems;
+            if (n_it > 0) { it = 0; return; }
+            tile += gridDim.x;
+        }
+        n_it = 0;
+    }
+    __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
+    __device__ __forceinline__ void next(const GemmParams &p, int stage_elems)
+    {
+        if (++it >= n_it) { tile += gridDim.x; seek(p, stage_elems); }
+    }
+};
+
 // mxf4 / 2D blocks: a stage covers 8 contraction blocks (two chunks of 4).  For 128 operand rows and one chunk
-// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3].
-__device__ __forceinline__ void build_scale_images_2d(const GemmParams &p, const Tile &t, int it, uint8_t *sf_stage,
-                                                      uint8_t *scratch, int lane)
+// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3].  Per stage a lane fetches one byte of
+// A's 2 x 4 x 4 and two bytes of B's 2 x 8 x 4 compact scale bytes.
+struct ScaleRegs2D { uint32_t a, b0, b1; };
+
+__device__ __forceinline__ ScaleRegs2D fetch_scales_2d(const GemmParams &p, const Tile &t, int it, int lane)
 {
-    {   // A: 2 chunks x 4 row tiles x 4 blocks = 32 bytes, one per lane
+    ScaleRegs2D r;
+    {
         const int c = lane >> 4, rt = (lane >> 2) & 3, kb = lane & 3;
-        scratch[lane] = load_scale(p.sfa, (t.a_row0 >> 5) + rt, (t.a_k0 >> 5) + it * 8 + c * 4 + kb);
+        r.a = load_scale(p.sfa, (t.a_row0 >> 5) + rt, (t.a_k0 >> 5) + it * 8 + c * 4 + kb);
     }
-#pragma unroll
-    for (int h = 0; h < 2; h++) {   // B: 2 chunks x 8 row tiles x 4 blocks = 64 bytes, two per lane
-        const int idx = lane + 32 * h, c = idx >> 5, rt = (idx >> 2) & 7, kb = idx & 3;
-        scratch[32 + idx] = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + c * 4 + kb);
+    {
+        const int c = lane >> 5, rt = (lane >> 2) & 7, kb = lane & 3;   // idx = lane: chunk 0
+        r.b0 = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + c * 4 + kb);
+        r.b1 = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + 4 + kb);   // idx = lane + 32: chunk 1
     }
+    return r;
+}
+
+__device__ __forceinline__ void write_scale_images_2d(const ScaleRegs2D &r, uint8_t *sf_stage, uint8_t *scratch, int lane)
+{
+    scratch[lane] = (uint8_t)r.a;            // [chunk][row tile 0..3][block]
+    scratch[32 + lane] = (uint8_t)r.b0;      // chunk 0: [row tile 0..7][block]
+    scratch[64 + lane] = (uint8_t)r.b1;      // chunk 1
     __syncwarp();
     const uint4 *s4 = reinterpret_cast<const uint4 *>(scratch);
     uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
@@ -244,28 +277,62 @@ __device__ __forceinline__ void build_scale_images_2d(const GemmParams &p, const
     __syncwarp();
 }
 
-// mxf8 / 1D blocks: a stage covers 4 contraction blocks (one chunk); image row l holds rows l, l+32, l+64, l+96.
-__device__ __forceinline__ void build_scale_images_1d(const GemmParams &p, const Tile &t, int it, uint8_t *sf_stage, int lane)
+// mxf8 / 1D blocks: a stage covers 4 contraction blocks (one chunk); image row l holds rows l, l+32, l+64, l+96,
+// four scale bytes each.
+struct ScaleRegs1D { uint32_t w[3][4]; };
+
+__device__ __forceinline__ uint32_t load_scale_word(const ScaleView &v, int row, int kb0)
 {
-    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
+    const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
+    if (row < v.n_row && kb0 + 4 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 3) == 0)
+        return __ldg(reinterpret_cast<const uint32_t *>(ptr));
+    uint32_t word = 0;
+#pragma unroll
+    for (int kb = 0; kb < 4; kb++) word |= (uint32_t)load_scale(v, row, kb0 + kb) << (8 * kb);
+    return word;
+}
+
+__device__ __forceinline__ ScaleRegs1D fetch_scales_1d(const GemmParams &p, const Tile &t, int it, int lane)
+{
+    ScaleRegs1D r;
 #pragma unroll
     for (int blk = 0; blk < 3; blk++) {   // 0: A rows 0..127; 1, 2: B rows 0..127, 128..255
         const ScaleView &v = blk == 0 ? p.sfa : p.sfb;
         const int row0 = blk == 0 ? t.a_row0 : t.b_row0 + (blk - 1) * 128;
         const int kb0 = ((blk == 0 ? t.a_k0 : t.b_k0) >> 5) + it * 4;
-        uint32_t w[4];
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const int row = row0 + lane + 32 * j;
-            uint32_t word = 0;
-#pragma unroll
-            for (int kb = 0; kb < 4; kb++) word |= (uint32_t)load_scale(v, row, kb0 + kb) << (8 * kb);
-            w[j] = word;
-        }
-        const int off = blk == 0 ? (kSfaOff >> 4) : (kSfbOff >> 4) + (blk - 1) * 32;
-        img[off + lane] = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int j = 0; j < 4; j++) r.w[blk][j] = load_scale_word(v, row0 + lane + 32 * j, kb0);
     }
+    return r;
+}
+
+__device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint8_t *sf_stage, int lane)
+{
+    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
+    img[(kSfaOff >> 4) + lane] = make_uint4(r.w[0][0], r.w[0][1], r.w[0][2], r.w[0][3]);
+    img[(kSfbOff >> 4) + lane] = make_uint4(r.w[1][0], r.w[1][1], r.w[1][2], r.w[1][3]);
+    img[(kSfbOff >> 4) + 32 + lane] = make_uint4(r.w[2][0], r.w[2][1], r.w[2][2], r.w[2][3]);
     __syncwarp();
+}
+
+template <int KIND> struct ScaleRegsOf { typedef ScaleRegs2D type; };
+template <> struct ScaleRegsOf<KIND_MXF8> { typedef ScaleRegs1D type; };
+
+__device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs2D &r)
+{
+    r = fetch_scales_2d(p, t, it, lane);
+}
+__device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs1D &r)
+{
+    r = fetch_scales_1d(p, t, it, lane);
+}
+__device__ __forceinline__ void write_scale_images(const ScaleRegs2D &r, uint8_t *sf_stage, uint8_t *scratch, int lane)
+{
+    write_scale_images_2d(r, sf_stage, scratch, lane);
+}
+__device__ __forceinline__ void write_scale_images(const ScaleRegs1D &r, uint8_t *sf_stage, uint8_t *, int lane)
+{
+    write_scale_images_1d(r, sf_stage, lane);
 }
 
 // ---------------------------------------------------------------------------------------- epilogue store
@@ -438,24 +505,38 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ scale loader
-        uint32_t stage = 0, phase = 0;
+        typename ScaleRegsOf<KIND>::type pre[kStages];
+        WorkIter fetch_it, write_it;
+        fetch_it.tile = write_it.tile = blockIdx.x;
+        fetch_it.seek(p, kStageElems);
+        write_it.seek(p, kStageElems);
+#pragma unroll
+        for (int d = 0; d < kStages; d++) {
+            if (fetch_it.valid(p)) {
+                fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[d]);
+                fetch_it.next(p, kStageElems);
+            }
+        }
+        uint32_t phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
-            Tile t;
-            decode_tile(p, tile, t);
-            const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
-            for (int it = 0; it < n_it; it++) {
+        while (ok && write_it.valid(p)) {
+#pragma unroll
+            for (int stage = 0; stage < kStages; stage++) {
+                if (!write_it.valid(p)) break;
                 if (lane == 0) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
-                uint8_t *sf_stage = smem_sf + stage * kSfStageBytes;
-                if (KIND == KIND_MXF4) build_scale_images_2d(p, t, it, sf_stage, scale_scratch, lane);
-                else build_scale_images_1d(p, t, it, sf_stage, lane);
+                write_scale_images(pre[stage], smem_sf + stage * kSfStageBytes, scale_scratch, lane);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full + 8 * stage);
-                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                if (fetch_it.valid(p)) {
+                    fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[stage]);
+                    fetch_it.next(p, kStageElems);
+                }
+                write_it.next(p, kStageElems);
             }
+            phase ^= 1u;
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue

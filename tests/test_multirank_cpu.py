@@ -1,0 +1,47 @@
+"""The N>1 path of the benchmark is 'replicas only': ranks run the same step on their own GPU and rank 0
+reports units of all ranks over the slowest rank's time.  The reduction is exercised here with two gloo
+ranks on the CPU."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = [10.0 + rank, 3.0 - rank]                  # rank 1 is slower on the first figure, faster on the second
+    red = bench.max_over_ranks(ms, dist, "cpu")
+    dist.barrier()
+    if rank == 0:
+        out.put((red, bench.aggregate_throughput(1000.0, world, red[0])))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_report_max_time_and_summed_units():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    red, thr = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert red == [11.0, 3.0]
+    assert abs(thr - 2 * 1000.0 / 11e-3) < 1e-6
+
+
+def test_single_process_passthrough():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks([1.5, 2.5], None) == [1.5, 2.5]
+    assert bench.aggregate_throughput(10.0, 1, 1000.0) == 10.0
