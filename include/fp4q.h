@@ -176,6 +176,25 @@ fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, i
                           int64_t N, void *Q_out, void *K_out, int64_t ldo, fp4q_out dt,
                           void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * fp4q_gemm_fwd_static_workspace -- no counterpart in the paper: the dense forward product of
+ * fp4q_gemm_fwd for callers that cannot allocate device memory (code living inside an application that
+ * owns the device heap, a loop that must stay out of the allocator, a sandbox restricted to buffers it was
+ * handed).  It calls no cudaMalloc, cudaFree or allocating library routine: the kernel's workspace is a
+ * fixed 1024-byte array inside the library's device image (held by every GPU that loads the library
+ * until the process exits).  A request is refused with FP4Q_ERR_WORKSPACE if the workspace the kernels
+ * need (fp4q_workspace_bytes()) exceeds those 1024 bytes; the workspace does not grow with T, N or K, so
+ * no problem size is refused on its account.  X, W, Y, ldy and dt mean what they mean for fp4q_gemm_fwd
+ * (dense form only).  status_out, if not NULL, is a DEVICE pointer to 4 bytes that receives the kernel's
+ * status word (0, or FP4Q_ERR_TIMEOUT) in stream order after the product.
+ * The first call on a device looks up the array's device address (and, like fp4q_gemm_fwd, sets the
+ * kernel's shared-memory attribute): make that first call before any stream capture.
+ * Every call shares the one array and clears it first: two calls that overlap on the GPU (different
+ * streams, or different host threads) race on it, so keep calls to this entry point in one stream order.
+ */
+fp4q_status fp4q_gemm_fwd_static_workspace(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy,
+                                           fp4q_out dt, uint32_t *status_out, void *stream);
+
 const char *fp4q_status_string(fp4q_status s);
 
 /* Library version: major*10000 + minor*100 + patch. */

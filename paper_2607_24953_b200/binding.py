@@ -25,7 +25,7 @@ INDEX_TRANSPOSED = 1
 
 EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgrad",
            "fp4q_mxfp8_quantize1d", "fp4q_mxfp8_qk", "fp4q_workspace_bytes", "fp4q_workspace_status",
-           "fp4q_status_string", "fp4q_version"]
+           "fp4q_status_string", "fp4q_version", "fp4q_gemm_fwd_static_workspace"]
 
 
 class Fp4qError(RuntimeError):
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
             L.fp4q_mxfp8_qk.restype = ci
             L.fp4q_mxfp8_qk.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, i64, i64, i64, vp, vp, i64,
                                         ci, vp, ctypes.c_size_t, vp]
+        if hasattr(L, "fp4q_gemm_fwd_static_workspace"):
+            L.fp4q_gemm_fwd_static_workspace.restype = ci
+            L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
+                                                         ci, vp, vp]
         _lib = L
     return _lib
 
@@ -219,6 +223,19 @@ def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offs
     """Y[T,N] = X^ W^^T. Grouped when row_offsets is given (W is then the expert stack [E*N, K])."""
     n = W.rows if row_offsets is None else W.rows // (row_offsets.numel() - 1)
     return _gemm("fp4q_gemm_fwd", X, W, X.rows, n, out, dt, row_offsets, ws, stream)
+
+
+def fp4q_gemm_fwd_static_workspace(X: QTensor, W: QTensor, out: torch.Tensor, dt: int = OUT_BF16,
+                                   status_out: Optional[torch.Tensor] = None, stream=None):
+    """Y = X^ W^^T through the entry point that allocates nothing: the caller supplies the output (and,
+    optionally, a 4-byte device tensor for the kernel's status word); the workspace is the library's own
+    fixed array.  Nothing is allocated here either."""
+    cx, cw = X.c_struct(), W.c_struct()
+    st = lib().fp4q_gemm_fwd_static_workspace(ctypes.byref(cx), ctypes.byref(cw), out.data_ptr(), out.stride(0), dt,
+                                              status_out.data_ptr() if status_out is not None else None,
+                                              _stream(stream))
+    _check(st, "fp4q_gemm_fwd_static_workspace")
+    return out
 
 
 def fp4q_gemm_dgrad(dY: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None):

@@ -824,3 +824,53 @@ extern "C" fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uin
     }
     return FP4Q_OK;
 }
+
+// ------------------------------------------------------------------------------------------------------
+// Forward product for callers that cannot allocate device memory.
+//
+// The GEMM kernel records device-side anomalies in a small workspace that the regular entry points take
+// from the caller.  Code that runs where cudaMalloc is off limits -- a plug-in inside a host application
+// that owns the device heap, a real-time loop that must not enter the allocator, a sandbox that only hands
+// out pre-registered buffers -- has no way to supply one.  For those callers the workspace lives in the
+// fixed array below, which every GPU that loads this library holds until the process exits.
+namespace fp4q {
+
+constexpr size_t kStaticWorkspaceBytes = 1024;   // stated maximum; the kernel's workspace must fit in it
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+constexpr int kMaxDevices = 64;
+static void *g_static_workspace_addr[kMaxDevices];   // device address of the array, per device
+
+// In host code the array's name is only a handle: the device address has to be asked for, once per device,
+// with that device current.
+static fp4q_status static_workspace_address(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP4Q_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return FP4Q_ERR_UNSUPPORTED;
+    if (g_static_workspace_addr[dev] == nullptr) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return FP4Q_ERR_CUDA;
+        g_static_workspace_addr[dev] = ptr;
+    }
+    *out = g_static_workspace_addr[dev];
+    return FP4Q_OK;
+}
+
+}  // namespace fp4q
+
+extern "C" fp4q_status fp4q_gemm_fwd_static_workspace(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy,
+                                                      fp4q_out dt, uint32_t *status_out, void *stream)
+{
+    if (fp4q_workspace_bytes() > kStaticWorkspaceBytes) return FP4Q_ERR_WORKSPACE;   // layout outgrew the array
+    void *ws = nullptr;
+    if (fp4q_status s = static_workspace_address(&ws)) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: the status words must start at zero
+    if (cudaMemsetAsync(ws, 0, sizeof(Workspace), st) != cudaSuccess) return FP4Q_ERR_CUDA;
+    if (fp4q_status s = fp4q_gemm_fwd(X, W, Y, ldy, dt, nullptr, ws, kStaticWorkspaceBytes, stream)) return s;
+    if (status_out &&
+        cudaMemcpyAsync(status_out, ws, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return FP4Q_ERR_CUDA;
+    return FP4Q_OK;
+}
