@@ -15,7 +15,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfp4q.so")
+LIB_PATH = os.environ.get("FP4Q_LIB") or os.path.join(_HERE, "libfp4q.so")   # FP4Q_LIB: load another build of the library
 
 ROUND_NEAREST = 0
 ROUND_STOCHASTIC = 1

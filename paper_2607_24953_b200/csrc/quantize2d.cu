@@ -3,16 +3,24 @@
 // One pass over HBM: 2 B/element read, 0.5 + 0.5 B/element written, 1 B per 1024 elements of scale.
 // A CTA of 4 warps owns a 128x128 element block; a warp owns 32 rows x 128 columns (four 32x32
 // blocks side by side); 8 lanes own one 32x32 block, each lane 8 rows x 16 consecutive columns
-// (two 128-bit loads per row).  The block maximum is reduced with warp shuffles over those
-// 8 lanes, the E2M1 codes of a row segment are produced 2 at a time on packed fp16 lanes, the
-// row-major payload goes straight to global memory (8 B per lane and row, 64 B contiguous per
-// row and warp) and the transposed payload is built with an in-register 8x8 nibble transpose,
-// staged through 8 KB of shared memory and written as 64 B contiguous segments.
+// (one 256-bit load per row, all eight issued before anything else).  While the loads are in flight
+// the lane draws its Philox bytes (they do not depend on the data) and parks them in shared memory.
+// The block maximum is reduced with warp shuffles over the 8 lanes, the E2M1 codes come from the
+// hardware converts, the row-major payload goes straight to global memory (8 B per lane and row,
+// 64 B contiguous per row and warp) and the transposed payload is built with an in-register 8x8
+// nibble transpose, staged through 8 KB of shared memory and written as 64 B contiguous segments.
+// CTAs whose tile lies fully inside an aligned tensor run a check-free body; ragged edges, unaligned
+// inputs, cols % 16 != 0 and the transposed index take a general body with the same arithmetic.
 //
-// Rounding works on the BF16 value scaled by 2^(-e-14) and converted (toward zero) to fp16: the
-// fp16 bit pattern of |x| 2^(-e-14) has the E2M1 magnitude code in bits 11..9 and the position
-// between the two neighbouring codes in bits 8..0, uniformly over normal and subnormal codes.
-// Adding 2*r8 (stochastic) or 0xFF + lsb (nearest-even) and taking bits 11..9 is the rounding.
+// Rounding: x 2^-e (exact in FP32) goes through the hardware converts cvt.rn.satfinite.e2m1x2.f32
+// (nearest even) or cvt.rs.satfinite.e2m1x4.f32 (stochastic).  The stochastic convert adds 16 random bits
+// below the kept mantissa bit and truncates; the elements that land in nibbles 0 and 2 take the upper 8
+// of their 16 bits from rbits[23:16] and rbits[31:24] and the lower 8 from rbits[7:0] and rbits[15:8]
+// (the other two inputs reuse the same bits in reversed order).  With the lower bytes zero and only
+// those two inputs used, the instruction computes exactly "up iff floor(256 p) + r8 >= 256" for two
+// elements at a time: the element's random byte is routed into place with one PRMT.  Blocks that
+// contain non-finite values take a scalar path that rounds on the fp16 bit pattern of |x| 2^(-e-14)
+// (magnitude code in bits 11..9, position between neighbours in bits 8..0).
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -35,7 +43,7 @@ struct Quant2dParams {
     int64_t grid_x;           // CTAs along the column direction
     uint32_t tensor_id;
     uint32_t flags;
-    int x_vec_ok;             // x 16-byte aligned and ld_x % 8 == 0: 128-bit loads are legal
+    int x_vec_ok;             // 2: x 32-byte aligned, ld_x % 16 == 0 (256-bit loads); 1: 16-byte aligned, ld_x % 8 == 0
     int rng_aligned;          // cols % 16 == 0 and index not transposed: one Philox block per 16-element segment
     PhiloxRoundKeys keys;
 };
@@ -92,6 +100,24 @@ __device__ __forceinline__ float inv_scale_f16_aligned(int code)
     return __uint_as_float(e > 0 ? (uint32_t)e << 23 : 1u << (22 + e));
 }
 
+// 2^-e = 2^(127-code): always a normal FP32 for code in [0, 253].
+__device__ __forceinline__ float inv_scale(int code) { return __uint_as_float((uint32_t)(254 - code) << 23); }
+
+// Four FP32 -> four E2M1 nibbles (e0 in bits 3..0), stochastic rounding with the hardware's byte routing.
+__device__ __forceinline__ uint32_t cvt_rs_e2m1x4(float e3, float e2, float e1, float e0, uint32_t rbits)
+{
+    uint16_t d;
+    asm("cvt.rs.satfinite.e2m1x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=h"(d) : "f"(e3), "f"(e2), "f"(e1), "f"(e0), "r"(rbits));
+    return d;
+}
+// Two FP32 -> two E2M1 nibbles (lo in bits 3..0), round to nearest even.
+__device__ __forceinline__ uint32_t cvt_rn_e2m1x2(float hi, float lo)
+{
+    uint16_t d;
+    asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; cvt.u16.u8 %0, t; }" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
 // One element, scalar: used for blocks that contain non-finite values.
 template <int MODE>
 __device__ __forceinline__ uint32_t quantize_scalar(uint32_t bits16, float inv, uint32_t r8)
@@ -112,32 +138,48 @@ __device__ __forceinline__ void round_segment(const uint32_t raw[8], float inv, 
 {
 #pragma unroll
     for (int g = 0; g < 2; g++) {
-        float v[8];
+        uint32_t half[2];
 #pragma unroll
-        for (int q = 0; q < 4; q++) {
-            const uint32_t w = raw[4 * g + q];
-            v[2 * q] = __uint_as_float(w << 16) * inv;
-            v[2 * q + 1] = __uint_as_float(w & 0xFFFF0000u) * inv;
+        for (int h = 0; h < 2; h++) {
+            const int q = 2 * g + h;                       // elements 4q .. 4q+3
+            const uint32_t w0 = raw[2 * q], w1 = raw[2 * q + 1];
+            const float v0 = __uint_as_float(w0 << 16) * inv, v1 = __uint_as_float(w0 & 0xFFFF0000u) * inv;
+            const float v2 = __uint_as_float(w1 << 16) * inv, v3 = __uint_as_float(w1 & 0xFFFF0000u) * inv;
+            if (MODE == FP4Q_ROUND_STOCHASTIC) {
+                // random bytes r0..r3 of the four elements; first convert: elements 0 and 2 (nibbles 0, 2),
+                // second convert: elements 1 and 3, merged one nibble higher
+                const uint32_t even = cvt_rs_e2m1x4(0.0f, v2, 0.0f, v0, __byte_perm(R[q], 0u, 0x2044));
+                const uint32_t odd = cvt_rs_e2m1x4(0.0f, v3, 0.0f, v1, __byte_perm(R[q], 0u, 0x3144));
+                half[h] = even | (odd << 4);
+            } else {
+                half[h] = cvt_rn_e2m1x2(v1, v0) | (cvt_rn_e2m1x2(v3, v2) << 8);
+            }
         }
+        W[g] = half[0] | (half[1] << 16);
+    }
+}
+
+// The same 16 elements through the scalar path, kept out of line: it is only taken by blocks that hold a
+// non-finite value, and inlining it into the row loop would triple the loop's instruction footprint.
+template <int MODE>
+__device__ __noinline__ uint2 round_segment_scalar(uint4 lo, uint4 hi, uint4 rnd, float inv16)
+{
+    const uint32_t raw[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    const uint32_t R[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+    uint32_t W[2];
+#pragma unroll
+    for (int g = 0; g < 2; g++) {
         uint32_t acc = 0;
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            // fp16 lanes: low = element 8g+j, high = element 8g+j+4 (nibbles j and j+4 are 16 bits apart)
-            const uint32_t h2 = cvt_rz_f16x2(v[j + 4], v[j]);
-            uint32_t b2;
-            if (MODE == FP4Q_ROUND_STOCHASTIC) {
-                const uint32_t sel = (uint32_t)j | ((uint32_t)j << 4) | ((uint32_t)(4 + j) << 8) | ((uint32_t)j << 12);
-                const uint32_t rm = __byte_perm(R[2 * g], R[2 * g + 1], sel) & 0x00FF00FFu;
-                b2 = h2 + (rm << 1);
-            } else {
-                b2 = h2 + 0x00FF00FFu + ((h2 >> 9) & 0x00010001u);
-            }
-            const uint32_t t = b2 | (b2 >> 3);   // sign (bit 15) next to the magnitude code (bits 11..9)
-            const uint32_t nib = (j < 3 ? t >> (9 - 4 * j) : t << 3) & (0x000F000Fu << (4 * j));
-            acc |= nib;
+        for (int e = 0; e < 8; e++) {
+            const int k = 8 * g + e;
+            const uint32_t bits = (raw[k >> 1] >> (16 * (k & 1))) & 0xFFFFu;
+            const uint32_t r8 = (R[k >> 2] >> (8 * (k & 3))) & 0xFFu;
+            acc |= quantize_scalar<MODE>(bits, inv16, r8) << (4 * e);
         }
         W[g] = acc;
     }
+    return make_uint2(W[0], W[1]);
 }
 
 // In-register transpose of an 8x8 matrix of nibbles: a[r] holds row r (nibble c = column c);
@@ -171,7 +213,12 @@ __device__ __forceinline__ void load_segment(const Quant2dParams &p, int64_t i, 
         return;
     }
     const uint16_t *src = p.x + i * p.ld_x + j0;
-    if (p.x_vec_ok && j0 + 16 <= p.cols) {
+    if (p.x_vec_ok == 2 && j0 + 16 <= p.cols) {
+        asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(out[0]), "=r"(out[1]), "=r"(out[2]), "=r"(out[3]), "=r"(out[4]), "=r"(out[5]), "=r"(out[6]),
+                       "=r"(out[7])
+                     : "l"(src));
+    } else if (p.x_vec_ok && j0 + 16 <= p.cols) {
         const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
         const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
         out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
@@ -186,14 +233,10 @@ __device__ __forceinline__ void load_segment(const Quant2dParams &p, int64_t i, 
     }
 }
 
-// The 16 random bytes of the row segment starting at element (i, j0).
+// The 16 random bytes of the row segment starting at element (i, j0), one Philox call per element: the slow
+// generic path for cols % 16 != 0 or the transposed index.
 __device__ __forceinline__ void segment_random_bytes(const Quant2dParams &p, int64_t i, int64_t j0, uint32_t R[4])
 {
-    if (p.rng_aligned) {
-        const uint64_t blk = ((uint64_t)i * (uint64_t)p.cols + (uint64_t)j0) >> 4;
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, R);
-        return;
-    }
 #pragma unroll
     for (int w = 0; w < 4; w++) {
         uint32_t word = 0;
@@ -211,11 +254,15 @@ __device__ __forceinline__ void segment_random_bytes(const Quant2dParams &p, int
     }
 }
 
-template <int MODE>
-__global__ void __launch_bounds__(128) quantize2d_kernel(const __grid_constant__ Quant2dParams p)
-{
-    __shared__ uint4 qt_stage[128 * 4];   // 128 transposed rows x 64 B (four 16-byte chunks, XOR-swizzled)
+#ifndef FP4Q_QUANT_MIN_BLOCKS
+#define FP4Q_QUANT_MIN_BLOCKS 4
+#endif
 
+// FAST = the CTA's 128x128 tile lies fully inside the tensor, rows are 32-byte aligned (256-bit loads) and
+// one Philox block covers each 16-element segment: no per-row bounds or path checks remain in the hot loop.
+template <int MODE, bool FAST>
+__device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_stage, uint4 *rnd_stage)
+{
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = lane >> 3;          // which of the warp's four 32x32 blocks
     const int rg = (lane >> 1) & 3;   // group of 8 rows inside the block
@@ -223,11 +270,35 @@ __global__ void __launch_bounds__(128) quantize2d_kernel(const __grid_constant__
     const int64_t bx = (int64_t)blockIdx.x % p.grid_x, by = (int64_t)blockIdx.x / p.grid_x;
     const int64_t tile_row0 = by * 128 + warp * 32, tile_col0 = bx * 128 + t * 32;
     const int64_t row0 = tile_row0 + rg * 8, col0 = tile_col0 + ch * 16;
-    const bool tile_exists = tile_row0 < p.rows && tile_col0 < p.cols;
+    const bool tile_exists = FAST || (tile_row0 < p.rows && tile_col0 < p.cols);
 
     uint32_t raw[8][8];
+    if (FAST) {
+        const uint16_t *src = p.x + row0 * p.ld_x + col0;
 #pragma unroll
-    for (int r = 0; r < 8; r++) load_segment(p, row0 + r, col0, raw[r]);
+        for (int r = 0; r < 8; r++)
+            asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(raw[r][0]), "=r"(raw[r][1]), "=r"(raw[r][2]), "=r"(raw[r][3]), "=r"(raw[r][4]),
+                           "=r"(raw[r][5]), "=r"(raw[r][6]), "=r"(raw[r][7])
+                         : "l"(src + r * p.ld_x));
+    } else {
+#pragma unroll
+        for (int r = 0; r < 8; r++) load_segment(p, row0 + r, col0, raw[r]);
+    }
+
+    // The random bytes do not depend on the data: draw them while the loads are in flight and park them in
+    // shared memory (each thread reads back only what it wrote), in a rolled loop that keeps the code small.
+    if (MODE == FP4Q_ROUND_STOCHASTIC && (FAST || p.rng_aligned)) {
+        uint64_t idx = (uint64_t)row0 * (uint64_t)p.cols + (uint64_t)col0;
+#pragma unroll 2
+        for (int r = 0; r < 8; r++) {
+            uint32_t R[4];
+            const uint64_t blk = idx >> 4;
+            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, R);
+            rnd_stage[r * 128 + threadIdx.x] = make_uint4(R[0], R[1], R[2], R[3]);
+            idx += (uint64_t)p.cols;
+        }
+    }
 
     // block maximum: packed BF16 |.| max with NaN propagation, so that any non-finite entry shows
     // up in the result and routes the block to the scalar path
@@ -266,37 +337,52 @@ __global__ void __launch_bounds__(128) quantize2d_kernel(const __grid_constant__
     }
 
     const int code = scale_code_from_max(mbits);
-    const float inv = inv_scale_f16_aligned(code);
+    const float inv = inv_scale(code);
     if (tile_exists && (lane & 7) == 0)
         p.scale[(tile_row0 >> 5) * p.ld_s + (tile_col0 >> 5)] = (uint8_t)code;
 
     uint32_t W[8][2];
+    uint8_t *dst_rm = p.q_rm + row0 * p.ld_rm + (col0 >> 1);
+    if (FAST && !nonfinite) {
+        // hot loop: no bounds checks, no path selection
 #pragma unroll
-    for (int r = 0; r < 8; r++) {
-        const int64_t i = row0 + r;
-        if (!tile_exists || i >= p.rows) {
-            W[r][0] = W[r][1] = 0u;
-            continue;
-        }
-        uint32_t R[4] = {0u, 0u, 0u, 0u};
-        if (MODE == FP4Q_ROUND_STOCHASTIC) segment_random_bytes(p, i, col0, R);
-        if (!nonfinite) {
-            round_segment<MODE>(raw[r], inv, R, W[r]);
-        } else {
-#pragma unroll
-            for (int g = 0; g < 2; g++) {
-                uint32_t acc = 0;
-#pragma unroll
-                for (int e = 0; e < 8; e++) {
-                    const int k = 8 * g + e;
-                    const uint32_t bits = (raw[r][k >> 1] >> (16 * (k & 1))) & 0xFFFFu;
-                    const uint32_t r8 = (R[k >> 2] >> (8 * (k & 3))) & 0xFFu;
-                    acc |= quantize_scalar<MODE>(bits, inv, r8) << (4 * e);
-                }
-                W[r][g] = acc;
+        for (int r = 0; r < 8; r++) {
+            uint32_t R[4] = {0u, 0u, 0u, 0u};
+            if (MODE == FP4Q_ROUND_STOCHASTIC) {
+                const uint4 v = rnd_stage[r * 128 + threadIdx.x];
+                R[0] = v.x; R[1] = v.y; R[2] = v.z; R[3] = v.w;
             }
+            round_segment<MODE>(raw[r], inv, R, W[r]);
+            *reinterpret_cast<uint2 *>(dst_rm + r * p.ld_rm) = make_uint2(W[r][0], W[r][1]);
         }
-        *reinterpret_cast<uint2 *>(p.q_rm + i * p.ld_rm + (col0 >> 1)) = make_uint2(W[r][0], W[r][1]);
+    } else {
+#pragma unroll
+        for (int r = 0; r < 8; r++) {
+            const int64_t i = row0 + r;
+            if (!tile_exists || i >= p.rows) {
+                W[r][0] = W[r][1] = 0u;
+                continue;
+            }
+            uint32_t R[4] = {0u, 0u, 0u, 0u};
+            if (MODE == FP4Q_ROUND_STOCHASTIC) {
+                if (FAST || p.rng_aligned) {
+                    const uint4 v = rnd_stage[r * 128 + threadIdx.x];
+                    R[0] = v.x; R[1] = v.y; R[2] = v.z; R[3] = v.w;
+                } else {
+                    segment_random_bytes(p, i, col0, R);
+                }
+            }
+            if (!nonfinite) {
+                round_segment<MODE>(raw[r], inv, R, W[r]);
+            } else {
+                const uint2 w = round_segment_scalar<MODE>(make_uint4(raw[r][0], raw[r][1], raw[r][2], raw[r][3]),
+                                                           make_uint4(raw[r][4], raw[r][5], raw[r][6], raw[r][7]),
+                                                           make_uint4(R[0], R[1], R[2], R[3]), inv_scale_f16_aligned(code));
+                W[r][0] = w.x;
+                W[r][1] = w.y;
+            }
+            *reinterpret_cast<uint2 *>(dst_rm + r * p.ld_rm) = make_uint2(W[r][0], W[r][1]);
+        }
     }
 
     if (p.q_t == nullptr) return;
@@ -323,11 +409,22 @@ __global__ void __launch_bounds__(128) quantize2d_kernel(const __grid_constant__
         const int row_local = (threadIdx.x >> 2) + 32 * k;   // transposed row = source column; its block index is k
         const int chunk = threadIdx.x & 3;                    // 32 source rows = one source warp
         const int64_t col = bx * 128 + row_local;
-        if (col < p.cols && by * 128 + chunk * 32 < p.rows) {
+        if (FAST || (col < p.cols && by * 128 + chunk * 32 < p.rows)) {
             const uint4 v = qt_stage[row_local * 4 + (chunk ^ k)];
             *reinterpret_cast<uint4 *>(p.q_t + col * p.ld_t + by * 64 + chunk * 16) = v;
         }
     }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(128, FP4Q_QUANT_MIN_BLOCKS) quantize2d_kernel(const __grid_constant__ Quant2dParams p)
+{
+    __shared__ uint4 qt_stage[128 * 4];   // 128 transposed rows x 64 B (four 16-byte chunks, XOR-swizzled)
+    __shared__ uint4 rnd_stage[MODE == FP4Q_ROUND_STOCHASTIC ? 8 * 128 : 1];   // per thread: 8 rows x 16 random bytes
+    const int64_t bx = (int64_t)blockIdx.x % p.grid_x, by = (int64_t)blockIdx.x / p.grid_x;
+    const bool full = p.x_vec_ok == 2 && p.rng_aligned && (by + 1) * 128 <= p.rows && (bx + 1) * 128 <= p.cols;
+    if (full) quantize_tile<MODE, true>(p, qt_stage, rnd_stage);
+    else quantize_tile<MODE, false>(p, qt_stage, rnd_stage);
 }
 
 static void philox_round_keys(uint64_t seed, PhiloxRoundKeys &k)
@@ -370,7 +467,7 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
     p.grid_x = ceil_div(cols, 128);
     p.tensor_id = tensor_id;
     p.flags = flags;
-    p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
+    p.x_vec_ok = (aligned(x_bf16, 32) && ld_x % 16 == 0) ? 2 : (aligned(x_bf16, 16) && ld_x % 8 == 0) ? 1 : 0;
     p.rng_aligned = cols % 16 == 0 && !(flags & FP4Q_INDEX_TRANSPOSED);
     philox_round_keys(seed, p.keys);
 
