@@ -8,8 +8,12 @@
 //
 // One persistent CTA per SM, 128x256 output tile, 12 warps:
 //   warp 0      TMA producer: A tile (128 rows x 128 B) and B tile (256 rows x 128 B) per stage, 128B swizzle
-//   warp 1      MMA issuer: tcgen05.cp of the stage's scale image smem -> TMEM, then 4 tcgen05.mma per stage
-//   warp 2      scale loader: compact scale bytes -> the 32-lane x 16-byte image tcgen05.cp expects
+//   warp 1      MMA issuer: tcgen05.cp of the stage's scale images smem -> TMEM, 4 tcgen05.mma per stage,
+//               tcgen05.commit to release the stage
+//   warp 3      scale cache builder (2D-block scales): once per tile gathers all compact scale bytes the tile
+//               needs into shared memory, arranged as 16-byte image rows (double-buffered across tiles)
+//   warp 2      scale image writer: per stage replicates six cached rows into the 32-lane x 16-byte images that
+//               tcgen05.cp expects (for MXFP8 per-row scales warps 2-3 alternate stages and load directly)
 //   warps 4-11  epilogue: tcgen05.ld of the 128x256 FP32 accumulator (each warp 32 lanes x 128 columns),
 //               release of the accumulator as soon as it sits in registers, then convert and store
 // Four smem stages (48 KB of operands + 3 KB of scale image each) form a ring guarded by mbarriers; the
@@ -31,12 +35,21 @@ constexpr int kSfStageBytes = 3072;          // SFA 2 x 512 B, SFB 2 x 1024 B
 constexpr int kSfaOff = 0, kSfbOff = 1024;
 constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
 constexpr int kSmemSf = kStages * kSfStageBytes;
-constexpr int kSmemTail = 256;               // barriers, TMEM base, abort flag, scale scratch
-constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemTail;
+constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
+constexpr int kCacheChunks = 128;            // scale cache: contraction chunks of 128 elements per unit (16384 elements)
+constexpr int kCacheBytes = kCacheChunks * 48;   // per chunk: 16 B for A (4 row tiles x 4 blocks) + 32 B for B (8 x 4)
+constexpr int kSmemCache = 2 * kCacheBytes;
+constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemCache + kSmemTail;
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
 constexpr uint32_t kWaitLimit = 1u << 22;
+#ifndef FP4Q_RELAXED_NS
+#define FP4Q_RELAXED_NS 64
+#endif
+#ifndef FP4Q_LAZY_NS
+#define FP4Q_LAZY_NS 256
+#endif
 constexpr uint8_t kScalePad = 127;           // UE8M0 code of 1.0 for scale slots beyond the tensor (their payload is 0)
 
 enum { KIND_MXF4 = 0, KIND_MXF8 = 1 };
@@ -93,17 +106,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // Bounded wait.  Returns false when the limit ran out (the timeout is then recorded) or when another
-// role of this CTA has already given up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                       uint32_t where)
+// role of this CTA has already given up.  Every poll of an mbarrier is a shared-memory transaction that
+// competes with the tensor core's operand reads and with the MMA thread's own waits, so roles that have
+// slack (everything but the MMA issuer) sleep between polls.
+template <int BACKOFF_NS>
+__device__ __forceinline__ bool mbar_wait_impl(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                               uint32_t where)
 {
     for (uint32_t it = 0; it < kWaitLimit; it++) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1u;
     if (atomicCAS(status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) status[1] = where;
     return false;
+}
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint32_t where)
+{
+    return mbar_wait_impl<0>(bar, parity, abort_flag, status, where);
+}
+__device__ __noinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                               uint32_t where)
+{
+    return mbar_wait_impl<FP4Q_RELAXED_NS>(bar, parity, abort_flag, status, where);
+}
+__device__ __noinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                            uint32_t where)
+{
+    return mbar_wait_impl<FP4Q_LAZY_NS>(bar, parity, abort_flag, status, where);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
@@ -213,9 +244,17 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, Tile 
 
 // ---------------------------------------------------------------------------------------- scale images
 
-__device__ __forceinline__ uint8_t load_scale(const ScaleView &v, int row, int kb)
+// Scale slots beyond the tensor read this byte instead (their payload is zero, any finite scale will do).
+__device__ const uint8_t g_scale_pad[4] = {kScalePad, kScalePad, kScalePad, kScalePad};
+
+// One compact scale byte.  The bounds check selects the ADDRESS, not the value, so that nothing depends on
+// the loaded byte until it is written into the image several stages later (an in-order warp stalls at the
+// first use of a pending load).
+__device__ __forceinline__ void load_scale(const ScaleView &v, int row, int kb, uint32_t &dst)
 {
-    return (row < v.n_row && kb < v.n_kb) ? __ldg(v.ptr + (int64_t)row * v.stride_row + (int64_t)kb * v.stride_kb) : kScalePad;
+    const uint8_t *ptr = (row < v.n_row && kb < v.n_kb) ? v.ptr + (int64_t)row * v.stride_row + (int64_t)kb * v.stride_kb
+                                                        : g_scale_pad;
+    asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(dst) : "l"(ptr));
 }
 
 // The scale loader runs ahead of the ring: the compact scale bytes of a stage are fetched into registers
@@ -241,69 +280,227 @@ struct WorkIter {
 };
 
 // mxf4 / 2D blocks: a stage covers 8 contraction blocks (two chunks of 4).  For 128 operand rows and one chunk
-// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3].  Per stage a lane fetches one byte of
-// A's 2 x 4 x 4 and two bytes of B's 2 x 8 x 4 compact scale bytes.
-struct ScaleRegs2D { uint32_t a, b0, b1; };
+// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3]; A needs 2 such rows per stage (one per
+// chunk), B (256 rows) 4.  The compact bytes are fetched with wide loads that every lane issues to the same
+// address (one broadcast transaction): 8 bytes along the contraction per row tile when the scale matrix is read
+// as stored, or the 4 / 8 row-tile bytes of one contraction block when it is read transposed (then a 4x4 byte
+// transpose in registers forms the rows).  Tiles at the edge of the scale matrix or with unaligned scales fall
+// back to one byte per lane gathered through a small shared-memory scratch.
+enum { SF_BYTES = 0, SF_ALONG_K = 1, SF_ALONG_ROWS = 2 };
+struct ScaleRegs2D { uint32_t a[8], b[16]; };
 
-__device__ __forceinline__ ScaleRegs2D fetch_scales_2d(const GemmParams &p, const Tile &t, int it, int lane)
+__device__ __forceinline__ int scale_mode_2d(const ScaleView &v, int rt0, int n_rt, int kb0)
 {
-    ScaleRegs2D r;
-    {
-        const int c = lane >> 4, rt = (lane >> 2) & 3, kb = lane & 3;
-        r.a = load_scale(p.sfa, (t.a_row0 >> 5) + rt, (t.a_k0 >> 5) + it * 8 + c * 4 + kb);
-    }
-    {
-        const int c = lane >> 5, rt = (lane >> 2) & 7, kb = lane & 3;   // idx = lane: chunk 0
-        r.b0 = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + c * 4 + kb);
-        r.b1 = load_scale(p.sfb, (t.b_row0 >> 5) + rt, (t.b_k0 >> 5) + it * 8 + 4 + kb);   // idx = lane + 32: chunk 1
-    }
-    return r;
+    if (rt0 + n_rt > v.n_row || kb0 + 8 > v.n_kb) return SF_BYTES;
+    const uintptr_t base = reinterpret_cast<uintptr_t>(v.ptr);
+    if (v.stride_kb == 1)
+        return (((base + (uintptr_t)rt0 * v.stride_row + kb0) & 7) == 0 && (v.stride_row & 7) == 0) ? SF_ALONG_K : SF_BYTES;
+    if (v.stride_row == 1)
+        return (((base + (uintptr_t)kb0 * v.stride_kb + rt0) & (n_rt - 1)) == 0 && (v.stride_kb & (n_rt - 1)) == 0)
+                   ? SF_ALONG_ROWS : SF_BYTES;
+    return SF_BYTES;
 }
 
-__device__ __forceinline__ void write_scale_images_2d(const ScaleRegs2D &r, uint8_t *sf_stage, uint8_t *scratch, int lane)
+__device__ __forceinline__ void ldg_b64(const uint8_t *ptr, uint32_t &lo, uint32_t &hi)
 {
-    scratch[lane] = (uint8_t)r.a;            // [chunk][row tile 0..3][block]
-    scratch[32 + lane] = (uint8_t)r.b0;      // chunk 0: [row tile 0..7][block]
-    scratch[64 + lane] = (uint8_t)r.b1;      // chunk 1
-    __syncwarp();
-    const uint4 *s4 = reinterpret_cast<const uint4 *>(scratch);
+    asm volatile("ld.global.nc.v2.b32 {%0, %1}, [%2];" : "=r"(lo), "=r"(hi) : "l"(ptr));
+}
+__device__ __forceinline__ void ldg_b32(const uint8_t *ptr, uint32_t &w)
+{
+    asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(w) : "l"(ptr));
+}
+
+__device__ __forceinline__ void fetch_scales_2d(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs2D &r)
+{
+    const int a_rt0 = t.a_row0 >> 5, a_kb0 = (t.a_k0 >> 5) + it * 8;
+    const int b_rt0 = t.b_row0 >> 5, b_kb0 = (t.b_k0 >> 5) + it * 8;
+    const int ma = scale_mode_2d(p.sfa, a_rt0, 4, a_kb0), mb = scale_mode_2d(p.sfb, b_rt0, 8, b_kb0);
+    if (ma == SF_ALONG_K) {
+#pragma unroll
+        for (int rt = 0; rt < 4; rt++)
+            ldg_b64(p.sfa.ptr + (int64_t)(a_rt0 + rt) * p.sfa.stride_row + a_kb0, r.a[2 * rt], r.a[2 * rt + 1]);
+    } else if (ma == SF_ALONG_ROWS) {
+#pragma unroll
+        for (int kb = 0; kb < 8; kb++) ldg_b32(p.sfa.ptr + (int64_t)(a_kb0 + kb) * p.sfa.stride_kb + a_rt0, r.a[kb]);
+    } else {
+        const int c = lane >> 4, rt = (lane >> 2) & 3, kb = lane & 3;
+        load_scale(p.sfa, a_rt0 + rt, a_kb0 + c * 4 + kb, r.a[0]);
+    }
+    if (mb == SF_ALONG_K) {
+#pragma unroll
+        for (int rt = 0; rt < 8; rt++)
+            ldg_b64(p.sfb.ptr + (int64_t)(b_rt0 + rt) * p.sfb.stride_row + b_kb0, r.b[2 * rt], r.b[2 * rt + 1]);
+    } else if (mb == SF_ALONG_ROWS) {
+#pragma unroll
+        for (int kb = 0; kb < 8; kb++)
+            ldg_b64(p.sfb.ptr + (int64_t)(b_kb0 + kb) * p.sfb.stride_kb + b_rt0, r.b[2 * kb], r.b[2 * kb + 1]);
+    } else {
+        const int rt = (lane >> 2) & 7, kb = lane & 3;
+        load_scale(p.sfb, b_rt0 + rt, b_kb0 + kb, r.b[0]);       // chunk 0
+        load_scale(p.sfb, b_rt0 + rt, b_kb0 + 4 + kb, r.b[1]);   // chunk 1
+    }
+}
+
+// Rows of a 4x4 byte matrix given by its columns: w[k] holds byte rt of column k in byte lane rt.
+__device__ __forceinline__ uint4 transpose4x4_bytes(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3)
+{
+    const uint32_t t0 = __byte_perm(w0, w1, 0x5140), t1 = __byte_perm(w2, w3, 0x5140);
+    const uint32_t t2 = __byte_perm(w0, w1, 0x7362), t3 = __byte_perm(w2, w3, 0x7362);
+    return make_uint4(__byte_perm(t0, t1, 0x5410), __byte_perm(t0, t1, 0x7632), __byte_perm(t2, t3, 0x5410),
+                      __byte_perm(t2, t3, 0x7632));
+}
+
+__device__ __forceinline__ void write_scale_images_2d(const GemmParams &p, const Tile &t, int it, const ScaleRegs2D &r,
+                                                      uint8_t *sf_stage, uint8_t *scratch, int lane)
+{
+    const int a_rt0 = t.a_row0 >> 5, a_kb0 = (t.a_k0 >> 5) + it * 8;
+    const int b_rt0 = t.b_row0 >> 5, b_kb0 = (t.b_k0 >> 5) + it * 8;
+    const int ma = scale_mode_2d(p.sfa, a_rt0, 4, a_kb0), mb = scale_mode_2d(p.sfb, b_rt0, 8, b_kb0);
+    uint4 rows[6];   // SFA chunk 0, 1; SFB chunk 0 rows 0..127, 128..255; SFB chunk 1 rows 0..127, 128..255
+    if (ma == SF_BYTES || mb == SF_BYTES) {
+        if (ma == SF_BYTES) scratch[lane] = (uint8_t)r.a[0];            // [chunk][row tile 0..3][block]
+        if (mb == SF_BYTES) {
+            scratch[32 + lane] = (uint8_t)r.b[0];                       // chunk 0: [row tile 0..7][block]
+            scratch[64 + lane] = (uint8_t)r.b[1];                       // chunk 1
+        }
+        __syncwarp();
+        const uint4 *s4 = reinterpret_cast<const uint4 *>(scratch);
+#pragma unroll
+        for (int q = 0; q < 6; q++) rows[q] = s4[q];
+        __syncwarp();
+    }
+    if (ma == SF_ALONG_K) {
+        rows[0] = make_uint4(r.a[0], r.a[2], r.a[4], r.a[6]);
+        rows[1] = make_uint4(r.a[1], r.a[3], r.a[5], r.a[7]);
+    } else if (ma == SF_ALONG_ROWS) {
+        rows[0] = transpose4x4_bytes(r.a[0], r.a[1], r.a[2], r.a[3]);
+        rows[1] = transpose4x4_bytes(r.a[4], r.a[5], r.a[6], r.a[7]);
+    }
+    if (mb == SF_ALONG_K) {
+        rows[2] = make_uint4(r.b[0], r.b[2], r.b[4], r.b[6]);
+        rows[3] = make_uint4(r.b[8], r.b[10], r.b[12], r.b[14]);
+        rows[4] = make_uint4(r.b[1], r.b[3], r.b[5], r.b[7]);
+        rows[5] = make_uint4(r.b[9], r.b[11], r.b[13], r.b[15]);
+    } else if (mb == SF_ALONG_ROWS) {
+        rows[2] = transpose4x4_bytes(r.b[0], r.b[2], r.b[4], r.b[6]);
+        rows[3] = transpose4x4_bytes(r.b[1], r.b[3], r.b[5], r.b[7]);
+        rows[4] = transpose4x4_bytes(r.b[8], r.b[10], r.b[12], r.b[14]);
+        rows[5] = transpose4x4_bytes(r.b[9], r.b[11], r.b[13], r.b[15]);
+    }
     uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
-    img[(kSfaOff >> 4) + lane] = s4[0];             // SFA chunk 0
-    img[(kSfaOff >> 4) + 32 + lane] = s4[1];        // SFA chunk 1
-    img[(kSfbOff >> 4) + lane] = s4[2];             // SFB chunk 0, rows 0..127
-    img[(kSfbOff >> 4) + 32 + lane] = s4[3];        // SFB chunk 0, rows 128..255
-    img[(kSfbOff >> 4) + 64 + lane] = s4[4];        // SFB chunk 1, rows 0..127
-    img[(kSfbOff >> 4) + 96 + lane] = s4[5];        // SFB chunk 1, rows 128..255
-    __syncwarp();
+    img[(kSfaOff >> 4) + lane] = rows[0];
+    img[(kSfaOff >> 4) + 32 + lane] = rows[1];
+    img[(kSfbOff >> 4) + lane] = rows[2];
+    img[(kSfbOff >> 4) + 32 + lane] = rows[3];
+    img[(kSfbOff >> 4) + 64 + lane] = rows[4];
+    img[(kSfbOff >> 4) + 96 + lane] = rows[5];
+}
+
+// Gathers the scale bytes of n_chunks contraction chunks (4 blocks each) for 2^log2_rt consecutive row tiles into
+// dst[(chunk << log2_rt) + rt] as 32-bit words (byte k = block 4*chunk + k): the 16-byte image rows of the chunk.
+// One warp; each lane takes items lane, lane + 32, ...  Slots beyond the tensor read the pad byte.
+__device__ __forceinline__ void build_scale_cache(const ScaleView &v, int rt0, int kb0, int n_chunks, int log2_rt,
+                                                  uint32_t *dst, int lane)
+{
+    const bool aligned4 = (reinterpret_cast<uintptr_t>(v.ptr) & 3) == 0;
+    if (v.stride_row == 1 && v.stride_kb != 1 && aligned4 && (v.stride_kb & 3) == 0 && (rt0 & 3) == 0) {
+        // transposed view: the row-tile bytes of one block are contiguous.  An item is a chunk and a group of four
+        // row tiles: four 32-bit loads (one per block) and a 4x4 byte transpose give the group's four words.
+        const int log2_g = log2_rt - 2, n_items = n_chunks << log2_g;
+        for (int base = 0; base < n_items; base += 32 * 2) {
+            uint32_t w[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const int q = base + 32 * j + lane;
+                const int chunk = q >> log2_g, rg = q & ((1 << log2_g) - 1);
+                const int row = rt0 + 4 * rg, kb = kb0 + 4 * chunk;
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    w[j][k] = kScalePad * 0x01010101u;
+                    if (q < n_items) {
+                        if (row + 4 <= v.n_row && kb + k < v.n_kb) {
+                            ldg_b32(v.ptr + (int64_t)(kb + k) * v.stride_kb + row, w[j][k]);
+                        } else {
+                            uint32_t b0, b1, b2, b3;
+                            load_scale(v, row, kb + k, b0);
+                            load_scale(v, row + 1, kb + k, b1);
+                            load_scale(v, row + 2, kb + k, b2);
+                            load_scale(v, row + 3, kb + k, b3);
+                            w[j][k] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const int q = base + 32 * j + lane;
+                if (q < n_items) reinterpret_cast<uint4 *>(dst)[q] = transpose4x4_bytes(w[j][0], w[j][1], w[j][2], w[j][3]);
+            }
+        }
+        return;
+    }
+    const int n_items = n_chunks << log2_rt;
+    const bool along_k = v.stride_kb == 1 && aligned4 && (v.stride_row & 3) == 0 && (kb0 & 3) == 0;
+    for (int base = 0; base < n_items; base += 32 * 4) {
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {   // loads of four items in flight before anything is used
+            const int q = base + 32 * j + lane;
+            const int chunk = q >> log2_rt, rt = q & ((1 << log2_rt) - 1);
+            const int row = rt0 + rt, kb = kb0 + 4 * chunk;
+            w[j] = 0;
+            if (q < n_items) {
+                if (along_k && row < v.n_row && kb + 4 <= v.n_kb) {
+                    ldg_b32(v.ptr + (int64_t)row * v.stride_row + kb, w[j]);
+                } else {
+                    uint32_t b0, b1, b2, b3;
+                    load_scale(v, row, kb, b0);
+                    load_scale(v, row, kb + 1, b1);
+                    load_scale(v, row, kb + 2, b2);
+                    load_scale(v, row, kb + 3, b3);
+                    w[j] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const int q = base + 32 * j + lane;
+            if (q < n_items) dst[q] = w[j];
+        }
+    }
 }
 
 // mxf8 / 1D blocks: a stage covers 4 contraction blocks (one chunk); image row l holds rows l, l+32, l+64, l+96,
 // four scale bytes each.
 struct ScaleRegs1D { uint32_t w[3][4]; };
 
-__device__ __forceinline__ uint32_t load_scale_word(const ScaleView &v, int row, int kb0)
+__device__ __forceinline__ void load_scale_word(const ScaleView &v, int row, int kb0, uint32_t &dst)
 {
     const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
-    if (row < v.n_row && kb0 + 4 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 3) == 0)
-        return __ldg(reinterpret_cast<const uint32_t *>(ptr));
+    if (row < v.n_row && kb0 + 4 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 3) == 0) {
+        asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(dst) : "l"(ptr));   // the common case: nothing depends on it yet
+        return;
+    }
     uint32_t word = 0;
 #pragma unroll
-    for (int kb = 0; kb < 4; kb++) word |= (uint32_t)load_scale(v, row, kb0 + kb) << (8 * kb);
-    return word;
+    for (int kb = 0; kb < 4; kb++) {
+        uint32_t b;
+        load_scale(v, row, kb0 + kb, b);
+        word |= b << (8 * kb);
+    }
+    dst = word;
 }
 
-__device__ __forceinline__ ScaleRegs1D fetch_scales_1d(const GemmParams &p, const Tile &t, int it, int lane)
+__device__ __forceinline__ void fetch_scales_1d(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs1D &r)
 {
-    ScaleRegs1D r;
 #pragma unroll
     for (int blk = 0; blk < 3; blk++) {   // 0: A rows 0..127; 1, 2: B rows 0..127, 128..255
         const ScaleView &v = blk == 0 ? p.sfa : p.sfb;
         const int row0 = blk == 0 ? t.a_row0 : t.b_row0 + (blk - 1) * 128;
         const int kb0 = ((blk == 0 ? t.a_k0 : t.b_k0) >> 5) + it * 4;
 #pragma unroll
-        for (int j = 0; j < 4; j++) r.w[blk][j] = load_scale_word(v, row0 + lane + 32 * j, kb0);
+        for (int j = 0; j < 4; j++) load_scale_word(v, row0 + lane + 32 * j, kb0, r.w[blk][j]);
     }
-    return r;
 }
 
 __device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint8_t *sf_stage, int lane)
@@ -312,7 +509,6 @@ __device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint
     img[(kSfaOff >> 4) + lane] = make_uint4(r.w[0][0], r.w[0][1], r.w[0][2], r.w[0][3]);
     img[(kSfbOff >> 4) + lane] = make_uint4(r.w[1][0], r.w[1][1], r.w[1][2], r.w[1][3]);
     img[(kSfbOff >> 4) + 32 + lane] = make_uint4(r.w[2][0], r.w[2][1], r.w[2][2], r.w[2][3]);
-    __syncwarp();
 }
 
 template <int KIND> struct ScaleRegsOf { typedef ScaleRegs2D type; };
@@ -320,17 +516,19 @@ template <> struct ScaleRegsOf<KIND_MXF8> { typedef ScaleRegs1D type; };
 
 __device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs2D &r)
 {
-    r = fetch_scales_2d(p, t, it, lane);
+    fetch_scales_2d(p, t, it, lane, r);
 }
 __device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs1D &r)
 {
-    r = fetch_scales_1d(p, t, it, lane);
+    fetch_scales_1d(p, t, it, lane, r);
 }
-__device__ __forceinline__ void write_scale_images(const ScaleRegs2D &r, uint8_t *sf_stage, uint8_t *scratch, int lane)
+__device__ __forceinline__ void write_scale_images(const GemmParams &p, const Tile &t, int it, const ScaleRegs2D &r,
+                                                   uint8_t *sf_stage, uint8_t *scratch, int lane)
 {
-    write_scale_images_2d(r, sf_stage, scratch, lane);
+    write_scale_images_2d(p, t, it, r, sf_stage, scratch, lane);
 }
-__device__ __forceinline__ void write_scale_images(const ScaleRegs1D &r, uint8_t *sf_stage, uint8_t *, int lane)
+__device__ __forceinline__ void write_scale_images(const GemmParams &, const Tile &, int, const ScaleRegs1D &r,
+                                                   uint8_t *sf_stage, uint8_t *, int lane)
 {
     write_scale_images_1d(r, sf_stage, lane);
 }
@@ -398,23 +596,30 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
     uint8_t *smem_sf = smem + kSmemOperands;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kSmemOperands + kSmemSf);
-    // bars[0..3] full, bars[4..7] empty, bars[8] accumulator full, bars[9] accumulator empty
-    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 10);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 10) + 1;
-    uint8_t *scale_scratch = reinterpret_cast<uint8_t *>(bars + 12);    // 96 bytes, 16-byte aligned
+    uint8_t *smem_cache = smem + kSmemOperands + kSmemSf;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kSmemOperands + kSmemSf + kSmemCache);
+    // bars[0..3] full, bars[4..7] empty, bars[8] accumulator full, bars[9] accumulator empty,
+    // bars[10..11] scale cache full, bars[12..13] scale cache empty
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 14);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 14) + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *scale_scratch = reinterpret_cast<uint8_t *>(bars + 16) + 128 * (warp & 1);   // 96 bytes per loader warp
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
     const uint32_t bar_acc_full = smem_u32(bars + 8), bar_acc_empty = smem_u32(bars + 9);
+    const uint32_t bar_cache_full = smem_u32(bars + 10), bar_cache_empty = smem_u32(bars + 12);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) {
-            mbar_init(bar_full + 8 * s, 2);     // producer's expect_tx arrival + scale loader's arrival
+            mbar_init(bar_full + 8 * s, 2);     // producer's expect_tx arrival + the scale loader's tcgen05.commit
             mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
         }
         mbar_init(bar_acc_full, 1);
         mbar_init(bar_acc_empty, 8);            // one arrival per epilogue warp
+        for (int b = 0; b < 2; b++) {
+            mbar_init(bar_cache_full + 8 * b, 1);
+            mbar_init(bar_cache_empty + 8 * b, 1);
+        }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
@@ -440,7 +645,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 decode_tile(p, tile, t);
                 const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
                 for (int it = 0; it < n_it; it++) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage))) break;
+                    ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
+                    if (!ok) break;
                     mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
                     tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA,
                                 (t.a_k0 + it * kStageElems) / kElemsPerByte, t.a_row0, bar_full + 8 * stage);
@@ -466,7 +672,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             if (!ok) break;
             acc_phase ^= 1u;
-            tcgen05_fence_after();
             for (int it = 0; it < n_it; it++) {
                 if (lane == 0) ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x210u + stage);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
@@ -503,40 +708,115 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp == 2) {
-        // ------------------------------------------------------------------ scale loader
-        typename ScaleRegsOf<KIND>::type pre[kStages];
+    } else if ((warp == 2 || warp == 3) && KIND == KIND_MXF8) {
+        // ------------------------------------------------------------------ scale loaders, per-row scales (MXFP8)
+        // Two warps share the ring: warp 2 serves the even stages of the stream, warp 3 the odd ones (ring slots
+        // {0, 2} and {1, 3}).  Each fetches the scale words of its next two stages ahead of time and, for the stage
+        // at hand, writes the images and arrives on the stage's "full" barrier.
+        const int which = warp - 2;
+        typename ScaleRegsOf<KIND>::type pre[2];
         WorkIter fetch_it, write_it;
         fetch_it.tile = write_it.tile = blockIdx.x;
         fetch_it.seek(p, kStageElems);
         write_it.seek(p, kStageElems);
+        if (which == 1) {
+            if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
+            if (write_it.valid(p)) write_it.next(p, kStageElems);
+        }
 #pragma unroll
-        for (int d = 0; d < kStages; d++) {
+        for (int d = 0; d < 2; d++) {
             if (fetch_it.valid(p)) {
                 fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[d]);
                 fetch_it.next(p, kStageElems);
+                if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
             }
         }
         uint32_t phase = 0;
         bool ok = true;
         while (ok && write_it.valid(p)) {
 #pragma unroll
-            for (int stage = 0; stage < kStages; stage++) {
+            for (int d = 0; d < 2; d++) {
                 if (!write_it.valid(p)) break;
-                if (lane == 0) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
+                const int stage = 2 * d + which;
+                if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
-                write_scale_images(pre[stage], smem_sf + stage * kSfStageBytes, scale_scratch, lane);
+                write_scale_images(p, write_it.t, write_it.it, pre[d], smem_sf + stage * kSfStageBytes, scale_scratch, lane);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full + 8 * stage);
                 if (fetch_it.valid(p)) {
-                    fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[stage]);
+                    fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[d]);
                     fetch_it.next(p, kStageElems);
+                    if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
                 }
                 write_it.next(p, kStageElems);
+                if (write_it.valid(p)) write_it.next(p, kStageElems);
             }
             phase ^= 1u;
+        }
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ scale cache builder, 2D-block scales
+        // Per unit (a tile, or a 16384-element slice of a longer contraction) gathers every compact scale byte the
+        // unit needs into shared memory, already arranged as the 16-byte image rows: per 128-element chunk one row
+        // for A [row tile 0..3][block 0..3] and two for B (row tiles 0..3 and 4..7).  Two buffers alternate, so
+        // the next unit's scales are gathered while the current unit runs; all global-memory latency of the
+        // scale path is paid here, once per unit, off the per-stage critical path.
+        uint32_t unit = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            Tile t;
+            decode_tile(p, tile, t);
+            for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
+                const int buf = unit & 1;
+                if (lane == 0) ok = mbar_wait_lazy(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
+                uint32_t *cache = reinterpret_cast<uint32_t *>(smem_cache + buf * kCacheBytes);
+                build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, cache, lane);
+                build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, cache + kCacheChunks * 4, lane);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ scale image writer, 2D-block scales
+        // Per stage: six 16-byte rows from the scale cache, replicated over the 32 image rows tcgen05.cp expects.
+        uint32_t unit = 0, stage = 0, phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            Tile t;
+            decode_tile(p, tile, t);
+            for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
+                const int buf = unit & 1;
+                if (lane == 0) ok = mbar_wait_relaxed(bar_cache_full + 8 * buf, (unit >> 1) & 1u, abort_flag, p.status, 0x510u + buf);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                const uint4 *cache_a = reinterpret_cast<const uint4 *>(smem_cache + buf * kCacheBytes);
+                const uint4 *cache_b = cache_a + kCacheChunks;
+                const int n_stage = (min(kCacheChunks * 128, t.k_len - k0) + kStageElems - 1) / kStageElems;
+                for (int it = 0; it < n_stage; it++) {
+                    if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                    if (!ok) break;
+                    uint4 *img = reinterpret_cast<uint4 *>(smem_sf + stage * kSfStageBytes);
+                    const uint4 a0 = cache_a[2 * it], a1 = cache_a[2 * it + 1];
+                    const uint4 b0 = cache_b[4 * it], b1 = cache_b[4 * it + 1], b2 = cache_b[4 * it + 2], b3 = cache_b[4 * it + 3];
+                    img[(kSfaOff >> 4) + lane] = a0;             // SFA chunk 0
+                    img[(kSfaOff >> 4) + 32 + lane] = a1;        // SFA chunk 1
+                    img[(kSfbOff >> 4) + lane] = b0;             // SFB chunk 0, rows 0..127
+                    img[(kSfbOff >> 4) + 32 + lane] = b1;        // SFB chunk 0, rows 128..255
+                    img[(kSfbOff >> 4) + 64 + lane] = b2;        // SFB chunk 1, rows 0..127
+                    img[(kSfbOff >> 4) + 96 + lane] = b3;        // SFB chunk 1, rows 128..255
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_full + 8 * stage);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_cache_empty + 8 * buf);
+            }
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
@@ -552,7 +832,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const bool row_ok = row_in_tile < t.m_valid;
             uint32_t v[4][32];
             if (t.k_len > 0) {
-                if (lane == 0) ok = mbar_wait(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
+                if (lane == 0) ok = mbar_wait_lazy(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
                 acc_phase ^= 1u;
