@@ -65,7 +65,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(prefix="fp4q_clocks_", suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -486,6 +486,48 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_kernel(args):
+    """--kernel: one kernel on one shape, a few launches, for ncu captures and quick checks (one JSON line)."""
+    import torch
+    from paper_2607_24953_b200 import binding, workloads
+    dev = torch.device("cuda", 0)
+    dims = [int(v) for v in args.shape.lower().split("x")]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    if args.kernel == "quantize":
+        rows, cols = dims
+        x = workloads.activations_student_t(rows, cols, 1, dev)
+        out = binding.alloc_qtensor(rows, cols, dev)
+        fn = lambda: binding.fp4q_quantize2d(x, out, mode=args.mode, seed=3, tensor_id=1)
+        units, unit = rows * cols * BYTES_PER_ELEMENT / 1e9, "GB/s"
+    else:
+        T, N, K = dims
+        ws = binding.alloc_workspace(dev)
+        qx = binding.fp4q_quantize2d(workloads.activations_student_t(T, K, 1, dev), mode=1, seed=3, tensor_id=1)
+        qw = binding.fp4q_quantize2d(workloads.weights(N, K, 2, dev), mode=1, seed=3, tensor_id=0)
+        qdy = binding.fp4q_quantize2d(workloads.gradients_rowscaled(T, N, 3, dev), mode=1, seed=3, tensor_id=2)
+        if args.kernel == "gemm_fwd":
+            out = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+            fn = lambda: binding.fp4q_gemm_fwd(qx, qw, out=out, ws=ws)
+        elif args.kernel == "gemm_dgrad":
+            out = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
+            fn = lambda: binding.fp4q_gemm_dgrad(qdy, qw, out=out, ws=ws)
+        else:
+            out = torch.empty((N, K), dtype=torch.float32, device=dev)
+            fn = lambda: binding.fp4q_gemm_wgrad(qdy, qx, out=out, ws=ws)
+        units, unit = 2.0 * T * N * K / 1e12, "TFLOP/s"
+    fn()
+    torch.cuda.synchronize()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(args.iters):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.iters
+    print(json.dumps({"kernel": args.kernel, "shape": args.shape, "iters": args.iters, "ms": ms,
+                      "value": units / (ms * 1e-3), "unit": unit}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -496,8 +538,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad"],
+                    help="run one kernel on --shape a few times (for profiler captures) instead of the benchmark")
+    ap.add_argument("--shape", default="16384x4096", help="RxC for quantize, TxNxK for the GEMMs")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--mode", type=int, default=1, help="quantize rounding mode: 0 nearest, 1 stochastic")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.kernel:
+        run_kernel(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
