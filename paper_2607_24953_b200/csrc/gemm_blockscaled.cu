@@ -27,19 +27,28 @@
 
 namespace fp4q {
 
-constexpr int BM = 128, BN = 256;
-constexpr int kStages = 4;
+constexpr int BM = 128, BN = 256;            // per-CTA accumulator: 128 rows x 256 columns (a CTA pair covers 256 x 256)
+constexpr int kMaxStages = 6;
 constexpr int kAStageBytes = BM * 128;
-constexpr int kBStageBytes = BN * 128;
 constexpr int kSfStageBytes = 3072;          // SFA 2 x 512 B, SFB 2 x 1024 B
 constexpr int kSfaOff = 0, kSfbOff = 1024;
-constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
-constexpr int kSmemSf = kStages * kSfStageBytes;
 constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
 constexpr int kCacheChunks = 128;            // scale cache: contraction chunks of 128 elements per unit (16384 elements)
 constexpr int kCacheBytes = kCacheChunks * 48;   // per chunk: 16 B for A (4 row tiles x 4 blocks) + 32 B for B (8 x 4)
 constexpr int kSmemCache = 2 * kCacheBytes;
-constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemCache + kSmemTail;
+
+// CTAS = 1: one CTA per 128x256 tile, it loads all 256 B rows.  CTAS = 2: a cluster of two CTAs shares a 256x256
+// tile through cta_group::2 MMAs; each CTA loads its own 128 A rows and half of the B rows, which halves the
+// B-operand shared-memory and L2 traffic per CTA and leaves room for two more ring stages.
+template <int CTAS>
+struct Cfg {
+    static constexpr int kStages = CTAS == 2 ? 6 : 4;
+    static constexpr int kBRows = CTAS == 2 ? 128 : 256;
+    static constexpr int kBStageBytes = kBRows * 128;
+    static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
+    static constexpr int kSmemSf = kStages * kSfStageBytes;
+    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemCache + kSmemTail;
+};
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
@@ -49,6 +58,28 @@ constexpr uint32_t kWaitLimit = 1u << 22;
 #endif
 #ifndef FP4Q_LAZY_NS
 #define FP4Q_LAZY_NS 256
+#endif
+// Developer diagnostic (off by default): -DFP4Q_TRACE makes CTA 0 add up clock64() intervals of its roles in
+// registers and leave them in the workspace's padding words (status[16 + 2*slot], 64-bit each).
+#ifdef FP4Q_TRACE
+#define TRACE_DECL(n) long long n = 0
+#define TRACE_T0(t) long long t = clock64()
+#define TRACE_ADD(acc, t) do { long long t_now = clock64(); acc += t_now - t; t = t_now; } while (0)
+#define TRACE_OUT(p, slot, v) do { if (blockIdx.x == 0) reinterpret_cast<long long *>(p.status + 16)[slot] = (v); } while (0)
+#ifdef FP4Q_TRACE_EVENTS
+__device__ long long g_trace_events[2][8][512][2];   // [CTA 0/1][kind][stream index][clock64, globaltimer]
+#define TRACE_EV(kind, idx) do { if (blockIdx.x < 2 && (idx) < 512) { long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); \
+    g_trace_events[blockIdx.x][kind][idx][0] = clock64(); g_trace_events[blockIdx.x][kind][idx][1] = gt; } } while (0)
+extern "C" int fp4q_debug_events(void *host) { return (int)cudaMemcpyFromSymbol(host, g_trace_events, sizeof(g_trace_events)); }
+#else
+#define TRACE_EV(kind, idx)
+#endif
+#else
+#define TRACE_EV(kind, idx)
+#define TRACE_DECL(n)
+#define TRACE_T0(t)
+#define TRACE_ADD(acc, t)
+#define TRACE_OUT(p, slot, v)
 #endif
 constexpr uint8_t kScalePad = 127;           // UE8M0 code of 1.0 for scale slots beyond the tensor (their payload is 0)
 
@@ -68,7 +99,8 @@ struct GemmParams {
     void *C;
     int64_t ldc;
     int32_t M, N, K;                 // per-problem output rows, output columns, contraction length (elements)
-    int32_t m_tiles, n_tiles, n_tile_total;
+    int32_t m_tiles, n_tiles, n_tile_total;   // m_tiles counts rows of 128 * ctas
+    int32_t ctas;                    // CTAs per tile (1, or 2 for cta_group::2 pairs)
     int32_t out_f32, accumulate;
     int32_t mode, n_groups;
     const int64_t *row_offsets;
@@ -78,7 +110,7 @@ struct GemmParams {
 };
 
 struct Tile {
-    int32_t a_row0, b_row0, a_k0, b_k0, k_len, c_row0, c_col0, m_valid, n_valid;
+    int32_t a_row0, b_row0, b_load_row0, a_k0, b_k0, k_len, c_row0, c_col0, m_valid, n_valid;
 };
 
 // ---------------------------------------------------------------------------------------- PTX helpers
@@ -105,16 +137,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Non-blocking probe of a barrier phase (the try_wait form may suspend the thread for a while).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t p;
+    asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xFFFFFFFF;\n selp.b32 %0, 1, 0, P;\n}" : "=r"(p));
+    return p != 0;
+}
+// Named barrier on which the MMA warp and the warp that watches a ring slot for it meet (64 threads).  Both sides
+// use the waiting form: with a non-waiting arrival a watcher that releases stages unseen (after a timeout) could
+// complete a barrier phase on its own and leave the MMA warp without a partner.
+__device__ __forceinline__ void named_sync(uint32_t id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
+
 // Bounded wait.  Returns false when the limit ran out (the timeout is then recorded) or when another
 // role of this CTA has already given up.  Every poll of an mbarrier is a shared-memory transaction that
 // competes with the tensor core's operand reads and with the MMA thread's own waits, so roles that have
 // slack (everything but the MMA issuer) sleep between polls.
-template <int BACKOFF_NS>
+template <int BACKOFF_NS, bool PROBE = false>
 __device__ __forceinline__ bool mbar_wait_impl(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
                                                uint32_t where)
 {
     for (uint32_t it = 0; it < kWaitLimit; it++) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (PROBE ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
@@ -136,6 +188,13 @@ __device__ __noinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volat
 {
     return mbar_wait_impl<FP4Q_LAZY_NS>(bar, parity, abort_flag, status, where);
 }
+// For barriers that another CTA of the cluster completes (a multicast tcgen05.commit): probe instead of try_wait,
+// whose suspended thread is not reliably woken early by a remote arrival.
+__device__ __noinline__ bool mbar_poll_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                               uint32_t where)
+{
+    return mbar_wait_impl<FP4Q_RELAXED_NS, true>(bar, parity, abort_flag, status, where);
+}
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
 {
@@ -143,23 +202,65 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// The same load issued by either CTA of a pair: the bytes are counted on the barrier at this address in the
+// pair's leader CTA (cta_group::2 permits the barrier to live in the peer).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t leader_bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
+// shared::cluster address of this CTA's shared-memory location `addr` as seen in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 
+template <int CTAS>
 __device__ __forceinline__ void tcgen05_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {   // arrives on the barrier at this offset in both CTAs of the pair
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tcgen05_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc)
 {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+    if (CTAS == 1) asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+    else asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 
-template <int KIND>
+template <int KIND, int CTAS>
 __device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
 {
-    if (KIND == KIND_MXF4) {
+    if (KIND == KIND_MXF4 && CTAS == 2) {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
+    } else if (KIND == KIND_MXF4) {
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                      " tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
                      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
@@ -185,12 +286,12 @@ __device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
 }
 
 // Instruction descriptor of the block-scaled MMA: formats, K-major operands, N, UE8M0 scales, M, scale byte ids.
-template <int KIND>
+template <int KIND, int CTAS>
 __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_id)
 {
     const uint32_t fmt = KIND == KIND_MXF4 ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
     return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) |
-           ((uint32_t)(BM >> 4) << 24) | (a_sf_id << 29);
+           ((uint32_t)((BM * CTAS) >> 4) << 24) | (a_sf_id << 29);
 }
 
 #define FP4Q_TMEM_LD_X32(taddr, v)                                                                              \
@@ -216,14 +317,15 @@ __device__ __forceinline__ int find_group(const int64_t *offs, int n_groups, int
     return lo;
 }
 
-__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, Tile &t)
+__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int rank, Tile &t)
 {
     const int per_problem = p.m_tiles * p.n_tiles;
     const int g = p.mode == MODE_GROUPED_K ? tile / per_problem : 0;
     const int local = tile - g * per_problem;
     const int m_blk = local % p.m_tiles, n_blk = local / p.m_tiles;
-    t.a_row0 = m_blk * BM;
+    t.a_row0 = (m_blk * p.ctas + rank) * BM;
     t.b_row0 = n_blk * BN;
+    t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * 128 : 0);
     t.a_k0 = t.b_k0 = 0;
     t.k_len = p.K;
     t.c_row0 = t.a_row0;
@@ -233,6 +335,7 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, Tile 
     if (p.mode == MODE_GROUPED_ROWS) {
         const int grp = find_group(p.row_offsets, p.n_groups, (int64_t)t.a_row0);
         t.b_row0 += grp * p.b_rows_per_group;
+        t.b_load_row0 += grp * p.b_rows_per_group;
         t.b_k0 = grp * p.b_k_per_group;
     } else if (p.mode == MODE_GROUPED_K) {
         const int64_t k0 = __ldg(p.row_offsets + g), k1 = __ldg(p.row_offsets + g + 1);
@@ -257,88 +360,35 @@ __device__ __forceinline__ void load_scale(const ScaleView &v, int row, int kb, 
     asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(dst) : "l"(ptr));
 }
 
-// The scale loader runs ahead of the ring: the compact scale bytes of a stage are fetched into registers
-// kStages iterations before its image is written, so that the global-memory latency is off the critical path.
-struct WorkIter {
-    int tile, it, n_it;
+// The stream of ring stages one CTA works through: its tiles in order, each with its contraction stages.
+struct StageIter {
+    int tile, step, rank, it, n_it;
     Tile t;
     __device__ __forceinline__ void seek(const GemmParams &p, int stage_elems)
     {
         while (tile < p.n_tile_total) {
-            decode_tile(p, tile, t);
+            decode_tile(p, tile, rank, t);
             n_it = (t.k_len + stage_elems - 1) / stage_elems;
             if (n_it > 0) { it = 0; return; }
-            tile += gridDim.x;
+            tile += step;
         }
         n_it = 0;
+    }
+    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, int stage_elems)
+    {
+        tile = first; step = step_; rank = rank_; it = 0;
+        seek(p, stage_elems);
     }
     __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
     __device__ __forceinline__ void next(const GemmParams &p, int stage_elems)
     {
-        if (++it >= n_it) { tile += gridDim.x; seek(p, stage_elems); }
+        if (++it >= n_it) { tile += step; seek(p, stage_elems); }
     }
 };
 
-// mxf4 / 2D blocks: a stage covers 8 contraction blocks (two chunks of 4).  For 128 operand rows and one chunk
-// the image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3]; A needs 2 such rows per stage (one per
-// chunk), B (256 rows) 4.  The compact bytes are fetched with wide loads that every lane issues to the same
-// address (one broadcast transaction): 8 bytes along the contraction per row tile when the scale matrix is read
-// as stored, or the 4 / 8 row-tile bytes of one contraction block when it is read transposed (then a 4x4 byte
-// transpose in registers forms the rows).  Tiles at the edge of the scale matrix or with unaligned scales fall
-// back to one byte per lane gathered through a small shared-memory scratch.
-enum { SF_BYTES = 0, SF_ALONG_K = 1, SF_ALONG_ROWS = 2 };
-struct ScaleRegs2D { uint32_t a[8], b[16]; };
-
-__device__ __forceinline__ int scale_mode_2d(const ScaleView &v, int rt0, int n_rt, int kb0)
-{
-    if (rt0 + n_rt > v.n_row || kb0 + 8 > v.n_kb) return SF_BYTES;
-    const uintptr_t base = reinterpret_cast<uintptr_t>(v.ptr);
-    if (v.stride_kb == 1)
-        return (((base + (uintptr_t)rt0 * v.stride_row + kb0) & 7) == 0 && (v.stride_row & 7) == 0) ? SF_ALONG_K : SF_BYTES;
-    if (v.stride_row == 1)
-        return (((base + (uintptr_t)kb0 * v.stride_kb + rt0) & (n_rt - 1)) == 0 && (v.stride_kb & (n_rt - 1)) == 0)
-                   ? SF_ALONG_ROWS : SF_BYTES;
-    return SF_BYTES;
-}
-
-__device__ __forceinline__ void ldg_b64(const uint8_t *ptr, uint32_t &lo, uint32_t &hi)
-{
-    asm volatile("ld.global.nc.v2.b32 {%0, %1}, [%2];" : "=r"(lo), "=r"(hi) : "l"(ptr));
-}
 __device__ __forceinline__ void ldg_b32(const uint8_t *ptr, uint32_t &w)
 {
     asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(w) : "l"(ptr));
-}
-
-__device__ __forceinline__ void fetch_scales_2d(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs2D &r)
-{
-    const int a_rt0 = t.a_row0 >> 5, a_kb0 = (t.a_k0 >> 5) + it * 8;
-    const int b_rt0 = t.b_row0 >> 5, b_kb0 = (t.b_k0 >> 5) + it * 8;
-    const int ma = scale_mode_2d(p.sfa, a_rt0, 4, a_kb0), mb = scale_mode_2d(p.sfb, b_rt0, 8, b_kb0);
-    if (ma == SF_ALONG_K) {
-#pragma unroll
-        for (int rt = 0; rt < 4; rt++)
-            ldg_b64(p.sfa.ptr + (int64_t)(a_rt0 + rt) * p.sfa.stride_row + a_kb0, r.a[2 * rt], r.a[2 * rt + 1]);
-    } else if (ma == SF_ALONG_ROWS) {
-#pragma unroll
-        for (int kb = 0; kb < 8; kb++) ldg_b32(p.sfa.ptr + (int64_t)(a_kb0 + kb) * p.sfa.stride_kb + a_rt0, r.a[kb]);
-    } else {
-        const int c = lane >> 4, rt = (lane >> 2) & 3, kb = lane & 3;
-        load_scale(p.sfa, a_rt0 + rt, a_kb0 + c * 4 + kb, r.a[0]);
-    }
-    if (mb == SF_ALONG_K) {
-#pragma unroll
-        for (int rt = 0; rt < 8; rt++)
-            ldg_b64(p.sfb.ptr + (int64_t)(b_rt0 + rt) * p.sfb.stride_row + b_kb0, r.b[2 * rt], r.b[2 * rt + 1]);
-    } else if (mb == SF_ALONG_ROWS) {
-#pragma unroll
-        for (int kb = 0; kb < 8; kb++)
-            ldg_b64(p.sfb.ptr + (int64_t)(b_kb0 + kb) * p.sfb.stride_kb + b_rt0, r.b[2 * kb], r.b[2 * kb + 1]);
-    } else {
-        const int rt = (lane >> 2) & 7, kb = lane & 3;
-        load_scale(p.sfb, b_rt0 + rt, b_kb0 + kb, r.b[0]);       // chunk 0
-        load_scale(p.sfb, b_rt0 + rt, b_kb0 + 4 + kb, r.b[1]);   // chunk 1
-    }
 }
 
 // Rows of a 4x4 byte matrix given by its columns: w[k] holds byte rt of column k in byte lane rt.
@@ -350,52 +400,9 @@ __device__ __forceinline__ uint4 transpose4x4_bytes(uint32_t w0, uint32_t w1, ui
                       __byte_perm(t2, t3, 0x7632));
 }
 
-__device__ __forceinline__ void write_scale_images_2d(const GemmParams &p, const Tile &t, int it, const ScaleRegs2D &r,
-                                                      uint8_t *sf_stage, uint8_t *scratch, int lane)
-{
-    const int a_rt0 = t.a_row0 >> 5, a_kb0 = (t.a_k0 >> 5) + it * 8;
-    const int b_rt0 = t.b_row0 >> 5, b_kb0 = (t.b_k0 >> 5) + it * 8;
-    const int ma = scale_mode_2d(p.sfa, a_rt0, 4, a_kb0), mb = scale_mode_2d(p.sfb, b_rt0, 8, b_kb0);
-    uint4 rows[6];   // SFA chunk 0, 1; SFB chunk 0 rows 0..127, 128..255; SFB chunk 1 rows 0..127, 128..255
-    if (ma == SF_BYTES || mb == SF_BYTES) {
-        if (ma == SF_BYTES) scratch[lane] = (uint8_t)r.a[0];            // [chunk][row tile 0..3][block]
-        if (mb == SF_BYTES) {
-            scratch[32 + lane] = (uint8_t)r.b[0];                       // chunk 0: [row tile 0..7][block]
-            scratch[64 + lane] = (uint8_t)r.b[1];                       // chunk 1
-        }
-        __syncwarp();
-        const uint4 *s4 = reinterpret_cast<const uint4 *>(scratch);
-#pragma unroll
-        for (int q = 0; q < 6; q++) rows[q] = s4[q];
-        __syncwarp();
-    }
-    if (ma == SF_ALONG_K) {
-        rows[0] = make_uint4(r.a[0], r.a[2], r.a[4], r.a[6]);
-        rows[1] = make_uint4(r.a[1], r.a[3], r.a[5], r.a[7]);
-    } else if (ma == SF_ALONG_ROWS) {
-        rows[0] = transpose4x4_bytes(r.a[0], r.a[1], r.a[2], r.a[3]);
-        rows[1] = transpose4x4_bytes(r.a[4], r.a[5], r.a[6], r.a[7]);
-    }
-    if (mb == SF_ALONG_K) {
-        rows[2] = make_uint4(r.b[0], r.b[2], r.b[4], r.b[6]);
-        rows[3] = make_uint4(r.b[8], r.b[10], r.b[12], r.b[14]);
-        rows[4] = make_uint4(r.b[1], r.b[3], r.b[5], r.b[7]);
-        rows[5] = make_uint4(r.b[9], r.b[11], r.b[13], r.b[15]);
-    } else if (mb == SF_ALONG_ROWS) {
-        rows[2] = transpose4x4_bytes(r.b[0], r.b[2], r.b[4], r.b[6]);
-        rows[3] = transpose4x4_bytes(r.b[1], r.b[3], r.b[5], r.b[7]);
-        rows[4] = transpose4x4_bytes(r.b[8], r.b[10], r.b[12], r.b[14]);
-        rows[5] = transpose4x4_bytes(r.b[9], r.b[11], r.b[13], r.b[15]);
-    }
-    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
-    img[(kSfaOff >> 4) + lane] = rows[0];
-    img[(kSfaOff >> 4) + 32 + lane] = rows[1];
-    img[(kSfbOff >> 4) + lane] = rows[2];
-    img[(kSfbOff >> 4) + 32 + lane] = rows[3];
-    img[(kSfbOff >> 4) + 64 + lane] = rows[4];
-    img[(kSfbOff >> 4) + 96 + lane] = rows[5];
-}
-
+// mxf4 / 2D blocks: a stage covers 8 contraction blocks (two chunks of 4).  For 128 operand rows and one chunk the
+// scale image is 32 identical rows of 16 bytes [row tile 0..3][block 0..3]; A needs 2 such rows per stage (one per
+// chunk), B (256 rows) 4.
 // Gathers the scale bytes of n_chunks contraction chunks (4 blocks each) for 2^log2_rt consecutive row tiles into
 // dst[(chunk << log2_rt) + rt] as 32-bit words (byte k = block 4*chunk + k): the 16-byte image rows of the chunk.
 // One warp; each lane takes items lane, lane + 32, ...  Slots beyond the tensor read the pad byte.
@@ -511,28 +518,6 @@ __device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint
     img[(kSfbOff >> 4) + 32 + lane] = make_uint4(r.w[2][0], r.w[2][1], r.w[2][2], r.w[2][3]);
 }
 
-template <int KIND> struct ScaleRegsOf { typedef ScaleRegs2D type; };
-template <> struct ScaleRegsOf<KIND_MXF8> { typedef ScaleRegs1D type; };
-
-__device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs2D &r)
-{
-    fetch_scales_2d(p, t, it, lane, r);
-}
-__device__ __forceinline__ void fetch_scales(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs1D &r)
-{
-    fetch_scales_1d(p, t, it, lane, r);
-}
-__device__ __forceinline__ void write_scale_images(const GemmParams &p, const Tile &t, int it, const ScaleRegs2D &r,
-                                                   uint8_t *sf_stage, uint8_t *scratch, int lane)
-{
-    write_scale_images_2d(p, t, it, r, sf_stage, scratch, lane);
-}
-__device__ __forceinline__ void write_scale_images(const GemmParams &, const Tile &, int, const ScaleRegs1D &r,
-                                                   uint8_t *sf_stage, uint8_t *, int lane)
-{
-    write_scale_images_1d(r, sf_stage, lane);
-}
-
 // ---------------------------------------------------------------------------------------- epilogue store
 
 __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row, int col0, int n_cols_valid,
@@ -582,7 +567,7 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
 
 // ---------------------------------------------------------------------------------------- kernel
 
-template <int KIND>
+template <int KIND, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ GemmParams p)
@@ -590,32 +575,42 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kStageElems = KIND == KIND_MXF4 ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = KIND == KIND_MXF4 ? 64 : 32;           // contraction elements per MMA (32 B per row)
     constexpr int kElemsPerByte = KIND == KIND_MXF4 ? 2 : 1;
+    constexpr int kStages = Cfg<CTAS>::kStages;
+    constexpr int kBStageBytes = Cfg<CTAS>::kBStageBytes;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_sf = smem + kSmemOperands;
-    uint8_t *smem_cache = smem + kSmemOperands + kSmemSf;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kSmemOperands + kSmemSf + kSmemCache);
-    // bars[0..3] full, bars[4..7] empty, bars[8] accumulator full, bars[9] accumulator empty,
-    // bars[10..11] scale cache full, bars[12..13] scale cache empty
-    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 14);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 14) + 1;
+    uint8_t *smem_sf = smem + Cfg<CTAS>::kSmemOperands;
+    uint8_t *smem_cache = smem_sf + Cfg<CTAS>::kSmemSf;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_cache + kSmemCache);
+    // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
+    // bars[14..15] scale cache full, bars[16..17] scale cache empty, bars[18] tensor pipe drained (abort path)
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 19);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 19) + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint8_t *scale_scratch = reinterpret_cast<uint8_t *>(bars + 16) + 128 * (warp & 1);   // 96 bytes per loader warp
-    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kStages);
-    const uint32_t bar_acc_full = smem_u32(bars + 8), bar_acc_empty = smem_u32(bars + 9);
-    const uint32_t bar_cache_full = smem_u32(bars + 10), bar_cache_empty = smem_u32(bars + 12);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
+    const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
+    const uint32_t bar_cache_full = smem_u32(bars + 14), bar_cache_empty = smem_u32(bars + 16);
+    const uint32_t bar_drain = smem_u32(bars + 18);
+
+    // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
+    const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
+    const bool leader = rank == 0;
+    const int first_tile = blockIdx.x / CTAS, tile_step = gridDim.x / CTAS;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) {
-            mbar_init(bar_full + 8 * s, 2);     // producer's expect_tx arrival + the scale loader's tcgen05.commit
+            // The producer's expect_tx arrival; in the leader of a pair also the arrival by which the second CTA's
+            // watcher reports that CTA's operands and scale images.  The watcher of the stage waits on it.
+            mbar_init(bar_full + 8 * s, (CTAS == 2 && leader) ? 2 : 1);
             mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
         }
         mbar_init(bar_acc_full, 1);
-        mbar_init(bar_acc_empty, 8);            // one arrival per epilogue warp
+        mbar_init(bar_drain, 1);
+        mbar_init(bar_acc_empty, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
         for (int b = 0; b < 2; b++) {
             mbar_init(bar_cache_full + 8 * b, 1);
             mbar_init(bar_cache_empty + 8 * b, 1);
@@ -626,12 +621,20 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_slot)),
-                     "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CTAS == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_slot)),
+                         "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_slot)),
+                         "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tcgen05_fence_before();
-    __syncthreads();
+    __syncwarp();
+    if (CTAS == 2) cluster_sync_all();   // the peer's barriers must exist before anything is signalled across CTAs
+    else __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
 
@@ -640,52 +643,76 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+            int ev_j = 0;
+            TRACE_DECL(c_empty); TRACE_DECL(c_issue);
+            TRACE_T0(tt);
+            for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
                 Tile t;
-                decode_tile(p, tile, t);
+                decode_tile(p, tile, rank, t);
                 const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
                 for (int it = 0; it < n_it; it++) {
-                    ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
+                    TRACE_ADD(c_issue, tt);
+                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage)
+                                   : mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
+                    TRACE_ADD(c_empty, tt);
+                    TRACE_EV(0, ev_j);
                     if (!ok) break;
+                    const int xa = (t.a_k0 + it * kStageElems) / kElemsPerByte, xb = (t.b_k0 + it * kStageElems) / kElemsPerByte;
+                    // each CTA counts its own bytes on its own barrier (in a pair the second CTA's watcher forwards)
                     mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
-                    tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA,
-                                (t.a_k0 + it * kStageElems) / kElemsPerByte, t.a_row0, bar_full + 8 * stage);
-                    tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB,
-                                (t.b_k0 + it * kStageElems) / kElemsPerByte, t.b_row0, bar_full + 8 * stage);
+                    tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, bar_full + 8 * stage);
+                    tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
+                    TRACE_EV(1, ev_j);
+                    ev_j++;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {   // give copies already in flight time to land before the CTA's shared memory is released
                 for (int i = 0; i < 200; i++) __nanosleep(1000);
             }
+            TRACE_OUT(p, 0, c_empty);
+            TRACE_OUT(p, 1, c_issue);
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        uint32_t stage = 0, phase = 0, acc_phase = 0;
+        // ------------------------------------------------------------------ MMA issuer (the leader CTA of a pair)
+        // The warp stays converged and one elected lane issues the tcgen05 instructions: their descriptors then live
+        // in uniform registers, and a scale copy costs about ten cycles of the issuing thread instead of fifty.  The
+        // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
+        // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
+        // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
+        uint32_t stage = 0, acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+        const bool issuer = elect_one();
+        int ev_j = 0;
+        TRACE_DECL(c_acc); TRACE_DECL(c_sync); TRACE_DECL(c_issue);
+        TRACE_T0(tt);
+        for (int tile = first_tile; leader && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, t);
+            decode_tile(p, tile, rank, t);
             const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
             if (n_it == 0) continue;
-            if (lane == 0) ok = mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
-            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-            if (!ok) break;
-            acc_phase ^= 1u;
+            if (KIND == KIND_MXF8) {   // per-row scales: the watchers alternate stages, so the accumulator is awaited here
+                if (ok) {
+                    if (lane == 0) ok = mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                }
+                acc_phase ^= 1u;
+            }
+            TRACE_ADD(c_acc, tt);
             for (int it = 0; it < n_it; it++) {
-                if (lane == 0) ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x210u + stage);
-                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                if (!ok) break;
-                if (lane == 0) {
-                    tcgen05_fence_after();
+                named_sync(1 + stage);   // the watcher has seen the operands and both scale images of this stage
+                tcgen05_fence_after();
+                TRACE_ADD(c_sync, tt);
+                if (lane == 0) TRACE_EV(2, ev_j);
+                if (issuer) {
                     const uint32_t sf_smem = smem_u32(smem_sf + stage * kSfStageBytes);
                     const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
                     constexpr int kChunks = KIND == KIND_MXF4 ? 2 : 1;
 #pragma unroll
                     for (int c = 0; c < kChunks; c++) {
-                        tcgen05_cp_32x128b_warpx4(sf_tmem + 4 * c, smem_desc_scale_image(sf_smem + kSfaOff + 512 * c));
-                        tcgen05_cp_32x128b_warpx4(sf_tmem + 8 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c));
-                        tcgen05_cp_32x128b_warpx4(sf_tmem + 12 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c + 512));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image(sf_smem + kSfaOff + 512 * c));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c + 512));
                     }
                     const uint64_t adesc = smem_desc_sw128(smem_u32(smem_a + stage * kAStageBytes));
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(smem_b + stage * kBStageBytes));
@@ -696,29 +723,41 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         if (i < n_mma) {
                             const int chunk = KIND == KIND_MXF4 ? (i >> 1) : 0;
                             const uint32_t sf_id = KIND == KIND_MXF4 ? 2u * (i & 1) : (uint32_t)i;
-                            tcgen05_mma_block_scaled<KIND>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
-                                                           instr_desc<KIND>(sf_id, sf_id), sf_tmem + 4 * chunk,
-                                                           sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
+                            tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
+                                                                 instr_desc<KIND, CTAS>(sf_id, sf_id), sf_tmem + 4 * chunk,
+                                                                 sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
                         }
                     }
-                    tcgen05_commit(bar_empty + 8 * stage);
-                    if (it == n_it - 1) tcgen05_commit(bar_acc_full);
+                    tcgen05_commit<CTAS>(bar_empty + 8 * stage);
+                    if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
                 }
-                __syncwarp();
-                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                TRACE_ADD(c_issue, tt);
+                if (lane == 0) TRACE_EV(3, ev_j);
+                ev_j++;
+                if (++stage == kStages) stage = 0;
             }
         }
+        if (leader && *abort_flag) {
+            // Some role gave up: the watchers then release every remaining stage unseen, and this warp has run
+            // through them.  Wait (bounded) until the tensor pipe is idle before tensor memory is freed.
+            if (issuer) tcgen05_commit<CTAS>(bar_drain);
+            __syncwarp();
+            if (lane == 0) mbar_wait_lazy(bar_drain, 0u, abort_flag, p.status, 0x220u);   // gives up after 256 polls (abort is set)
+            __syncwarp();
+        }
+        if (lane == 0) { TRACE_OUT(p, 2, c_acc); TRACE_OUT(p, 3, c_sync); TRACE_OUT(p, 4, c_issue); }
     } else if ((warp == 2 || warp == 3) && KIND == KIND_MXF8) {
         // ------------------------------------------------------------------ scale loaders, per-row scales (MXFP8)
         // Two warps share the ring: warp 2 serves the even stages of the stream, warp 3 the odd ones (ring slots
         // {0, 2} and {1, 3}).  Each fetches the scale words of its next two stages ahead of time and, for the stage
-        // at hand, writes the images and arrives on the stage's "full" barrier.
+        // at hand, writes the images, waits for the operands ("full") and releases the MMA warp through the stage's
+        // named barrier.  After a timeout the remaining stages are released without waiting, so that the MMA warp,
+        // which cannot time out on a named barrier, always runs to its end.  (One CTA per tile only.)
         const int which = warp - 2;
-        typename ScaleRegsOf<KIND>::type pre[2];
-        WorkIter fetch_it, write_it;
-        fetch_it.tile = write_it.tile = blockIdx.x;
-        fetch_it.seek(p, kStageElems);
-        write_it.seek(p, kStageElems);
+        ScaleRegs1D pre[2];
+        StageIter fetch_it, write_it;
+        fetch_it.init(p, first_tile, tile_step, rank, kStageElems);
+        write_it.init(p, first_tile, tile_step, rank, kStageElems);
         if (which == 1) {
             if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
             if (write_it.valid(p)) write_it.next(p, kStageElems);
@@ -726,27 +765,32 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
         for (int d = 0; d < 2; d++) {
             if (fetch_it.valid(p)) {
-                fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[d]);
+                fetch_scales_1d(p, fetch_it.t, fetch_it.it, lane, pre[d]);
                 fetch_it.next(p, kStageElems);
                 if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
             }
         }
         uint32_t phase = 0;
         bool ok = true;
-        while (ok && write_it.valid(p)) {
+        while (write_it.valid(p)) {
 #pragma unroll
             for (int d = 0; d < 2; d++) {
                 if (!write_it.valid(p)) break;
                 const int stage = 2 * d + which;
-                if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
-                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                if (!ok) break;
-                write_scale_images(p, write_it.t, write_it.it, pre[d], smem_sf + stage * kSfStageBytes, scale_scratch, lane);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_full + 8 * stage);
-                if (fetch_it.valid(p)) {
-                    fetch_scales(p, fetch_it.t, fetch_it.it, lane, pre[d]);
+                if (ok) {
+                    if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                }
+                if (ok) {
+                    write_scale_images_1d(pre[d], smem_sf + stage * kSfStageBytes, lane);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
+                    __syncwarp();
+                    if (lane == 0) ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x310u + stage);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                }
+                named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
+                if (ok && fetch_it.valid(p)) {
+                    fetch_scales_1d(p, fetch_it.t, fetch_it.it, lane, pre[d]);
                     fetch_it.next(p, kStageElems);
                     if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
                 }
@@ -761,12 +805,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // unit needs into shared memory, already arranged as the 16-byte image rows: per 128-element chunk one row
         // for A [row tile 0..3][block 0..3] and two for B (row tiles 0..3 and 4..7).  Two buffers alternate, so
         // the next unit's scales are gathered while the current unit runs; all global-memory latency of the
-        // scale path is paid here, once per unit, off the per-stage critical path.
+        // scale path is paid here, once per unit, off the per-stage critical path.  In a pair each CTA gathers the
+        // scales of its own 128 A rows and of all 256 B rows.
         uint32_t unit = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+        for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, t);
+            decode_tile(p, tile, rank, t);
             for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
                 const int buf = unit & 1;
                 if (lane == 0) ok = mbar_wait_lazy(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
@@ -781,28 +826,46 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
         }
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ scale image writer, 2D-block scales
-        // Per stage: six 16-byte rows from the scale cache, replicated over the 32 image rows tcgen05.cp expects.
-        uint32_t unit = 0, stage = 0, phase = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
-            Tile t;
-            decode_tile(p, tile, t);
-            for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
+        // ------------------------------------------------------------------ scale image writer and watcher, 2D-block scales
+        // Two cursors run over this CTA's stream of stages.  The writing cursor waits for a ring slot to be free,
+        // copies six 16-byte rows from the scale cache into the slot's images (each replicated over the 32 image
+        // rows tcgen05.cp expects) and, in the second CTA of a pair, arrives on the leader's "full" barrier.  The
+        // signalling cursor (one CTA, or the leader) waits for the slot's "full" barrier - the operand bytes of
+        // both CTAs and the peer's images - and, at the first stage of a tile, for the accumulator to be drained,
+        // then meets the MMA warp at the slot's named barrier.  Neither cursor waits on an mbarrier: both
+        // conditions are probed, so a slot can be filled while an earlier one is still in flight.  After a timeout every remaining stage is released unseen, so
+        // that the MMA warp, which cannot time out on a named barrier, always runs to its end.
+        constexpr int kUnitStages = kCacheChunks * 128 / kStageElems;
+        const bool signals = CTAS == 1 || leader;
+        StageIter wr, sg;
+        wr.init(p, first_tile, tile_step, rank, kStageElems);
+        sg = wr;
+        uint32_t wstage = 0, wphase = 0, sstage = 0, sphase = 0, acc_phase = 0, unit = 0;
+        uint32_t n_written = 0, n_signalled = 0, idle = 0;
+        bool unit_open = false, ok = true;
+        TRACE_DECL(c_write); TRACE_DECL(c_meet); TRACE_DECL(c_poll);
+        TRACE_T0(tt);
+        while (sg.valid(p) && (signals || ok)) {
+            bool progress = false;
+            if (ok && wr.valid(p)) {
                 const int buf = unit & 1;
-                if (lane == 0) ok = mbar_wait_relaxed(bar_cache_full + 8 * buf, (unit >> 1) & 1u, abort_flag, p.status, 0x510u + buf);
-                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                if (!ok) break;
-                const uint4 *cache_a = reinterpret_cast<const uint4 *>(smem_cache + buf * kCacheBytes);
-                const uint4 *cache_b = cache_a + kCacheChunks;
-                const int n_stage = (min(kCacheChunks * 128, t.k_len - k0) + kStageElems - 1) / kStageElems;
-                for (int it = 0; it < n_stage; it++) {
-                    if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
-                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                    if (!ok) break;
-                    uint4 *img = reinterpret_cast<uint4 *>(smem_sf + stage * kSfStageBytes);
-                    const uint4 a0 = cache_a[2 * it], a1 = cache_a[2 * it + 1];
-                    const uint4 b0 = cache_b[4 * it], b1 = cache_b[4 * it + 1], b2 = cache_b[4 * it + 2], b3 = cache_b[4 * it + 3];
+                bool ready = false;
+                if (lane == 0) {
+                    ready = mbar_test_wait(bar_empty + 8 * wstage, wphase ^ 1u);
+                    if (ready && !unit_open) ready = mbar_test_wait(bar_cache_full + 8 * buf, (unit >> 1) & 1u);
+                }
+                ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
+                TRACE_ADD(c_poll, tt);
+                if (ready) {
+                    if (lane == 0) TRACE_EV(4, (int)n_written);
+                    unit_open = true;
+                    const int in_unit = wr.it & (kUnitStages - 1);
+                    const uint4 *cache_a = reinterpret_cast<const uint4 *>(smem_cache + buf * kCacheBytes);
+                    const uint4 *cache_b = cache_a + kCacheChunks;
+                    uint4 *img = reinterpret_cast<uint4 *>(smem_sf + wstage * kSfStageBytes);
+                    const uint4 a0 = cache_a[2 * in_unit], a1 = cache_a[2 * in_unit + 1];
+                    const uint4 b0 = cache_b[4 * in_unit], b1 = cache_b[4 * in_unit + 1];
+                    const uint4 b2 = cache_b[4 * in_unit + 2], b3 = cache_b[4 * in_unit + 3];
                     img[(kSfaOff >> 4) + lane] = a0;             // SFA chunk 0
                     img[(kSfaOff >> 4) + 32 + lane] = a1;        // SFA chunk 1
                     img[(kSfbOff >> 4) + lane] = b0;             // SFB chunk 0, rows 0..127
@@ -811,29 +874,76 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     img[(kSfbOff >> 4) + 96 + lane] = b3;        // SFB chunk 1, rows 128..255
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_full + 8 * stage);
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    if (lane == 0 && (in_unit == kUnitStages - 1 || wr.it == wr.n_it - 1)) mbar_arrive(bar_cache_empty + 8 * buf);
+                    if (in_unit == kUnitStages - 1 || wr.it == wr.n_it - 1) { unit++; unit_open = false; }
+                    if (lane == 0) TRACE_EV(5, (int)n_written);
+                    if (++wstage == kStages) { wstage = 0; wphase ^= 1u; }
+                    wr.next(p, kStageElems);
+                    n_written++;
+                    progress = true;
+                    TRACE_ADD(c_write, tt);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_cache_empty + 8 * buf);
+            }
+            if (n_signalled < n_written || !ok) {
+                bool ready = true;
+                if (ok) {
+                    if (lane == 0) {
+                        ready = mbar_test_wait(bar_full + 8 * sstage, sphase);
+                        if (ready && signals && sg.it == 0) ready = mbar_test_wait(bar_acc_empty, acc_phase ^ 1u);
+                    }
+                    ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
+                }
+                TRACE_ADD(c_poll, tt);
+                if (ready) {
+                    if (lane == 0) TRACE_EV(6, (int)n_signalled);
+                    if (signals) named_sync(1 + sstage);   // rendezvous: the MMA warp is at most one stage behind
+                    else if (lane == 0) mbar_arrive_cluster(cluster_addr(bar_full + 8 * sstage, 0));   // this CTA's half is in place
+                    TRACE_ADD(c_meet, tt);
+                    if (sg.it == 0) acc_phase ^= 1u;
+                    if (++sstage == kStages) { sstage = 0; sphase ^= 1u; }
+                    sg.next(p, kStageElems);
+                    n_signalled++;
+                    progress = true;
+                }
+            }
+            if (progress) {
+                idle = 0;
+            } else if (ok) {
+                if (++idle >= kWaitLimit) {
+                    ok = false;
+                    if (lane == 0) {
+                        *abort_flag = 1u;
+                        if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = 0x300u + sstage;
+                    }
+                } else if ((idle & 255u) == 255u && *abort_flag) {
+                    ok = false;
+                }
             }
         }
+        if (lane == 0) { TRACE_OUT(p, 5, c_write); TRACE_OUT(p, 6, c_meet); TRACE_OUT(p, 7, c_poll); }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 (hardware: warp id mod 4)
         const int half = (warp - 4) >> 2;        // accumulator columns 128*half .. +127
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.n_tile_total; tile += gridDim.x) {
+        int ev_t = 0;
+        TRACE_DECL(c_wait); TRACE_DECL(c_ld); TRACE_DECL(c_store);
+        TRACE_T0(tt);
+        for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, t);
+            decode_tile(p, tile, rank, t);
             const int row_in_tile = 32 * quarter + lane;
             const int64_t row = (int64_t)t.c_row0 + row_in_tile;
             const bool row_ok = row_in_tile < t.m_valid;
             uint32_t v[4][32];
             if (t.k_len > 0) {
-                if (lane == 0) ok = mbar_wait_lazy(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
+                if (lane == 0)
+                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp)
+                                   : mbar_wait_lazy(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                TRACE_ADD(c_wait, tt);
+                if (lane == 0) TRACE_EV(7, 16 * ev_t + 2 * (warp - 4));
                 if (!ok) break;
                 acc_phase ^= 1u;
                 tcgen05_fence_after();
@@ -845,7 +955,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acc_empty);     // the accumulator now lives in registers
+                if (lane == 0) {   // the accumulator now lives in registers; the leader's MMA thread waits for both CTAs
+                    if (CTAS == 1 || leader) mbar_arrive(bar_acc_empty);
+                    else mbar_arrive_cluster(cluster_addr(bar_acc_empty, 0));
+                }
+                TRACE_ADD(c_ld, tt);
+                if (lane == 0) TRACE_EV(7, 16 * ev_t + 2 * (warp - 4) + 1);
+                ev_t++;
             } else {
 #pragma unroll
                 for (int j = 0; j < 4; j++)
@@ -859,14 +975,21 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     store_row_chunk(p, row, t.c_col0 + col_in_tile, t.n_valid - col_in_tile, v[j]);
                 }
             }
+            TRACE_ADD(c_store, tt);
         }
+        if (warp == 4 && lane == 0) { TRACE_OUT(p, 8, c_wait); TRACE_OUT(p, 9, c_ld); TRACE_OUT(p, 10, c_store); }
     }
 
     tcgen05_fence_before();
-    __syncthreads();
+    __syncwarp();
+    if (CTAS == 2) cluster_sync_all();   // the peer's shared memory and tensor memory stay alive until the pair is done
+    else __syncthreads();
     if (warp == 1) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (CTAS == 1)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -923,6 +1046,40 @@ static int sm_count()
     return n;
 }
 
+template <int KIND, int CTAS>
+static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmParams &p, void *stream)
+{
+    CUtensorMap tmA, tmB;
+    if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<CTAS>::kBRows)) return FP4Q_ERR_CUDA;
+    p.ctas = CTAS;
+    p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
+    p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg<CTAS>::kSmemBytes) != cudaSuccess)
+            return FP4Q_ERR_CUDA;
+        attr_set = true;
+    }
+    const int slots = sm_count() / CTAS;
+    const int grid = CTAS * (p.n_tile_total < slots ? p.n_tile_total : slots);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Cfg<CTAS>::kSmemBytes;
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CTAS == 2 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS>, tmA, tmB, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
+
 template <int KIND>
 static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p, void *ws, size_t ws_bytes, void *stream)
 {
@@ -932,24 +1089,15 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     const size_t esize = p.out_f32 ? 4 : 2;
     if (!aligned(p.C, 16) || (p.ldc * esize) % 16) return FP4Q_ERR_ALIGN;
     if (p.n_tile_total <= 0) return FP4Q_OK;
-
-    CUtensorMap tmA, tmB;
-    if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
-    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, BN)) return FP4Q_ERR_CUDA;
     p.sfa = A.sf;
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
-
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[KIND]) {
-        if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
-            cudaSuccess)
-            return FP4Q_ERR_CUDA;
-        attr_set[KIND] = true;
-    }
-    const int grid = p.n_tile_total < sm_count() ? p.n_tile_total : sm_count();
-    gemm_block_scaled_kernel<KIND><<<grid, kThreads, kSmemBytes, static_cast<cudaStream_t>(stream)>>>(tmA, tmB, p);
-    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    // Dense FP4 products with more than one row tile run as cta_group::2 pairs (256x256 tiles); grouped products
+    // (token groups are only 128-row aligned) and the MXFP8 path keep one CTA per 128x256 tile.
+#ifndef FP4Q_FORCE_SINGLE
+    if (KIND == KIND_MXF4 && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND_MXF4, 2>(A, B, p, stream);
+#endif
+    return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
 
 static bool tensor_ok(const fp4q_tensor *t) { return t && t->rows >= 0 && t->cols >= 0; }
