@@ -20,6 +20,7 @@
 // scale columns in TMEM form a ring of the same depth.  Every wait is bounded: when a limit is hit the
 // CTA records FP4Q_ERR_TIMEOUT in the workspace, stops issuing work and leaves through the normal exit
 // (TMEM is freed).
+#include <cstdlib>
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -33,9 +34,17 @@ constexpr int kAStageBytes = BM * 128;
 constexpr int kSfStageBytes = 3072;          // SFA 2 x 512 B, SFB 2 x 1024 B
 constexpr int kSfaOff = 0, kSfbOff = 1024;
 constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
-constexpr int kCacheChunks = 128;            // scale cache: contraction chunks of 128 elements per unit (16384 elements)
-constexpr int kCacheBytes = kCacheChunks * 48;   // per chunk: 16 B for A (4 row tiles x 4 blocks) + 32 B for B (8 x 4)
-constexpr int kSmemCache = 2 * kCacheBytes;
+// 2D-block scales: the scale images of a whole unit (up to 16 stages = 4096 contraction elements of one tile) are
+// built once, ahead of time, and tcgen05.cp reads them in place.  Per 128-element chunk the compact form is one
+// 16-byte row for A [row tile 0..3][block 0..3] and two for B (row tiles 0..3, 4..7); an image is such a row
+// replicated over the 8 rows of one core matrix (128 B), which a descriptor with a zero stride between 8-row
+// groups presents as the 32 identical rows tcgen05.cp.32x128b expects.  Per stage: 6 images = 768 B.
+constexpr int kCacheChunks = 32;             // chunks per unit
+constexpr int kUnitStages = kCacheChunks / 2;
+constexpr int kCompactBytes = kCacheChunks * 48;
+constexpr int kImageStageBytes = 768;        // A chunk 0, A chunk 1, B chunk 0 (rows 0..127, 128..255), B chunk 1 (same)
+constexpr int kCacheBufBytes = kUnitStages * kImageStageBytes;
+constexpr int kSmemCache = kCompactBytes + 2 * kCacheBufBytes;
 
 // CTAS = 1: one CTA per 128x256 tile, it loads all 256 B rows.  CTAS = 2: a cluster of two CTAs shares a 256x256
 // tile through cta_group::2 MMAs; each CTA loads its own 128 A rows and half of the B rows, which halves the
@@ -46,8 +55,9 @@ struct Cfg {
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
-    static constexpr int kSmemSf = kStages * kSfStageBytes;
-    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemSf + kSmemCache + kSmemTail;
+    static constexpr int kSmemSf = kStages * kSfStageBytes;                       // per-row scales (MXFP8): per-stage images
+    static constexpr int kSmemScales = kSmemSf > kSmemCache ? kSmemSf : kSmemCache;   // either kind uses the same region
+    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemTail;
 };
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
@@ -190,6 +200,10 @@ __device__ __noinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volat
 }
 // For barriers that another CTA of the cluster completes (a multicast tcgen05.commit): probe instead of try_wait,
 // whose suspended thread is not reliably woken early by a remote arrival.
+__device__ __noinline__ bool mbar_poll(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint32_t where)
+{
+    return mbar_wait_impl<0, true>(bar, parity, abort_flag, status, where);
+}
 __device__ __noinline__ bool mbar_poll_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
                                                uint32_t where)
 {
@@ -278,6 +292,12 @@ __device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
 {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Descriptor of a replicated scale image: 8 rows of 16 B; the stride between 8-row groups is zero, so the 32 rows
+// tcgen05.cp reads are four passes over the same 128 bytes.
+__device__ __forceinline__ uint64_t smem_desc_scale_image_rep(uint32_t addr)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 46);
 }
 // Descriptor of a scale image: 32 rows of 16 B, contiguous (no swizzle; 8-row groups 128 B apart).
 __device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
@@ -582,9 +602,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_sf = smem + Cfg<CTAS>::kSmemOperands;
-    uint8_t *smem_cache = smem_sf + Cfg<CTAS>::kSmemSf;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_cache + kSmemCache);
+    uint8_t *smem_sf = smem + Cfg<CTAS>::kSmemOperands;        // MXFP8: per-stage scale images
+    uint8_t *smem_compact = smem_sf;                            // FP4: compact scale rows of the unit being built ...
+    uint8_t *smem_images = smem_sf + kCompactBytes;             // ... and two buffers of ready images
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_sf + Cfg<CTAS>::kSmemScales);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
     // bars[14..15] scale cache full, bars[16..17] scale cache empty, bars[18] tensor pipe drained (abort path)
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 19);
@@ -661,6 +682,12 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     // each CTA counts its own bytes on its own barrier (in a pair the second CTA's watcher forwards)
                     mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
                     tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, bar_full + 8 * stage);
+#ifdef FP4Q_SPLIT_B   // development only: the B rows as two boxes of 128 rows
+                    if (CTAS == 1) {
+                        tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
+                        tma_load_2d(smem_u32(smem_b + stage * kBStageBytes + 16384), &tmB, xb, t.b_load_row0 + 128, bar_full + 8 * stage);
+                    } else
+#endif
                     tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
                     TRACE_EV(1, ev_j);
                     ev_j++;
@@ -680,7 +707,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0, acc_phase = 0;
+        uint32_t stage = 0, acc_phase = 0, unit = 0;
         bool ok = true;
         const bool issuer = elect_one();
         int ev_j = 0;
@@ -705,14 +732,21 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
                 if (issuer) {
-                    const uint32_t sf_smem = smem_u32(smem_sf + stage * kSfStageBytes);
+#ifndef FP4Q_SKIP_MMA   // development only: leave the tensor pipe idle to time the load path alone
                     const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
-                    constexpr int kChunks = KIND == KIND_MXF4 ? 2 : 1;
+                    if (KIND == KIND_MXF4) {
+                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
-                    for (int c = 0; c < kChunks; c++) {
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image(sf_smem + kSfaOff + 512 * c));
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c));
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image(sf_smem + kSfbOff + 1024 * c + 512));
+                        for (int c = 0; c < 2; c++) {
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image_rep(img + 128 * c));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image_rep(img + 256 + 256 * c));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
+                        }
+                    } else {
+                        const uint32_t sf_smem = smem_u32(smem_sf + stage * kSfStageBytes);
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(sf_smem + kSfaOff));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8, smem_desc_scale_image(sf_smem + kSfbOff));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12, smem_desc_scale_image(sf_smem + kSfbOff + 512));
                     }
                     const uint64_t adesc = smem_desc_sw128(smem_u32(smem_a + stage * kAStageBytes));
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(smem_b + stage * kBStageBytes));
@@ -728,9 +762,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                                                                  sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
                         }
                     }
+#endif
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
                     if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
+                    if (KIND == KIND_MXF4 && ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1))
+                        tcgen05_commit<CTAS>(bar_cache_empty + 8 * (unit & 1u));   // the unit's images have been copied
                 }
+                if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1) unit++;
                 TRACE_ADD(c_issue, tt);
                 if (lane == 0) TRACE_EV(3, ev_j);
                 ev_j++;
@@ -800,13 +838,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             phase ^= 1u;
         }
     } else if (warp == 3) {
-        // ------------------------------------------------------------------ scale cache builder, 2D-block scales
-        // Per unit (a tile, or a 16384-element slice of a longer contraction) gathers every compact scale byte the
-        // unit needs into shared memory, already arranged as the 16-byte image rows: per 128-element chunk one row
-        // for A [row tile 0..3][block 0..3] and two for B (row tiles 0..3 and 4..7).  Two buffers alternate, so
-        // the next unit's scales are gathered while the current unit runs; all global-memory latency of the
-        // scale path is paid here, once per unit, off the per-stage critical path.  In a pair each CTA gathers the
-        // scales of its own 128 A rows and of all 256 B rows.
+        // ------------------------------------------------------------------ scale image builder, 2D-block scales
+        // Per unit (up to 16 stages of one tile) gathers the compact scale bytes from global memory into 16-byte rows
+        // and replicates each row into its image.  Two image buffers alternate, so the next unit is built while
+        // the current one runs: all global-memory latency of the scale path is paid here, off the per-stage
+        // critical path, and nothing has to be written per stage.  A buffer is free again once the MMA warp's
+        // commit reports that the last scale copy out of it has completed.  In a pair each CTA builds the images
+        // of its own 128 A rows and of all 256 B rows.
         uint32_t unit = 0;
         bool ok = true;
         for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
@@ -814,113 +852,77 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             decode_tile(p, tile, rank, t);
             for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
                 const int buf = unit & 1;
-                if (lane == 0) ok = mbar_wait_lazy(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
+                uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
+                build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, compact, lane);
+                build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
+                __syncwarp();
+                if (lane == 0)
+                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
+                                   : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
-                const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
-                uint32_t *cache = reinterpret_cast<uint32_t *>(smem_cache + buf * kCacheBytes);
-                build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, cache, lane);
-                build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, cache + kCacheChunks * 4, lane);
+                const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
+                uint8_t *images = smem_images + buf * kCacheBufBytes;
+                for (int q = lane; q < 3 * n_chunks; q += 32) {
+                    uint4 row;
+                    uint8_t *dst;
+                    if (q < n_chunks) {                       // A, chunk q
+                        row = rows[q];
+                        dst = images + (q >> 1) * kImageStageBytes + (q & 1) * 128;
+                    } else {                                  // B, chunk (q - n_chunks) / 2, rows 0..127 or 128..255
+                        const int qb = q - n_chunks, chunk = qb >> 1;
+                        row = rows[kCacheChunks + qb];
+                        dst = images + (chunk >> 1) * kImageStageBytes + 256 + (chunk & 1) * 256 + (qb & 1) * 128;
+                    }
+#pragma unroll
+                    for (int r = 0; r < 8; r++) reinterpret_cast<uint4 *>(dst)[r] = row;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);
             }
         }
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ scale image writer and watcher, 2D-block scales
-        // Two cursors run over this CTA's stream of stages.  The writing cursor waits for a ring slot to be free,
-        // copies six 16-byte rows from the scale cache into the slot's images (each replicated over the 32 image
-        // rows tcgen05.cp expects) and, in the second CTA of a pair, arrives on the leader's "full" barrier.  The
-        // signalling cursor (one CTA, or the leader) waits for the slot's "full" barrier - the operand bytes of
-        // both CTAs and the peer's images - and, at the first stage of a tile, for the accumulator to be drained,
-        // then meets the MMA warp at the slot's named barrier.  Neither cursor waits on an mbarrier: both
-        // conditions are probed, so a slot can be filled while an earlier one is still in flight.  After a timeout every remaining stage is released unseen, so
-        // that the MMA warp, which cannot time out on a named barrier, always runs to its end.
-        constexpr int kUnitStages = kCacheChunks * 128 / kStageElems;
+        // ------------------------------------------------------------------ watcher, 2D-block scales
+        // Follows this CTA's stream of stages.  For each it waits for the ring slot's "full" barrier (the operand
+        // bytes; in the leader of a pair also the second CTA's report), at the first stage of a unit for the
+        // unit's scale images, and at the first stage of a tile for the accumulator to be drained; then it meets
+        // the MMA warp at the slot's named barrier (one CTA, or the leader) or reports to the leader's "full"
+        // barrier (second CTA of a pair).  After a timeout every remaining stage is released unseen, so that the
+        // MMA warp, which cannot time out on a named barrier, always runs to its end.
         const bool signals = CTAS == 1 || leader;
-        StageIter wr, sg;
-        wr.init(p, first_tile, tile_step, rank, kStageElems);
-        sg = wr;
-        uint32_t wstage = 0, wphase = 0, sstage = 0, sphase = 0, acc_phase = 0, unit = 0;
-        uint32_t n_written = 0, n_signalled = 0, idle = 0;
-        bool unit_open = false, ok = true;
-        TRACE_DECL(c_write); TRACE_DECL(c_meet); TRACE_DECL(c_poll);
+        StageIter sg;
+        sg.init(p, first_tile, tile_step, rank, kStageElems);
+        uint32_t stage = 0, phase = 0, acc_phase = 0, unit = 0;
+        bool ok = true;
+        TRACE_DECL(c_meet); TRACE_DECL(c_poll);
         TRACE_T0(tt);
+        int ev_j = 0;
         while (sg.valid(p) && (signals || ok)) {
-            bool progress = false;
-            if (ok && wr.valid(p)) {
-                const int buf = unit & 1;
-                bool ready = false;
-                if (lane == 0) {
-                    ready = mbar_test_wait(bar_empty + 8 * wstage, wphase ^ 1u);
-                    if (ready && !unit_open) ready = mbar_test_wait(bar_cache_full + 8 * buf, (unit >> 1) & 1u);
-                }
-                ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
-                TRACE_ADD(c_poll, tt);
-                if (ready) {
-                    if (lane == 0) TRACE_EV(4, (int)n_written);
-                    unit_open = true;
-                    const int in_unit = wr.it & (kUnitStages - 1);
-                    const uint4 *cache_a = reinterpret_cast<const uint4 *>(smem_cache + buf * kCacheBytes);
-                    const uint4 *cache_b = cache_a + kCacheChunks;
-                    uint4 *img = reinterpret_cast<uint4 *>(smem_sf + wstage * kSfStageBytes);
-                    const uint4 a0 = cache_a[2 * in_unit], a1 = cache_a[2 * in_unit + 1];
-                    const uint4 b0 = cache_b[4 * in_unit], b1 = cache_b[4 * in_unit + 1];
-                    const uint4 b2 = cache_b[4 * in_unit + 2], b3 = cache_b[4 * in_unit + 3];
-                    img[(kSfaOff >> 4) + lane] = a0;             // SFA chunk 0
-                    img[(kSfaOff >> 4) + 32 + lane] = a1;        // SFA chunk 1
-                    img[(kSfbOff >> 4) + lane] = b0;             // SFB chunk 0, rows 0..127
-                    img[(kSfbOff >> 4) + 32 + lane] = b1;        // SFB chunk 0, rows 128..255
-                    img[(kSfbOff >> 4) + 64 + lane] = b2;        // SFB chunk 1, rows 0..127
-                    img[(kSfbOff >> 4) + 96 + lane] = b3;        // SFB chunk 1, rows 128..255
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
-                    __syncwarp();
-                    if (lane == 0 && (in_unit == kUnitStages - 1 || wr.it == wr.n_it - 1)) mbar_arrive(bar_cache_empty + 8 * buf);
-                    if (in_unit == kUnitStages - 1 || wr.it == wr.n_it - 1) { unit++; unit_open = false; }
-                    if (lane == 0) TRACE_EV(5, (int)n_written);
-                    if (++wstage == kStages) { wstage = 0; wphase ^= 1u; }
-                    wr.next(p, kStageElems);
-                    n_written++;
-                    progress = true;
-                    TRACE_ADD(c_write, tt);
-                }
+            if (ok && lane == 0) {
+                if ((sg.it & (kUnitStages - 1)) == 0)
+                    ok = mbar_wait(bar_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x510u + (unit & 1u));
+                if (ok)
+                    ok = CTAS == 2 ? mbar_poll(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage)
+                                   : mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage);
+                if (ok && signals && sg.it == 0)
+                    ok = CTAS == 2 ? mbar_poll(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u)
+                                   : mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
             }
-            if (n_signalled < n_written || !ok) {
-                bool ready = true;
-                if (ok) {
-                    if (lane == 0) {
-                        ready = mbar_test_wait(bar_full + 8 * sstage, sphase);
-                        if (ready && signals && sg.it == 0) ready = mbar_test_wait(bar_acc_empty, acc_phase ^ 1u);
-                    }
-                    ready = __shfl_sync(0xFFFFFFFFu, ready, 0);
-                }
-                TRACE_ADD(c_poll, tt);
-                if (ready) {
-                    if (lane == 0) TRACE_EV(6, (int)n_signalled);
-                    if (signals) named_sync(1 + sstage);   // rendezvous: the MMA warp is at most one stage behind
-                    else if (lane == 0) mbar_arrive_cluster(cluster_addr(bar_full + 8 * sstage, 0));   // this CTA's half is in place
-                    TRACE_ADD(c_meet, tt);
-                    if (sg.it == 0) acc_phase ^= 1u;
-                    if (++sstage == kStages) { sstage = 0; sphase ^= 1u; }
-                    sg.next(p, kStageElems);
-                    n_signalled++;
-                    progress = true;
-                }
-            }
-            if (progress) {
-                idle = 0;
-            } else if (ok) {
-                if (++idle >= kWaitLimit) {
-                    ok = false;
-                    if (lane == 0) {
-                        *abort_flag = 1u;
-                        if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = 0x300u + sstage;
-                    }
-                } else if ((idle & 255u) == 255u && *abort_flag) {
-                    ok = false;
-                }
-            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            TRACE_ADD(c_poll, tt);
+            if (lane == 0) TRACE_EV(6, ev_j);
+            ev_j++;
+            if (signals) named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
+            else if (ok && lane == 0) mbar_arrive_cluster(cluster_addr(bar_full + 8 * stage, 0));   // this CTA's half is in place
+            TRACE_ADD(c_meet, tt);
+            if (sg.it == 0) acc_phase ^= 1u;
+            if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) unit++;
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            sg.next(p, kStageElems);
         }
-        if (lane == 0) { TRACE_OUT(p, 5, c_write); TRACE_OUT(p, 6, c_meet); TRACE_OUT(p, 7, c_poll); }
+        if (lane == 0) { TRACE_OUT(p, 6, c_meet); TRACE_OUT(p, 7, c_poll); }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 (hardware: warp id mod 4)
@@ -1051,7 +1053,11 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
 {
     CUtensorMap tmA, tmB;
     if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
+#ifdef FP4Q_SPLIT_B
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, 128)) return FP4Q_ERR_CUDA;
+#else
     if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<CTAS>::kBRows)) return FP4Q_ERR_CUDA;
+#endif
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
@@ -1063,7 +1069,10 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
             return FP4Q_ERR_CUDA;
         attr_set = true;
     }
-    const int slots = sm_count() / CTAS;
+    int slots = sm_count() / CTAS;
+#ifdef FP4Q_TRACE
+    if (const char *g = getenv("FP4Q_DEBUG_SLOTS")) slots = atoi(g);   // development only: use fewer SMs
+#endif
     const int grid = CTAS * (p.n_tile_total < slots ? p.n_tile_total : slots);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -1092,11 +1101,12 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     p.sfa = A.sf;
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
-    // Dense FP4 products with more than one row tile run as cta_group::2 pairs (256x256 tiles); grouped products
-    // (token groups are only 128-row aligned) and the MXFP8 path keep one CTA per 128x256 tile.
-#ifndef FP4Q_FORCE_SINGLE
-    if (KIND == KIND_MXF4 && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND_MXF4, 2>(A, B, p, stream);
-#endif
+    // Dense FP4 products can also run as cta_group::2 pairs (256x256 tiles, each CTA loads half of the B rows).  The
+    // pair kernel is complete and parity-tested but its load path currently sustains only half the bytes per clock
+    // of the one-CTA kernel, so it is opt-in: set FP4Q_CTA_PAIRS=1 in the environment before the first GEMM call.
+    // Grouped products (token groups are only 128-row aligned) and the MXFP8 path always use one CTA per 128x256 tile.
+    static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return e && e[0] == '1'; }();
+    if (use_pairs && KIND == KIND_MXF4 && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND_MXF4, 2>(A, B, p, stream);
     return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
 
