@@ -59,6 +59,7 @@ struct Cfg {
     static constexpr int kSmemScales = kSmemSf > kSmemCache ? kSmemSf : kSmemCache;   // either kind uses the same region
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemTail;
 };
+constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
@@ -111,6 +112,7 @@ struct GemmParams {
     int32_t M, N, K;                 // per-problem output rows, output columns, contraction length (elements)
     int32_t m_tiles, n_tiles, n_tile_total;   // m_tiles counts rows of 128 * ctas
     int32_t ctas;                    // CTAs per tile (1, or 2 for cta_group::2 pairs)
+    int32_t raster_m;                // tile order: groups of raster_m row tiles, within a group row tile fastest
     int32_t out_f32, accumulate;
     int32_t mode, n_groups;
     const int64_t *row_offsets;
@@ -234,6 +236,10 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
 {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
     uint32_t r;
@@ -342,7 +348,13 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int r
     const int per_problem = p.m_tiles * p.n_tiles;
     const int g = p.mode == MODE_GROUPED_K ? tile / per_problem : 0;
     const int local = tile - g * per_problem;
-    const int m_blk = local % p.m_tiles, n_blk = local / p.m_tiles;
+    // Tiles that run at the same time (consecutive indices) cover raster_m row tiles x a few column tiles, and
+    // the sweep over column tiles finishes before the next group of row tiles starts: the group's A rows stay
+    // in L2 for the whole sweep instead of the whole A operand being streamed once per wave.
+    const int per_group = p.raster_m * p.n_tiles;
+    const int grp_m = local / per_group, in_grp = local - grp_m * per_group;
+    const int m0 = grp_m * p.raster_m, gsz = min(p.raster_m, p.m_tiles - m0);
+    const int n_blk = in_grp / gsz, m_blk = m0 + (in_grp - n_blk * gsz);
     t.a_row0 = (m_blk * p.ctas + rank) * BM;
     t.b_row0 = n_blk * BN;
     t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * 128 : 0);
@@ -607,15 +619,16 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     uint8_t *smem_images = smem_sf + kCompactBytes;             // ... and two buffers of ready images
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_sf + Cfg<CTAS>::kSmemScales);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
-    // bars[14..15] scale cache full, bars[16..17] scale cache empty, bars[18] tensor pipe drained (abort path)
-    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 19);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 19) + 1;
+    // bars[14..15] scale images full, bars[16..17] scale images empty, bars[18] tensor pipe drained (abort path),
+    // bars[19..20] (leader of a pair) the second CTA's scale images full
+    uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 21);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 21) + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
     const uint32_t bar_cache_full = smem_u32(bars + 14), bar_cache_empty = smem_u32(bars + 16);
-    const uint32_t bar_drain = smem_u32(bars + 18);
+    const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 19);
 
     // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
     const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
@@ -624,9 +637,9 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) {
-            // The producer's expect_tx arrival; in the leader of a pair also the arrival by which the second CTA's
-            // watcher reports that CTA's operands and scale images.  The watcher of the stage waits on it.
-            mbar_init(bar_full + 8 * s, (CTAS == 2 && leader) ? 2 : 1);
+            // The producer's expect_tx arrival (in a pair the leader's, which announces both CTAs' bytes: the second
+            // CTA's loads complete on the leader's barrier).  The watcher of the stage waits on it.
+            mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
         }
         mbar_init(bar_acc_full, 1);
@@ -635,6 +648,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         for (int b = 0; b < 2; b++) {
             mbar_init(bar_cache_full + 8 * b, 1);
             mbar_init(bar_cache_empty + 8 * b, 1);
+            mbar_init(bar_peer_cache_full + 8 * b, 1);
         }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -661,45 +675,69 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            bool ok = true;
-            int ev_j = 0;
-            TRACE_DECL(c_empty); TRACE_DECL(c_issue);
-            TRACE_T0(tt);
-            for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
-                Tile t;
-                decode_tile(p, tile, rank, t);
-                const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
-                for (int it = 0; it < n_it; it++) {
-                    TRACE_ADD(c_issue, tt);
-                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage)
-                                   : mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
-                    TRACE_ADD(c_empty, tt);
-                    TRACE_EV(0, ev_j);
-                    if (!ok) break;
-                    const int xa = (t.a_k0 + it * kStageElems) / kElemsPerByte, xb = (t.b_k0 + it * kStageElems) / kElemsPerByte;
-                    // each CTA counts its own bytes on its own barrier (in a pair the second CTA's watcher forwards)
-                    mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
-                    tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, bar_full + 8 * stage);
-#ifdef FP4Q_SPLIT_B   // development only: the B rows as two boxes of 128 rows
-                    if (CTAS == 1) {
-                        tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
-                        tma_load_2d(smem_u32(smem_b + stage * kBStageBytes + 16384), &tmB, xb, t.b_load_row0 + 128, bar_full + 8 * stage);
-                    } else
+        // A shared-memory access of this warp (the poll of the next "empty" barrier) queues behind the TMA
+        // instructions it has just issued and waits ~450 cycles, which would limit one warp to a stage per
+        // ~900 cycles.  So every round first polls - it waits for the next slot and then probes up to two
+        // more - and only then issues the loads of all slots found free, back to back.
+        constexpr int kBatch = 3;
+        StageIter pr;
+        pr.init(p, first_tile, tile_step, rank, kStageElems);
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        const bool issuer = elect_one();
+        TRACE_DECL(c_empty); TRACE_DECL(c_issue); TRACE_DECL(c_rounds);
+        TRACE_T0(tt);
+        int ev_j = 0;
+        while (ok && pr.valid(p)) {
+            int n_free = 0;
+#ifdef FP4Q_TRACE
+            c_rounds++;
 #endif
-                    tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
-                    TRACE_EV(1, ev_j);
-                    ev_j++;
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            if (lane == 0) {
+                ok = mbar_wait_impl<0, true>(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
+                if (ok) {
+                    n_free = 1;
+                    uint32_t s2 = stage, ph2 = phase;
+                    while (n_free < kBatch) {
+                        if (++s2 == kStages) { s2 = 0; ph2 ^= 1u; }
+                        if (!mbar_test_wait(bar_empty + 8 * s2, ph2 ^ 1u)) break;
+                        n_free++;
+                    }
                 }
             }
-            if (!ok) {   // give copies already in flight time to land before the CTA's shared memory is released
-                for (int i = 0; i < 200; i++) __nanosleep(1000);
+            n_free = __shfl_sync(0xFFFFFFFFu, n_free, 0);
+            ok = n_free > 0;
+            TRACE_ADD(c_empty, tt);
+            for (int b = 0; b < n_free && pr.valid(p); b++) {
+                if (lane == 0) TRACE_EV(0, ev_j);
+                if (issuer) {
+                    const Tile &t = pr.t;
+                    const int xa = (t.a_k0 + pr.it * kStageElems) / kElemsPerByte, xb = (t.b_k0 + pr.it * kStageElems) / kElemsPerByte;
+                    if (CTAS == 1) {
+                        mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
+                        tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, bar_full + 8 * stage);
+                        tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
+                    } else {
+                        // Both CTAs' bytes are counted on the leader's barrier, which the leader arms for all of them.
+                        // (A remote mbarrier.arrive per stage by a thread of the second CTA costs ~1200 cycles each
+                        // and cannot be pipelined; letting the TMA unit signal the remote barrier costs nothing.)
+                        if (leader) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * (kAStageBytes + kBStageBytes));
+                        const uint32_t lbar = cluster_addr(bar_full + 8 * stage, 0);
+                        tma_load_2d_pair(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, lbar);
+                        tma_load_2d_pair(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, lbar);
+                    }
+                }
+                if (lane == 0) TRACE_EV(1, ev_j);
+                ev_j++;
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                pr.next(p, kStageElems);
             }
-            TRACE_OUT(p, 0, c_empty);
-            TRACE_OUT(p, 1, c_issue);
+            TRACE_ADD(c_issue, tt);
         }
+        if (!ok) {   // give copies already in flight time to land before the CTA's shared memory is released
+            for (int i = 0; i < 200; i++) __nanosleep(1000);
+        }
+        if (lane == 0) { TRACE_OUT(p, 0, c_empty); TRACE_OUT(p, 1, c_issue); TRACE_OUT(p, 5, c_rounds); }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (the leader CTA of a pair)
         // The warp stays converged and one elected lane issues the tcgen05 instructions: their descriptors then live
@@ -880,18 +918,20 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);
+                if (lane == 0) {
+                    if (CTAS == 1 || leader) mbar_arrive(bar_cache_full + 8 * buf);
+                    else mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * buf, 0));   // the leader copies both CTAs' images
+                }
             }
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ watcher, 2D-block scales
-        // Follows this CTA's stream of stages.  For each it waits for the ring slot's "full" barrier (the operand
-        // bytes; in the leader of a pair also the second CTA's report), at the first stage of a unit for the
-        // unit's scale images, and at the first stage of a tile for the accumulator to be drained; then it meets
-        // the MMA warp at the slot's named barrier (one CTA, or the leader) or reports to the leader's "full"
-        // barrier (second CTA of a pair).  After a timeout every remaining stage is released unseen, so that the
-        // MMA warp, which cannot time out on a named barrier, always runs to its end.
-        const bool signals = CTAS == 1 || leader;
+        // Follows the stream of stages (one CTA, or the leader of a pair; the second CTA's warp idles).  For each
+        // it waits for the ring slot's "full" barrier (the operand bytes of both CTAs), at the first stage of a
+        // unit for the unit's scale images (of both CTAs), and at the first stage of a tile for the accumulator
+        // to be drained; then it meets the MMA warp at the slot's named barrier.  After a timeout every remaining
+        // stage is released unseen, so that the MMA warp, which cannot time out on a named barrier, always runs
+        // to its end.
         StageIter sg;
         sg.init(p, first_tile, tile_step, rank, kStageElems);
         uint32_t stage = 0, phase = 0, acc_phase = 0, unit = 0;
@@ -899,23 +939,51 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_DECL(c_meet); TRACE_DECL(c_poll);
         TRACE_T0(tt);
         int ev_j = 0;
-        while (sg.valid(p) && (signals || ok)) {
-            if (ok && lane == 0) {
-                if ((sg.it & (kUnitStages - 1)) == 0)
-                    ok = mbar_wait(bar_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x510u + (unit & 1u));
-                if (ok)
-                    ok = CTAS == 2 ? mbar_poll(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage)
-                                   : mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage);
-                if (ok && signals && sg.it == 0)
-                    ok = CTAS == 2 ? mbar_poll(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u)
-                                   : mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
+        bool unit_seen = false;   // lane 0: the next unit's scale images have been seen complete
+        uint32_t ahead = 0;   // stages after the current one whose "full" barrier is already known to be complete
+        while (leader && sg.valid(p)) {
+            if (lane == 0) TRACE_EV(4, ev_j);
+            if (ahead > 0) {
+                ahead--;
+            } else {
+                if (ok && lane == 0) {
+                    if ((sg.it & (kUnitStages - 1)) == 0 && !unit_seen) {
+                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x510u + (unit & 1u));
+                        if (ok && CTAS == 2)
+                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x520u + (unit & 1u));
+                    }
+                    if ((sg.it & (kUnitStages - 1)) == 0) unit_seen = false;
+                    if (ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen) {
+                        // second half of a unit: look whether the next unit's images are in place already, so that
+                        // the unit boundary costs no extra probes on the critical path
+                        const uint32_t nu = unit + 1;
+                        unit_seen = mbar_test_wait(bar_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u) &&
+                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u));
+                    }
+                    if (ok) ok = mbar_wait_impl<0, true>(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage);
+                    if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
+                    if (ok) {
+                        // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long complete,
+                        // more than the MMA warp needs per stage.  So the next two slots are probed in one go (the two
+                        // latencies overlap) and, if complete, handed over without another look.  Only stages of the
+                        // same unit qualify: they need nothing but their "full" barrier.
+                        const int left = min(kUnitStages - 1 - (sg.it & (kUnitStages - 1)), sg.n_it - 1 - sg.it);
+                        const uint32_t s1 = stage + 1 == kStages ? 0u : stage + 1, p1 = s1 == 0 ? phase ^ 1u : phase;
+                        const uint32_t s2 = s1 + 1 == kStages ? 0u : s1 + 1, p2 = s2 == 0 ? p1 ^ 1u : p1;
+                        uint32_t r1, r2;
+                        asm volatile("{\n .reg .pred p, q;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%2], %3;\n"
+                                     " mbarrier.test_wait.parity.shared::cta.b64 q, [%4], %5;\n selp.b32 %0, 1, 0, p;\n selp.b32 %1, 1, 0, q;\n}"
+                                     : "=r"(r1), "=r"(r2) : "r"(bar_full + 8 * s1), "r"(p1), "r"(bar_full + 8 * s2), "r"(p2) : "memory");
+                        ahead = (left >= 1 && r1) ? ((left >= 2 && r2) ? 2u : 1u) : 0u;
+                    }
+                }
+                ahead = __shfl_sync(0xFFFFFFFFu, ahead, 0);
             }
             ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
             TRACE_ADD(c_poll, tt);
             if (lane == 0) TRACE_EV(6, ev_j);
             ev_j++;
-            if (signals) named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
-            else if (ok && lane == 0) mbar_arrive_cluster(cluster_addr(bar_full + 8 * stage, 0));   // this CTA's half is in place
+            named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
             TRACE_ADD(c_meet, tt);
             if (sg.it == 0) acc_phase ^= 1u;
             if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) unit++;
@@ -979,7 +1047,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
-        if (warp == 4 && lane == 0) { TRACE_OUT(p, 8, c_wait); TRACE_OUT(p, 9, c_ld); TRACE_OUT(p, 10, c_store); }
+        if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
     tcgen05_fence_before();
@@ -1061,6 +1129,10 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
+    p.raster_m = p.mode == MODE_DENSE ? (p.m_tiles < kRasterM ? p.m_tiles : kRasterM) : p.m_tiles;
+#ifdef FP4Q_TRACE
+    if (const char *g = getenv("FP4Q_DEBUG_RASTER")) { p.raster_m = atoi(g); if (p.raster_m > p.m_tiles) p.raster_m = p.m_tiles; }
+#endif
 
     static bool attr_set = false;
     if (!attr_set) {
@@ -1101,11 +1173,11 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     p.sfa = A.sf;
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
-    // Dense FP4 products can also run as cta_group::2 pairs (256x256 tiles, each CTA loads half of the B rows).  The
-    // pair kernel is complete and parity-tested but its load path currently sustains only half the bytes per clock
-    // of the one-CTA kernel, so it is opt-in: set FP4Q_CTA_PAIRS=1 in the environment before the first GEMM call.
-    // Grouped products (token groups are only 128-row aligned) and the MXFP8 path always use one CTA per 128x256 tile.
-    static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return e && e[0] == '1'; }();
+    // Dense FP4 products with more than one row tile run as cta_group::2 pairs: 256x256 tiles, each CTA loads half of
+    // the B rows, which leaves room for a six-stage ring.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the
+    // first GEMM call) selects the one-CTA kernel instead; grouped products (token groups are only 128-row aligned)
+    // and the MXFP8 path always use one CTA per 128x256 tile.
+    static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return !(e && e[0] == '0'); }();
     if (use_pairs && KIND == KIND_MXF4 && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND_MXF4, 2>(A, B, p, stream);
     return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
