@@ -114,6 +114,7 @@ struct GemmParams {
     int32_t ctas;                    // CTAs per tile (1, or 2 for cta_group::2 pairs)
     int32_t raster_m;                // tile order: groups of raster_m row tiles, within a group row tile fastest
     int32_t out_f32, accumulate;
+    int32_t wide_stores;             // output base and row pitch are 32-byte aligned: 256-bit stores (whole sectors)
     int32_t mode, n_groups;
     const int64_t *row_offsets;
     int32_t b_rows_per_group;        // grouped rows: B row offset per group (forward)
@@ -552,6 +553,13 @@ __device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint
 
 // ---------------------------------------------------------------------------------------- epilogue store
 
+// One whole 32-byte sector per lane (a 16-byte store leaves half a sector to a second transaction).
+__device__ __forceinline__ void st_global_v8(void *dst, const uint32_t *w)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+
 __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row, int col0, int n_cols_valid,
                                                 const uint32_t v[32])
 {
@@ -559,7 +567,10 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
     if (n_cols_valid <= 0) return;
     if (p.out_f32) {
         float *dst = static_cast<float *>(p.C) + row * p.ldc + col0;
-        if (n_cols_valid >= 32) {
+        if (n_cols_valid >= 32 && p.wide_stores && !p.accumulate) {
+#pragma unroll
+            for (int q = 0; q < 4; q++) st_global_v8(dst + 8 * q, v + 8 * q);
+        } else if (n_cols_valid >= 32) {
 #pragma unroll
             for (int q = 0; q < 8; q++) {
                 float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
@@ -577,7 +588,16 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
         }
     } else {
         __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.C) + row * p.ldc + col0;
-        if (n_cols_valid >= 32) {
+        if (n_cols_valid >= 32 && p.wide_stores) {
+            uint32_t w[16];
+#pragma unroll
+            for (int e = 0; e < 16; e++) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+                w[e] = *reinterpret_cast<const uint32_t *>(&b);
+            }
+            st_global_v8(dst, w);
+            st_global_v8(dst + 16, w + 8);
+        } else if (n_cols_valid >= 32) {
 #pragma unroll
             for (int q = 0; q < 4; q++) {
                 uint32_t w[4];
@@ -1170,6 +1190,7 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     const size_t esize = p.out_f32 ? 4 : 2;
     if (!aligned(p.C, 16) || (p.ldc * esize) % 16) return FP4Q_ERR_ALIGN;
     if (p.n_tile_total <= 0) return FP4Q_OK;
+    p.wide_stores = aligned(p.C, 32) && (p.ldc * esize) % 32 == 0;
     p.sfa = A.sf;
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
