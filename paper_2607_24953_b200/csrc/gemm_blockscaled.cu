@@ -980,21 +980,42 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         unit_seen = mbar_test_wait(bar_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u) &&
                                     (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u));
                     }
-                    if (ok) ok = mbar_wait_impl<0, true>(bar_full + 8 * stage, phase, abort_flag, p.status, 0x300u + stage);
                     if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
                     if (ok) {
-                        // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long complete,
-                        // more than the MMA warp needs per stage.  So the next two slots are probed in one go (the two
-                        // latencies overlap) and, if complete, handed over without another look.  Only stages of the
-                        // same unit qualify: they need nothing but their "full" barrier.
+                        // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long
+                        // complete, more than the MMA warp needs per stage.  So the slot's "full" barrier and those of
+                        // the next three slots are probed in one go (the latencies overlap); slots found complete are
+                        // handed over later without another look.  Only stages of the same unit qualify: they need
+                        // nothing but their "full" barrier.
                         const int left = min(kUnitStages - 1 - (sg.it & (kUnitStages - 1)), sg.n_it - 1 - sg.it);
-                        const uint32_t s1 = stage + 1 == kStages ? 0u : stage + 1, p1 = s1 == 0 ? phase ^ 1u : phase;
-                        const uint32_t s2 = s1 + 1 == kStages ? 0u : s1 + 1, p2 = s2 == 0 ? p1 ^ 1u : p1;
-                        uint32_t r1, r2;
-                        asm volatile("{\n .reg .pred p, q;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%2], %3;\n"
-                                     " mbarrier.test_wait.parity.shared::cta.b64 q, [%4], %5;\n selp.b32 %0, 1, 0, p;\n selp.b32 %1, 1, 0, q;\n}"
-                                     : "=r"(r1), "=r"(r2) : "r"(bar_full + 8 * s1), "r"(p1), "r"(bar_full + 8 * s2), "r"(p2) : "memory");
-                        ahead = (left >= 1 && r1) ? ((left >= 2 && r2) ? 2u : 1u) : 0u;
+                        uint32_t sl[4], ph[4];
+                        sl[0] = stage; ph[0] = phase;
+#pragma unroll
+                        for (int q = 1; q < 4; q++) {
+                            sl[q] = sl[q - 1] + 1 == kStages ? 0u : sl[q - 1] + 1;
+                            ph[q] = sl[q] == 0 ? ph[q - 1] ^ 1u : ph[q - 1];
+                        }
+                        uint32_t r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+                        for (uint32_t spin = 0; ; spin++) {
+                            asm volatile("{\n .reg .pred p0, p1, p2, p3;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p0, [%4], %5;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p1, [%6], %7;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p2, [%8], %9;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p3, [%10], %11;\n"
+                                         " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n selp.b32 %2, 1, 0, p2;\n selp.b32 %3, 1, 0, p3;\n}"
+                                         : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                                         : "r"(bar_full + 8 * sl[0]), "r"(ph[0]), "r"(bar_full + 8 * sl[1]), "r"(ph[1]),
+                                           "r"(bar_full + 8 * sl[2]), "r"(ph[2]), "r"(bar_full + 8 * sl[3]), "r"(ph[3]) : "memory");
+                            if (r0) break;
+                            if (spin >= kWaitLimit) {
+                                ok = false;
+                                *abort_flag = 1u;
+                                if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = 0x300u + stage;
+                                break;
+                            }
+                            if ((spin & 255u) == 255u && *abort_flag) { ok = false; break; }
+                        }
+                        ahead = !ok ? 0u : (left >= 1 && r1) ? ((left >= 2 && r2) ? ((left >= 3 && r3) ? 3u : 2u) : 1u) : 0u;
                     }
                 }
                 ahead = __shfl_sync(0xFFFFFFFFu, ahead, 0);
