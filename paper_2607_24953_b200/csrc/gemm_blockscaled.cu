@@ -6,20 +6,25 @@
 //                   contraction block kb is scale[r/32][kb] or, for a transposed view, scale[kb][r/32].
 //   kind::mxf8f6f4  E4M3 payload, one UE8M0 scale per row and 32 contraction elements (MXFP8).
 //
-// One persistent CTA per SM, 128x256 output tile, 12 warps:
-//   warp 0      TMA producer: A tile (128 rows x 128 B) and B tile (256 rows x 128 B) per stage, 128B swizzle
-//   warp 1      MMA issuer: tcgen05.cp of the stage's scale images smem -> TMEM, 4 tcgen05.mma per stage,
-//               tcgen05.commit to release the stage
-//   warp 3      scale cache builder (2D-block scales): once per tile gathers all compact scale bytes the tile
-//               needs into shared memory, arranged as 16-byte image rows (double-buffered across tiles)
-//   warp 2      scale image writer: per stage replicates six cached rows into the 32-lane x 16-byte images that
-//               tcgen05.cp expects (for MXFP8 per-row scales warps 2-3 alternate stages and load directly)
+// Persistent kernel, one CTA per SM, 12 warps.  Dense FP4 products run as clusters of two CTAs that share a 256x256
+// tile through cta_group::2 MMAs (each CTA holds 128 rows of the accumulator, loads its own 128 A rows and half of
+// the B rows); grouped products and MXFP8 use one CTA per 128x256 tile.
+//   warp 0      TMA producer: per stage the A tile (128 rows x 128 B) and the B tile (256 or 128 rows x 128 B),
+//               128B swizzle; polls all free slots first, then issues their loads back to back
+//   warp 1      MMA issuer: stays converged, one elected lane issues per stage 6 tcgen05.cp (scale images -> TMEM),
+//               4 tcgen05.mma and the tcgen05.commit that frees the slot; it never reads shared memory in the loop
+//   warp 2      watcher (2D-block scales): polls the slots' "full" barriers (several at a time), the scale images
+//               and the accumulator's "empty" barrier and meets the MMA warp at a named barrier per stage
+//   warp 3      scale image builder (2D-block scales): per unit of 16 stages gathers the compact scale bytes and
+//               writes the replicated images tcgen05.cp reads in place (double-buffered)
+//               (MXFP8 per-row scales: warps 2-3 alternate stages, load the scale words, write per-stage images
+//               and act as watchers of their stages)
 //   warps 4-11  epilogue: tcgen05.ld of the 128x256 FP32 accumulator (each warp 32 lanes x 128 columns),
-//               release of the accumulator as soon as it sits in registers, then convert and store
-// Four smem stages (48 KB of operands + 3 KB of scale image each) form a ring guarded by mbarriers; the
-// scale columns in TMEM form a ring of the same depth.  Every wait is bounded: when a limit is hit the
-// CTA records FP4Q_ERR_TIMEOUT in the workspace, stops issuing work and leaves through the normal exit
-// (TMEM is freed).
+//               release of the accumulator as soon as it sits in registers, then convert and store (256-bit stores)
+// A ring of four (one CTA: 48 KB of operands per stage) or six (pair: 32 KB) shared-memory stages is guarded by
+// mbarriers; the scale columns in TMEM form a ring of the same depth.  Every mbarrier wait is bounded: when a limit
+// is hit the CTA records FP4Q_ERR_TIMEOUT in the workspace, releases the MMA warp from its named barriers, stops
+// issuing work and leaves through the normal exit (TMEM is freed).
 #include <cstdlib>
 #include <cuda.h>
 #include <cuda_bf16.h>

@@ -254,3 +254,19 @@ def test_mxfp8_quantize_edge_values():
     bits[3, :64] = np.arange(64)               # subnormals
     _mxfp8_operand(workloads.bits_to_bf16(bits, "cuda"))
     _mxfp8_operand(workloads.activations_student_t(70, 200, 9, "cuda", nu=3))   # ragged columns
+
+
+def test_one_cta_kernel_for_dense_products():
+    """Dense FP4 products default to cta_group::2 pairs; FP4Q_CTA_PAIRS=0 (read once per process) selects the
+    one-CTA kernel.  The dense parity cases are repeated in a child process with that switch."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("FP4Q_CTA_PAIRS") == "0":
+        pytest.skip("already running with the one-CTA kernel")
+    env = dict(os.environ, FP4Q_CTA_PAIRS="0")
+    here = os.path.dirname(os.path.abspath(__file__))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_gemm.py"), "-m", "gpu", "-q", "-x",
+                        "-k", "tiny_linear or ragged or exact_case or scale_layout or multi_tile"],
+                       env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
