@@ -50,19 +50,24 @@ constexpr int kCompactBytes = kCacheChunks * 48;
 constexpr int kImageStageBytes = 768;        // A chunk 0, A chunk 1, B chunk 0 (rows 0..127, 128..255), B chunk 1 (same)
 constexpr int kCacheBufBytes = kUnitStages * kImageStageBytes;
 constexpr int kSmemCache = kCompactBytes + 2 * kCacheBufBytes;
+// Epilogue staging of the pair kernel: each of the 8 epilogue warps owns 32 rows x 128 bytes, written from registers
+// (128-byte swizzle: the 16-byte pieces of 8 rows fall into different banks) and drained by a TMA store, which keeps
+// the output off the load/store unit that the MMA warp's instructions also pass through.
+constexpr int kStagingWarpBytes = 32 * 128;
 
 // CTAS = 1: one CTA per 128x256 tile, it loads all 256 B rows.  CTAS = 2: a cluster of two CTAs shares a 256x256
 // tile through cta_group::2 MMAs; each CTA loads its own 128 A rows and half of the B rows, which halves the
 // B-operand shared-memory and L2 traffic per CTA and leaves room for two more ring stages.
 template <int CTAS>
 struct Cfg {
-    static constexpr int kStages = CTAS == 2 ? 6 : 4;
+    static constexpr int kStages = CTAS == 2 ? 5 : 4;
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemSf = kStages * kSfStageBytes;                       // per-row scales (MXFP8): per-stage images
-    static constexpr int kSmemScales = kSmemSf > kSmemCache ? kSmemSf : kSmemCache;   // either kind uses the same region
-    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemTail;
+    static constexpr int kSmemScales = ((kSmemSf > kSmemCache ? kSmemSf : kSmemCache) + 1023) / 1024 * 1024;   // either kind uses the same region
+    static constexpr int kSmemStaging = CTAS == 2 ? 8 * kStagingWarpBytes : 0;
+    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail;
 };
 constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
@@ -256,6 +261,19 @@ __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+
+// TMA stores out of shared memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int32_t x, int32_t y, uint32_t src)
+{
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -558,6 +576,26 @@ __device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint
 
 // ---------------------------------------------------------------------------------------- epilogue store
 
+// One round of the pair kernel's epilogue: 32 words per lane (this lane's row, 128 bytes) into the warp's swizzled
+// staging rows, then one TMA store (kind 0: BF16 bytes, 1: FP32 bytes, 2: FP32 add-reduction) of the 32 x 128 B box.
+__device__ __forceinline__ void stage_and_store(const CUtensorMap *map, const uint32_t *w, uint32_t stg_row, uint32_t swz,
+                                                uint32_t stg, int col, int32_t y, int kind, int lane)
+{
+    if (lane == 0) bulk_wait_read_all();   // the previous round's store has read the staging rows
+    __syncwarp();
+#pragma unroll
+    for (int c = 0; c < 8; c++)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg_row + ((c ^ swz) << 4)), "r"(w[4 * c]), "r"(w[4 * c + 1]),
+                     "r"(w[4 * c + 2]), "r"(w[4 * c + 3]) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> TMA store
+    __syncwarp();
+    if (lane == 0) {
+        if (kind == 2) tma_reduce_add_2d(map, col, y, stg);                 // x in FP32 elements
+        else tma_store_2d(map, col * (kind == 1 ? 4 : 2), y, stg);          // x in bytes
+        bulk_commit();
+    }
+}
+
 // One whole 32-byte sector per lane (a 16-byte store leaves half a sector to a second transaction).
 __device__ __forceinline__ void st_global_v8(void *dst, const uint32_t *w)
 {
@@ -627,7 +665,7 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
 template <int KIND, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                         const __grid_constant__ GemmParams p)
+                         const __grid_constant__ CUtensorMap tmC, const __grid_constant__ GemmParams p)
 {
     constexpr int kStageElems = KIND == KIND_MXF4 ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = KIND == KIND_MXF4 ? 64 : 32;           // contraction elements per MMA (32 B per row)
@@ -642,7 +680,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     uint8_t *smem_sf = smem + Cfg<CTAS>::kSmemOperands;        // MXFP8: per-stage scale images
     uint8_t *smem_compact = smem_sf;                            // FP4: compact scale rows of the unit being built ...
     uint8_t *smem_images = smem_sf + kCompactBytes;             // ... and two buffers of ready images
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_sf + Cfg<CTAS>::kSmemScales);
+    uint8_t *smem_staging = smem_sf + Cfg<CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<CTAS>::kSmemStaging);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
     // bars[14..15] scale images full, bars[16..17] scale images empty, bars[18] tensor pipe drained (abort path),
     // bars[19..20] (leader of a pair) the second CTA's scale images full
@@ -679,6 +718,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+        if (CTAS == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
     }
     if (warp == 1) {
         if (CTAS == 1) {
@@ -1084,7 +1124,42 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
                     for (int q = 0; q < 32; q++) v[j][q] = 0u;
             }
-            if (row_ok) {
+#ifdef FP4Q_SKIP_STORE   // development only: results are dropped
+            if (row_ok && p.M < 0) {
+#else
+            if (CTAS == 2) {
+                // Pair kernel (dense products only): 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
+                // through this warp's staging rows and leave by a TMA store, which clips rows and columns past the
+                // output's edge.  With accumulation the store is the TMA's FP32 add-reduction.
+                if (t.m_valid > 32 * quarter) {
+                    uint8_t *stg = smem_staging + (warp - 4) * kStagingWarpBytes;
+                    const uint32_t stg_row = smem_u32(stg) + lane * 128, swz = (uint32_t)(lane & 7);
+                    const int32_t y = t.c_row0 + 32 * quarter;
+                    if (p.out_f32) {
+#pragma unroll
+                        for (int h = 0; h < 4; h++) {
+                            const int col_in_tile = 128 * half + 32 * h;
+                            if (col_in_tile < t.n_valid)
+                                stage_and_store(&tmC, v[h], stg_row, swz, smem_u32(stg), t.c_col0 + col_in_tile, y, p.accumulate ? 2 : 1, lane);
+                        }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 2; h++) {
+                            const int col_in_tile = 128 * half + 64 * h;
+                            if (col_in_tile >= t.n_valid) continue;
+                            uint32_t w[32];
+#pragma unroll
+                            for (int e = 0; e < 32; e++) {
+                                const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[2 * h + (e >> 4)][(2 * e) & 31]),
+                                                                               __uint_as_float(v[2 * h + (e >> 4)][(2 * e + 1) & 31]));
+                                w[e] = *reinterpret_cast<const uint32_t *>(&b);
+                            }
+                            stage_and_store(&tmC, w, stg_row, swz, smem_u32(stg), t.c_col0 + col_in_tile, y, 0, lane);
+                        }
+                    }
+                }
+            } else if (row_ok) {
+#endif
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const int col_in_tile = 128 * half + 32 * j;
@@ -1093,6 +1168,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
+        if (CTAS == 2 && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
         if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
@@ -1145,6 +1221,22 @@ static bool make_operand_map(CUtensorMap *map, const void *base, int64_t rows, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output map for the pair kernel's TMA stores: box = 128 bytes x 32 rows, 128-byte swizzle.  Plain stores address the
+// output as bytes; accumulation uses the TMA add-reduction, which needs the element type (FP32, 32 per box row).
+static bool make_output_map(CUtensorMap *map, void *base, int64_t rows, int64_t cols, int64_t ld, bool f32, bool reduce)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const int64_t esize = f32 ? 4 : 2;
+    const cuuint64_t dims[2] = {(cuuint64_t)(reduce ? cols : cols * esize), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)(ld * esize)};
+    const cuuint32_t box[2] = {reduce ? 32u : 128u, 32u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, reduce ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Operand {
     const uint8_t *payload;
     int64_t rows, row_bytes, ld_bytes;
@@ -1165,7 +1257,9 @@ static int sm_count()
 template <int KIND, int CTAS>
 static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmParams &p, void *stream)
 {
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmC;
+    const int64_t out_rows = p.mode == MODE_GROUPED_K ? (int64_t)p.n_groups * p.M : p.M;
+    if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
     if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
 #ifdef FP4Q_SPLIT_B
     if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, 128)) return FP4Q_ERR_CUDA;
@@ -1204,7 +1298,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = CTAS == 2 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS>, tmA, tmB, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS>, tmA, tmB, tmC, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }
 
 template <int KIND>
