@@ -13,15 +13,15 @@
 //               128B swizzle; polls all free slots first, then issues their loads back to back
 //   warp 1      MMA issuer: stays converged, one elected lane issues per stage 6 tcgen05.cp (scale images -> TMEM),
 //               4 tcgen05.mma and the tcgen05.commit that frees the slot; it never reads shared memory in the loop
-//   warp 2      watcher (2D-block scales): polls the slots' "full" barriers (several at a time), the scale images
-//               and the accumulator's "empty" barrier and meets the MMA warp at a named barrier per stage
-//   warp 3      scale image builder (2D-block scales): per unit of 16 stages gathers the compact scale bytes and
-//               writes the replicated images tcgen05.cp reads in place (double-buffered)
-//               (MXFP8 per-row scales: warps 2-3 alternate stages, load the scale words, write per-stage images
-//               and act as watchers of their stages)
+//   warp 2      watcher: polls the slots' "full" barriers (several at a time), the scale images and the
+//               accumulator's "empty" barrier and meets the MMA warp at a named barrier per stage
+//   warp 3      scale image builder: per unit of 16 (FP4) or 8 (MXFP8) stages gathers the scale bytes and writes the
+//               images tcgen05.cp reads in place (double-buffered); 2D-block scales as replicated 8-row images,
+//               per-row scales as real 32-row images
 //   warps 4-11  epilogue: tcgen05.ld of the 128x256 FP32 accumulator (each warp 32 lanes x 128 columns),
-//               release of the accumulator as soon as it sits in registers, then convert and store (256-bit stores)
-// A ring of four (one CTA: 48 KB of operands per stage) or six (pair: 32 KB) shared-memory stages is guarded by
+//               release of the accumulator as soon as it sits in registers, then convert and store (pair kernel:
+//               through staging rows and TMA stores; one CTA: 256-bit stores)
+// A ring of four (one CTA: 48 KB of operands per stage) or five (pair: 32 KB) shared-memory stages is guarded by
 // mbarriers; the scale columns in TMEM form a ring of the same depth.  Every mbarrier wait is bounded: when a limit
 // is hit the CTA records FP4Q_ERR_TIMEOUT in the workspace, releases the MMA warp from its named barriers, stops
 // issuing work and leaves through the normal exit (TMEM is freed).
@@ -36,8 +36,6 @@ namespace fp4q {
 constexpr int BM = 128, BN = 256;            // per-CTA accumulator: 128 rows x 256 columns (a CTA pair covers 256 x 256)
 constexpr int kMaxStages = 6;
 constexpr int kAStageBytes = BM * 128;
-constexpr int kSfStageBytes = 3072;          // SFA 2 x 512 B, SFB 2 x 1024 B
-constexpr int kSfaOff = 0, kSfbOff = 1024;
 constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
 // 2D-block scales: the scale images of a whole unit (up to 16 stages = 4096 contraction elements of one tile) are
 // built once, ahead of time, and tcgen05.cp reads them in place.  Per 128-element chunk the compact form is one
@@ -45,10 +43,16 @@ constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag,
 // replicated over the 8 rows of one core matrix (128 B), which a descriptor with a zero stride between 8-row
 // groups presents as the 32 identical rows tcgen05.cp.32x128b expects.  Per stage: 6 images = 768 B.
 constexpr int kCacheChunks = 32;             // chunks per unit
-constexpr int kUnitStages = kCacheChunks / 2;
+constexpr int kUnitStagesMxf4 = kCacheChunks / 2;
+// Per-row scales (MXFP8): a stage covers 4 contraction blocks; its three images (A rows, B rows 0..127, B rows
+// 128..255) are real 32-row x 16-byte images (512 B each), row l holding rows l, l+32, l+64, l+96 of the operand.
+// A unit is 8 stages, so that a buffer has the same size as for 2D-block scales.
+constexpr int kUnitStagesMxf8 = 8;
+constexpr int kImageStageBytesMxf8 = 1536;
 constexpr int kCompactBytes = kCacheChunks * 48;
 constexpr int kImageStageBytes = 768;        // A chunk 0, A chunk 1, B chunk 0 (rows 0..127, 128..255), B chunk 1 (same)
-constexpr int kCacheBufBytes = kUnitStages * kImageStageBytes;
+constexpr int kCacheBufBytes = kUnitStagesMxf4 * kImageStageBytes;
+static_assert(kUnitStagesMxf8 * kImageStageBytesMxf8 == kCacheBufBytes, "both kinds share the image buffers");
 constexpr int kSmemCache = kCompactBytes + 2 * kCacheBufBytes;
 // Epilogue staging of the pair kernel: each of the 8 epilogue warps owns 32 rows x 128 bytes, written from registers
 // (128-byte swizzle: the 16-byte pieces of 8 rows fall into different banks) and drained by a TMA store, which keeps
@@ -64,8 +68,7 @@ struct Cfg {
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
-    static constexpr int kSmemSf = kStages * kSfStageBytes;                       // per-row scales (MXFP8): per-stage images
-    static constexpr int kSmemScales = ((kSmemSf > kSmemCache ? kSmemSf : kSmemCache) + 1023) / 1024 * 1024;   // either kind uses the same region
+    static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
     static constexpr int kSmemStaging = CTAS == 2 ? 8 * kStagingWarpBytes : 0;
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail;
 };
@@ -533,10 +536,7 @@ __device__ __forceinline__ void build_scale_cache(const ScaleView &v, int rt0, i
     }
 }
 
-// mxf8 / 1D blocks: a stage covers 4 contraction blocks (one chunk); image row l holds rows l, l+32, l+64, l+96,
-// four scale bytes each.
-struct ScaleRegs1D { uint32_t w[3][4]; };
-
+// Per-row scales (MXFP8): one 32-bit word = the four scale bytes of one row and one stage.
 __device__ __forceinline__ void load_scale_word(const ScaleView &v, int row, int kb0, uint32_t &dst)
 {
     const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
@@ -554,24 +554,40 @@ __device__ __forceinline__ void load_scale_word(const ScaleView &v, int row, int
     dst = word;
 }
 
-__device__ __forceinline__ void fetch_scales_1d(const GemmParams &p, const Tile &t, int it, int lane, ScaleRegs1D &r)
+__device__ __forceinline__ void ldg_v4(const uint8_t *ptr, uint32_t *w)
 {
-#pragma unroll
-    for (int blk = 0; blk < 3; blk++) {   // 0: A rows 0..127; 1, 2: B rows 0..127, 128..255
-        const ScaleView &v = blk == 0 ? p.sfa : p.sfb;
-        const int row0 = blk == 0 ? t.a_row0 : t.b_row0 + (blk - 1) * 128;
-        const int kb0 = ((blk == 0 ? t.a_k0 : t.b_k0) >> 5) + it * 4;
-#pragma unroll
-        for (int j = 0; j < 4; j++) load_scale_word(v, row0 + lane + 32 * j, kb0, r.w[blk][j]);
-    }
+    asm volatile("ld.global.nc.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(ptr));
 }
 
-__device__ __forceinline__ void write_scale_images_1d(const ScaleRegs1D &r, uint8_t *sf_stage, int lane)
+// Builds the scale images of one unit (up to 8 stages = 32 contraction blocks from k0) for per-row scales.  Lane l
+// takes operand rows l, l+32, ... (4 of A, 8 of B); the 32 scale bytes of a row for the whole unit are contiguous
+// in the scale matrix, so the common case is two 16-byte loads per row, all 24 issued before any use.
+__device__ __forceinline__ void build_row_scale_images(const GemmParams &p, const Tile &t, int k0, int n_stages, uint8_t *images, int lane)
 {
-    uint4 *img = reinterpret_cast<uint4 *>(sf_stage);
-    img[(kSfaOff >> 4) + lane] = make_uint4(r.w[0][0], r.w[0][1], r.w[0][2], r.w[0][3]);
-    img[(kSfbOff >> 4) + lane] = make_uint4(r.w[1][0], r.w[1][1], r.w[1][2], r.w[1][3]);
-    img[(kSfbOff >> 4) + 32 + lane] = make_uint4(r.w[2][0], r.w[2][1], r.w[2][2], r.w[2][3]);
+    uint32_t w[12][8];
+#pragma unroll
+    for (int q = 0; q < 12; q++) {
+        const ScaleView &v = q < 4 ? p.sfa : p.sfb;
+        const int row = q < 4 ? t.a_row0 + lane + 32 * q : t.b_row0 + lane + 32 * (q - 4);
+        const int kb0 = ((q < 4 ? t.a_k0 : t.b_k0) + k0) >> 5;
+        const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
+        if (row < v.n_row && kb0 + 32 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 15) == 0) {
+            ldg_v4(ptr, w[q]);
+            ldg_v4(ptr + 16, w[q] + 4);
+        } else {
+#pragma unroll
+            for (int st = 0; st < 8; st++) load_scale_word(v, row, kb0 + 4 * st, w[q][st]);
+        }
+    }
+#pragma unroll
+    for (int st = 0; st < 8; st++) {
+        if (st < n_stages) {
+            uint4 *img = reinterpret_cast<uint4 *>(images + st * kImageStageBytesMxf8);
+            img[lane] = make_uint4(w[0][st], w[1][st], w[2][st], w[3][st]);           // A
+            img[32 + lane] = make_uint4(w[4][st], w[5][st], w[6][st], w[7][st]);      // B rows 0..127
+            img[64 + lane] = make_uint4(w[8][st], w[9][st], w[10][st], w[11][st]);    // B rows 128..255
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------- epilogue store
@@ -672,15 +688,15 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kElemsPerByte = KIND == KIND_MXF4 ? 2 : 1;
     constexpr int kStages = Cfg<CTAS>::kStages;
     constexpr int kBStageBytes = Cfg<CTAS>::kBStageBytes;
+    constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : kUnitStagesMxf8;   // stages whose scale images are built together
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_sf = smem + Cfg<CTAS>::kSmemOperands;        // MXFP8: per-stage scale images
-    uint8_t *smem_compact = smem_sf;                            // FP4: compact scale rows of the unit being built ...
-    uint8_t *smem_images = smem_sf + kCompactBytes;             // ... and two buffers of ready images
-    uint8_t *smem_staging = smem_sf + Cfg<CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
+    uint8_t *smem_compact = smem + Cfg<CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
+    uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and two buffers of ready scale images (either kind)
+    uint8_t *smem_staging = smem_compact + Cfg<CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<CTAS>::kSmemStaging);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
     // bars[14..15] scale images full, bars[16..17] scale images empty, bars[18] tensor pipe drained (abort path),
@@ -810,8 +826,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0, acc_phase = 0, unit = 0;
-        bool ok = true;
+        uint32_t stage = 0, unit = 0;
         const bool issuer = elect_one();
         int ev_j = 0;
         TRACE_DECL(c_acc); TRACE_DECL(c_sync); TRACE_DECL(c_issue);
@@ -821,13 +836,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             decode_tile(p, tile, rank, t);
             const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
             if (n_it == 0) continue;
-            if (KIND == KIND_MXF8) {   // per-row scales: the watchers alternate stages, so the accumulator is awaited here
-                if (ok) {
-                    if (lane == 0) ok = mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
-                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                }
-                acc_phase ^= 1u;
-            }
             TRACE_ADD(c_acc, tt);
             for (int it = 0; it < n_it; it++) {
                 named_sync(1 + stage);   // the watcher has seen the operands and both scale images of this stage
@@ -846,10 +854,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
                         }
                     } else {
-                        const uint32_t sf_smem = smem_u32(smem_sf + stage * kSfStageBytes);
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(sf_smem + kSfaOff));
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8, smem_desc_scale_image(sf_smem + kSfbOff));
-                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12, smem_desc_scale_image(sf_smem + kSfbOff + 512));
+                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(img));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8, smem_desc_scale_image(img + 512));
+                        tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12, smem_desc_scale_image(img + 1024));
                     }
                     const uint64_t adesc = smem_desc_sw128(smem_u32(smem_a + stage * kAStageBytes));
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(smem_b + stage * kBStageBytes));
@@ -868,7 +876,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #endif
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
                     if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
-                    if (KIND == KIND_MXF4 && ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1))
+                    if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
                         tcgen05_commit<CTAS>(bar_cache_empty + 8 * (unit & 1u));   // the unit's images have been copied
                 }
                 if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1) unit++;
@@ -887,63 +895,11 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             __syncwarp();
         }
         if (lane == 0) { TRACE_OUT(p, 2, c_acc); TRACE_OUT(p, 3, c_sync); TRACE_OUT(p, 4, c_issue); }
-    } else if ((warp == 2 || warp == 3) && KIND == KIND_MXF8) {
-        // ------------------------------------------------------------------ scale loaders, per-row scales (MXFP8)
-        // Two warps share the ring: warp 2 serves the even stages of the stream, warp 3 the odd ones (ring slots
-        // {0, 2} and {1, 3}).  Each fetches the scale words of its next two stages ahead of time and, for the stage
-        // at hand, writes the images, waits for the operands ("full") and releases the MMA warp through the stage's
-        // named barrier.  After a timeout the remaining stages are released without waiting, so that the MMA warp,
-        // which cannot time out on a named barrier, always runs to its end.  (One CTA per tile only.)
-        const int which = warp - 2;
-        ScaleRegs1D pre[2];
-        StageIter fetch_it, write_it;
-        fetch_it.init(p, first_tile, tile_step, rank, kStageElems);
-        write_it.init(p, first_tile, tile_step, rank, kStageElems);
-        if (which == 1) {
-            if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
-            if (write_it.valid(p)) write_it.next(p, kStageElems);
-        }
-#pragma unroll
-        for (int d = 0; d < 2; d++) {
-            if (fetch_it.valid(p)) {
-                fetch_scales_1d(p, fetch_it.t, fetch_it.it, lane, pre[d]);
-                fetch_it.next(p, kStageElems);
-                if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
-            }
-        }
-        uint32_t phase = 0;
-        bool ok = true;
-        while (write_it.valid(p)) {
-#pragma unroll
-            for (int d = 0; d < 2; d++) {
-                if (!write_it.valid(p)) break;
-                const int stage = 2 * d + which;
-                if (ok) {
-                    if (lane == 0) ok = mbar_wait_relaxed(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x300u + stage);
-                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                }
-                if (ok) {
-                    write_scale_images_1d(pre[d], smem_sf + stage * kSfStageBytes, lane);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
-                    __syncwarp();
-                    if (lane == 0) ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status, 0x310u + stage);
-                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                }
-                named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
-                if (ok && fetch_it.valid(p)) {
-                    fetch_scales_1d(p, fetch_it.t, fetch_it.it, lane, pre[d]);
-                    fetch_it.next(p, kStageElems);
-                    if (fetch_it.valid(p)) fetch_it.next(p, kStageElems);
-                }
-                write_it.next(p, kStageElems);
-                if (write_it.valid(p)) write_it.next(p, kStageElems);
-            }
-            phase ^= 1u;
-        }
     } else if (warp == 3) {
-        // ------------------------------------------------------------------ scale image builder, 2D-block scales
-        // Per unit (up to 16 stages of one tile) gathers the compact scale bytes from global memory into 16-byte rows
-        // and replicates each row into its image.  Two image buffers alternate, so the next unit is built while
+        // ------------------------------------------------------------------ scale image builder
+        // 2D-block scales: per unit (up to 16 stages of one tile) gathers the compact scale bytes from global memory
+        // into 16-byte rows and replicates each row into its image; per-row scales: loads the unit's scale words and
+        // writes the 32-row images directly.  Two image buffers alternate, so the next unit is built while
         // the current one runs: all global-memory latency of the scale path is paid here, off the per-stage
         // critical path, and nothing has to be written per stage.  A buffer is free again once the MMA warp's
         // commit reports that the last scale copy out of it has completed.  In a pair each CTA builds the images
@@ -953,33 +909,42 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
             decode_tile(p, tile, rank, t);
-            for (int k0 = 0; ok && k0 < t.k_len; k0 += kCacheChunks * 128, unit++) {
+            for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, unit++) {
                 const int buf = unit & 1;
-                const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
-                uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
-                build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, compact, lane);
-                build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
-                __syncwarp();
-                if (lane == 0)
-                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
-                                   : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
-                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                if (!ok) break;
-                const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
                 uint8_t *images = smem_images + buf * kCacheBufBytes;
-                for (int q = lane; q < 3 * n_chunks; q += 32) {
-                    uint4 row;
-                    uint8_t *dst;
-                    if (q < n_chunks) {                       // A, chunk q
-                        row = rows[q];
-                        dst = images + (q >> 1) * kImageStageBytes + (q & 1) * 128;
-                    } else {                                  // B, chunk (q - n_chunks) / 2, rows 0..127 or 128..255
-                        const int qb = q - n_chunks, chunk = qb >> 1;
-                        row = rows[kCacheChunks + qb];
-                        dst = images + (chunk >> 1) * kImageStageBytes + 256 + (chunk & 1) * 256 + (qb & 1) * 128;
-                    }
+                if (KIND == KIND_MXF8) {
+                    // per-row scales: straight from global memory into the images
+                    if (lane == 0)
+                        ok = mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                    if (!ok) break;
+                    build_row_scale_images(p, t, k0, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images, lane);
+                } else {
+                    const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
+                    uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
+                    build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, compact, lane);
+                    build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
+                    __syncwarp();
+                    if (lane == 0)
+                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
+                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                    if (!ok) break;
+                    const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
+                    for (int q = lane; q < 3 * n_chunks; q += 32) {
+                        uint4 row;
+                        uint8_t *dst;
+                        if (q < n_chunks) {                       // A, chunk q
+                            row = rows[q];
+                            dst = images + (q >> 1) * kImageStageBytes + (q & 1) * 128;
+                        } else {                                  // B, chunk (q - n_chunks) / 2, rows 0..127 or 128..255
+                            const int qb = q - n_chunks, chunk = qb >> 1;
+                            row = rows[kCacheChunks + qb];
+                            dst = images + (chunk >> 1) * kImageStageBytes + 256 + (chunk & 1) * 256 + (qb & 1) * 128;
+                        }
 #pragma unroll
-                    for (int r = 0; r < 8; r++) reinterpret_cast<uint4 *>(dst)[r] = row;
+                        for (int r = 0; r < 8; r++) reinterpret_cast<uint4 *>(dst)[r] = row;
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
@@ -990,7 +955,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
         }
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ watcher, 2D-block scales
+        // ------------------------------------------------------------------ watcher
         // Follows the stream of stages (one CTA, or the leader of a pair; the second CTA's warp idles).  For each
         // it waits for the ring slot's "full" barrier (the operand bytes of both CTAs), at the first stage of a
         // unit for the unit's scale images (of both CTAs), and at the first stage of a tile for the accumulator
@@ -1095,8 +1060,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             uint32_t v[4][32];
             if (t.k_len > 0) {
                 if (lane == 0)
-                    ok = CTAS == 2 ? mbar_poll_relaxed(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp)
-                                   : mbar_wait_lazy(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
+                    ok = CTAS == 2 ? mbar_poll(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp)
+                                   : mbar_wait_relaxed(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 TRACE_ADD(c_wait, tt);
                 if (lane == 0) TRACE_EV(7, 16 * ev_t + 2 * (warp - 4));
