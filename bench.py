@@ -324,6 +324,7 @@ def run_gpu(args):
                                "match the %s regime" % (peaks["source"], regime, bf16_peak, FP4_OVER_BF16, regime),
                 "frac_of_burst_peak": achieved_tf / (peaks["bf16_tflops"] * FP4_OVER_BF16),
                 "frac_of_sustained_peak": achieved_tf / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16),
+                "frac_of_nominal_9pf": achieved_tf / 9000.0,
                 "flops_per_launch": 3 * gemm_flops / (3 * len(ops)), "ms_per_launch": gemm_ms_per_launch,
                 "time_share_of_step": (f_ms + d_ms + w_ms) / ms_per_step}
     q_gbs_1 = quant_bytes / (q_ms * 1e-3) / 1e9

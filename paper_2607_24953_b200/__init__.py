@@ -3,4 +3,4 @@
 The product is the C-ABI library ``libfp4q.so`` (declared in ``include/fp4q.h``); ``binding`` is its
 thin Python face and ``workloads`` the seeded synthetic input generators.
 """
-__all__ = ["binding", "workloads", "build"]
+__all__ = ["binding", "workloads", "build", "autograd"]
