@@ -403,7 +403,21 @@ def run_extras(torch, binding, workloads, dev, ws):
     out["mxfp8_qk"] = {"workload": "Q and K projections, %d tokens, %dx%d each" % (T, H, H),
                        "quantize_gbs": T * H * (3.0 + 1 / 32) / (ms_q * 1e-3) / 1e9,
                        "gemm_tflops": 2 * 2.0 * T * H * H / (ms_g * 1e-3) / 1e12, "gemm_ms": ms_g}
-    del X, Wq, Wk, xq, xs, wqq, wqs, wkq, wks
+    del xq, xs, wqq, wqs, wkq, wks
+
+    # --- forward product with the output quantization fused into the epilogue, against product + separate quantize
+    qx4, qw4 = binding.fp4q_quantize2d(X), binding.fp4q_quantize2d(Wq)
+    y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+    qy = binding.alloc_qtensor(T, H, dev)
+    SR = binding.ROUND_STOCHASTIC
+    ms_f = timed(lambda: binding.fp4q_gemm_fwd_quantized(qx4, qw4, out=qy, mode=SR, seed=1, tensor_id=2, ws=ws))
+    ms_p = timed(lambda: binding.fp4q_gemm_fwd(qx4, qw4, out=y, ws=ws))
+    ms_s = timed(lambda: binding.fp4q_quantize2d(y, out=qy, mode=SR, seed=1, tensor_id=2))
+    out["fused_epilogue_quantization"] = {
+        "workload": "Y = X W^T, %d x %d x %d, output as 2D-block FP4 (stochastic rounding)" % (T, H, H),
+        "fused_ms": ms_f, "product_ms": ms_p, "separate_quantize_ms": ms_s,
+        "fused_tflops": 2.0 * T * H * H / (ms_f * 1e-3) / 1e12, "speedup_vs_unfused": (ms_p + ms_s) / ms_f}
+    del X, Wq, Wk, qx4, qw4, y, qy
 
     # --- grouped MoE expert layer: 128 experts, hidden 2048, expert FFN 768, top-8 of 16384 tokens
     moe = workloads.CONFIG_MOE

@@ -177,6 +177,21 @@ fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, i
                           void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * fp4q_gemm_fwd_quantized -- the dense forward product with the output quantization fused into the GEMM's epilogue
+ * (Section 3.1 feeds each layer's BF16 output to the next layer's quantizer; here the tile is quantized while it is
+ * still in registers):
+ *   Y = X^ W^^T with FP32 accumulation, rounded to BF16, then Yq = 2D-block FP4 of Y exactly as fp4q_quantize2d
+ *   computes it from that BF16 matrix with the same mode, seed and tensor_id (element index i*N + j): same block
+ *   maxima, scales, codes, both payload layouts; Y itself is never written.
+ * X [T,K], W [N,K] as for fp4q_gemm_fwd (dense form).  Yq: rows = T, cols = N, layouts and alignment as for
+ * fp4q_quantize2d (q_t may be NULL).  N must be a multiple of 16 (FP4Q_ERR_UNSUPPORTED otherwise); T is free.
+ * ws/ws_bytes/stream and the asynchronous FP4Q_ERR_TIMEOUT report are those of fp4q_gemm_fwd.
+ */
+fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, const fp4q_tensor *Yq,
+                                    fp4q_round mode, uint64_t seed, uint32_t tensor_id,
+                                    void *ws, size_t ws_bytes, void *stream);
+
+/*
  * fp4q_gemm_fwd_static_workspace -- no counterpart in the paper: the dense forward product of
  * fp4q_gemm_fwd for callers that cannot allocate device memory (code living inside an application that
  * owns the device heap, a loop that must stay out of the allocator, a sandbox restricted to buffers it was

@@ -86,6 +86,10 @@ def lib() -> ctypes.CDLL:
             L.fp4q_gemm_fwd_static_workspace.restype = ci
             L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
                                                          ci, vp, vp]
+        if hasattr(L, "fp4q_gemm_fwd_quantized"):
+            L.fp4q_gemm_fwd_quantized.restype = ci
+            L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
+                                                  ctypes.POINTER(_CTensor), ci, u64, u32, vp, ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -223,6 +227,21 @@ def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offs
     """Y[T,N] = X^ W^^T. Grouped when row_offsets is given (W is then the expert stack [E*N, K])."""
     n = W.rows if row_offsets is None else W.rows // (row_offsets.numel() - 1)
     return _gemm("fp4q_gemm_fwd", X, W, X.rows, n, out, dt, row_offsets, ws, stream)
+
+
+def fp4q_gemm_fwd_quantized(X: QTensor, W: QTensor, out: Optional[QTensor] = None, mode: int = ROUND_NEAREST,
+                            seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None) -> QTensor:
+    """Yq = 2D-block FP4 of the BF16-rounded product X^ W^^T, quantized in the GEMM's epilogue."""
+    dev = X.q_rm.device
+    if out is None:
+        out = alloc_qtensor(X.rows, W.rows, dev, want_t)
+    if ws is None:
+        ws = alloc_workspace(dev)
+    cx, cw, cy = X.c_struct(), W.c_struct(), out.c_struct()
+    st = lib().fp4q_gemm_fwd_quantized(ctypes.byref(cx), ctypes.byref(cw), ctypes.byref(cy), mode, seed, tensor_id,
+                                       ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "fp4q_gemm_fwd_quantized")
+    return out
 
 
 def fp4q_gemm_fwd_static_workspace(X: QTensor, W: QTensor, out: torch.Tensor, dt: int = OUT_BF16,

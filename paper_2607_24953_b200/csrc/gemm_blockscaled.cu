@@ -30,6 +30,7 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include "quant_device.cuh"
 
 namespace fp4q {
 
@@ -133,7 +134,15 @@ struct GemmParams {
     int32_t b_rows_per_group;        // grouped rows: B row offset per group (forward)
     int32_t b_k_per_group;           // grouped rows: B contraction offset per group (dgrad)
     uint32_t *status;
+    // quantizing epilogue (EPI_QUANT): the output leaves as a 2D-block FP4 tensor instead of BF16/FP32
+    uint8_t *q_rm, *q_t, *q_scale;
+    int64_t q_ld_rm, q_ld_t, q_ld_s;
+    int32_t q_mode;                  // FP4Q_ROUND_NEAREST or FP4Q_ROUND_STOCHASTIC
+    uint32_t q_tensor_id;
+    PhiloxRoundKeys q_keys;
 };
+
+enum { EPI_STORE = 0, EPI_QUANT = 1 };
 
 struct Tile {
     int32_t a_row0, b_row0, b_load_row0, a_k0, b_k0, k_len, c_row0, c_col0, m_valid, n_valid;
@@ -678,7 +687,7 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
 
 // ---------------------------------------------------------------------------------------- kernel
 
-template <int KIND, int CTAS>
+template <int KIND, int CTAS, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmC, const __grid_constant__ GemmParams p)
@@ -1092,7 +1101,73 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #ifdef FP4Q_SKIP_STORE   // development only: results are dropped
             if (row_ok && p.M < 0) {
 #else
-            if (CTAS == 2) {
+            if (EPI == EPI_QUANT) {
+                // The output tile leaves as 2D-block FP4: each warp owns four 32x32 blocks (its 32 rows x 32 columns
+                // per chunk).  The accumulator is rounded to BF16 first, so the result equals fp4q_quantize2d applied
+                // to the BF16 output of the plain product: block maximum over the warp, truncation-free scale, E2M1
+                // codes by the same converts, row-major payload from the lane's own row, transposed payload gathered
+                // through the warp's staging rows.
+                uint32_t *stg = reinterpret_cast<uint32_t *>(smem_staging + (warp - 4) * kStagingWarpBytes);
+                const int64_t row_g = (int64_t)t.c_row0 + row_in_tile;
+                const int row0_blk = t.c_row0 + 32 * quarter;
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const int col0 = t.c_col0 + 128 * half + 32 * j;
+                    if (col0 >= p.N || row0_blk >= p.M) continue;   // warp-uniform
+                    uint32_t raw[16], mx = 0;
+                    bool nonfinite = false;
+#pragma unroll
+                    for (int e = 0; e < 16; e++) {
+                        const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(v[j][2 * e]), __uint_as_float(v[j][2 * e + 1]));
+                        raw[e] = *reinterpret_cast<const uint32_t *>(&b);
+                        const uint32_t m0 = raw[e] & 0x7FFFu, m1 = (raw[e] >> 16) & 0x7FFFu;
+                        nonfinite |= m0 >= 0x7F80u || m1 >= 0x7F80u;
+                        mx = max(mx, max(m0 >= 0x7F80u ? 0u : m0, m1 >= 0x7F80u ? 0u : m1));
+                    }
+                    mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+                    nonfinite = __any_sync(0xFFFFFFFFu, nonfinite);
+                    const int code = scale_code_from_max(mx);
+                    uint32_t W[4];
+#pragma unroll
+                    for (int sg = 0; sg < 2; sg++) {
+                        uint32_t R[4] = {0u, 0u, 0u, 0u};
+                        if (p.q_mode == FP4Q_ROUND_STOCHASTIC) {
+                            const uint64_t blk = (uint64_t)(row_g * p.N + col0 + 16 * sg) >> 4;   // N % 16 == 0
+                            philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.q_tensor_id, 0u, p.q_keys, R);
+                        }
+                        if (nonfinite) {
+                            const uint4 lo = make_uint4(raw[8 * sg], raw[8 * sg + 1], raw[8 * sg + 2], raw[8 * sg + 3]);
+                            const uint4 hi = make_uint4(raw[8 * sg + 4], raw[8 * sg + 5], raw[8 * sg + 6], raw[8 * sg + 7]);
+                            const uint4 rn = make_uint4(R[0], R[1], R[2], R[3]);
+                            const uint2 w = p.q_mode == FP4Q_ROUND_STOCHASTIC
+                                                ? round_segment_scalar<FP4Q_ROUND_STOCHASTIC>(lo, hi, rn, inv_scale_f16_aligned(code))
+                                                : round_segment_scalar<FP4Q_ROUND_NEAREST>(lo, hi, rn, inv_scale_f16_aligned(code));
+                            W[2 * sg] = w.x;
+                            W[2 * sg + 1] = w.y;
+                        } else if (p.q_mode == FP4Q_ROUND_STOCHASTIC) {
+                            round_segment<FP4Q_ROUND_STOCHASTIC>(raw + 8 * sg, inv_scale(code), R, W + 2 * sg);
+                        } else {
+                            round_segment<FP4Q_ROUND_NEAREST>(raw + 8 * sg, inv_scale(code), R, W + 2 * sg);
+                        }
+                    }
+                    if (row_ok) *reinterpret_cast<uint4 *>(p.q_rm + row_g * p.q_ld_rm + (col0 >> 1)) = make_uint4(W[0], W[1], W[2], W[3]);
+                    if (lane == 0) p.q_scale[(int64_t)(row0_blk >> 5) * p.q_ld_s + (col0 >> 5)] = (uint8_t)code;
+                    if (p.q_t != nullptr) {
+                        // lane r parks its row's 32 nibbles; lane c then collects nibble c of every row
+                        __syncwarp();
+                        *reinterpret_cast<uint4 *>(stg + 4 * lane) = make_uint4(W[0], W[1], W[2], W[3]);
+                        __syncwarp();
+                        uint32_t T4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                        for (int r = 0; r < 32; r++) {
+                            const uint32_t word = stg[4 * r + (lane >> 3)];
+                            T4[r >> 3] |= ((word >> (4 * (lane & 7))) & 0xFu) << (4 * (r & 7));
+                        }
+                        if (col0 + lane < p.N)
+                            *reinterpret_cast<uint4 *>(p.q_t + (int64_t)(col0 + lane) * p.q_ld_t + (row0_blk >> 1)) = make_uint4(T4[0], T4[1], T4[2], T4[3]);
+                    }
+                }
+            } else if (CTAS == 2) {
                 // Pair kernel (dense products only): 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
                 // through this warp's staging rows and leave by a TMA store, which clips rows and columns past the
                 // output's edge.  With accumulation the store is the TMA's FP32 add-reduction.
@@ -1219,13 +1294,14 @@ static int sm_count()
     return n;
 }
 
-template <int KIND, int CTAS>
+template <int KIND, int CTAS, int EPI = EPI_STORE>
 static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmParams &p, void *stream)
 {
     CUtensorMap tmA, tmB, tmC;
     const int64_t out_rows = p.mode == MODE_GROUPED_K ? (int64_t)p.n_groups * p.M : p.M;
-    if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
     if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
+    if (EPI == EPI_QUANT) tmC = tmA;   // unused by the quantizing epilogue
+    else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
 #ifdef FP4Q_SPLIT_B
     if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, 128)) return FP4Q_ERR_CUDA;
 #else
@@ -1241,7 +1317,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
 
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  Cfg<CTAS>::kSmemBytes) != cudaSuccess)
             return FP4Q_ERR_CUDA;
         attr_set = true;
@@ -1263,7 +1339,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = CTAS == 2 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS>, tmA, tmB, tmC, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS, EPI>, tmA, tmB, tmC, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }
 
 template <int KIND>
@@ -1357,6 +1433,39 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
         p.b_rows_per_group = (int32_t)N; p.b_k_per_group = 0;
     }
     return launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, const fp4q_tensor *Yq, fp4q_round mode,
+                                               uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(X) || !tensor_ok(W) || !tensor_ok(Yq)) return X && W && Yq ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
+    if (X->cols != W->cols) return FP4Q_ERR_SHAPE;
+    const int64_t T = X->rows, K = X->cols, N = W->rows;
+    if (Yq->rows != T || Yq->cols != N) return FP4Q_ERR_SHAPE;
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (N % 16 != 0) return FP4Q_ERR_UNSUPPORTED;   // one Philox block per 16-element row segment of the output
+    if (T == 0 || N == 0) return FP4Q_OK;
+    if (!X->q_rm || !W->q_rm || !X->scale || !W->scale || !Yq->q_rm || !Yq->scale) return FP4Q_ERR_NULL;
+    if (Yq->ld_rm < round_up(N, 32) / 2 || Yq->ld_s < ceil_div(N, 32)) return FP4Q_ERR_SHAPE;
+    if (Yq->q_t && Yq->ld_t < round_up(T, 32) / 2) return FP4Q_ERR_SHAPE;
+    if (!aligned(Yq->q_rm, 16) || Yq->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
+    if (Yq->q_t && (!aligned(Yq->q_t, 16) || Yq->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
+    if (!ws || ws_bytes < sizeof(Workspace)) return FP4Q_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return FP4Q_ERR_ALIGN;
+    const Operand A = operand_rm(X), B = operand_rm(W);
+    if (!aligned(A.payload, 16) || !aligned(B.payload, 16) || A.ld_bytes % 16 || B.ld_bytes % 16) return FP4Q_ERR_ALIGN;
+    GemmParams p = {};
+    p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)K;
+    dense_tiles(p);
+    p.sfa = A.sf; p.sfb = B.sf;
+    p.status = reinterpret_cast<uint32_t *>(ws);
+    p.q_rm = Yq->q_rm; p.q_ld_rm = Yq->ld_rm;
+    p.q_t = Yq->q_t; p.q_ld_t = Yq->ld_t;
+    p.q_scale = Yq->scale; p.q_ld_s = Yq->ld_s;
+    p.q_mode = (int32_t)mode; p.q_tensor_id = tensor_id;
+    philox_round_keys(seed, p.q_keys);
+    return launch_gemm_impl<KIND_MXF4, 2, EPI_QUANT>(A, B, p, stream);
 }
 
 extern "C" fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt,

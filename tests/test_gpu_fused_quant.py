@@ -1,0 +1,79 @@
+"""GPU parity of fp4q_gemm_fwd_quantized: the forward product whose epilogue emits the 2D-block FP4 encoding of its
+own BF16-rounded output.
+
+Oracle: quantize2d(BF16(gemm_fwd(X^, W^))).  FP32 accumulation order is not the oracle's, so a bit-exact comparison
+with the oracle needs operands for which every partial sum is exact (E2M1-grid values times a power of two): then
+the GPU's BF16 output is the oracle's and payloads and scales must agree bit for bit.  On general operands the fused
+call is compared, bit for bit, with the unfused chain (fp4q_gemm_fwd to BF16, then fp4q_quantize2d), whose two
+halves are each tied to the oracle by their own tests."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_24953_b200 import binding, workloads
+from tests.gpu_util import assert_matches_oracle, dequant_from_gpu, logical
+
+pytestmark = pytest.mark.gpu
+
+
+def compare_logical(got, want_rm, want_t, want_s, rows, cols):
+    g_rm, g_t, g_s = logical(got)
+    assert np.array_equal(g_s, want_s), "scales differ"
+    w = (cols + 1) // 2
+    assert np.array_equal(g_rm[:, :w], want_rm[:, :w]), "row-major payload differs"
+    assert not g_rm[:, w:(cols + 31) // 32 * 16].any(), "row-major block padding is not zero"
+    h = (rows + 1) // 2
+    assert np.array_equal(g_t[:, :h], want_t[:, :h]), "transposed payload differs"
+    assert not g_t[:, h:(rows + 31) // 32 * 16].any(), "transposed block padding is not zero"
+
+
+@pytest.mark.parametrize("T", [256, 200, 97])
+@pytest.mark.parametrize("mode", [oracle.MODE_NEAREST, oracle.MODE_STOCHASTIC])
+def test_exact_operands_match_the_oracle_bit_for_bit(T, mode):
+    g = torch.Generator(device="cuda").manual_seed(5)
+    grid = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6], device="cuda")
+
+    def draw(r, c, e):
+        v = grid[torch.randint(0, 8, (r, c), generator=g, device="cuda")]
+        s = torch.randint(0, 2, (r, c), generator=g, device="cuda") * 2 - 1
+        return (v * s * 2.0 ** e).to(torch.bfloat16)
+
+    N, K = 400, 512
+    X, W = draw(T, K, -3), draw(N, K, 5)
+    qx = assert_matches_oracle(X, 0, seed=0, tensor_id=0)
+    qw = assert_matches_oracle(W, 0, seed=0, tensor_id=1)
+    xd, wd = dequant_from_gpu(qx), dequant_from_gpu(qw)
+    ws = binding.alloc_workspace("cuda")
+    yq = binding.fp4q_gemm_fwd_quantized(qx, qw, mode=mode, seed=9, tensor_id=4, ws=ws)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    y = oracle.bf16_round(oracle.gemm_fwd(xd, wd))                       # exact sums, rounded to BF16
+    y_bits = workloads.bf16_bits(torch.from_numpy(y).to(torch.bfloat16))  # already representable: no second rounding
+    o_rm, o_t, o_s = oracle.quantize2d(y_bits, mode, 9, 4)
+    compare_logical(yq, o_rm, o_t, o_s, T, N)
+
+
+@pytest.mark.parametrize("T,N,K", [(128, 256, 256), (300, 272, 1000), (1000, 1040, 320), (33, 16, 64)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_fused_equals_product_then_quantize(T, N, K, mode):
+    X = workloads.activations_student_t(T, K, 700, "cuda")
+    W = workloads.weights(N, K, 701, "cuda")
+    qx = binding.fp4q_quantize2d(X, mode=0)
+    qw = binding.fp4q_quantize2d(W, mode=0)
+    ws = binding.alloc_workspace("cuda")
+    fused = binding.fp4q_gemm_fwd_quantized(qx, qw, mode=mode, seed=3, tensor_id=8, ws=ws)
+    y = binding.fp4q_gemm_fwd(qx, qw, dt=binding.OUT_BF16, ws=ws)
+    chain = binding.fp4q_quantize2d(y.contiguous(), mode=mode, seed=3, tensor_id=8)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    c_rm, c_t, c_s = logical(chain)
+    compare_logical(fused, c_rm, c_t, c_s, T, N)
+
+
+def test_output_width_must_be_a_multiple_of_16():
+    X = workloads.weights(64, 64, 1, "cuda")
+    W = workloads.weights(40, 64, 2, "cuda")
+    qx, qw = binding.fp4q_quantize2d(X), binding.fp4q_quantize2d(W)
+    with pytest.raises(binding.Fp4qError):
+        binding.fp4q_gemm_fwd_quantized(qx, qw)
