@@ -471,8 +471,20 @@ def cpu_baseline_quantize(workloads, cfg, seconds=12.0):
     t0 = time.perf_counter()
     oracle.quantize2d(x, oracle.MODE_STOCHASTIC, seed=cfg.philox_seed, tensor_id=7)
     dt = time.perf_counter() - t0
+    # the GEMM oracle (dequantize + float64 matmul) on a row sample of the largest forward product
+    g_rows = 256
+    xs = x[:g_rows]
+    wbits = workloads.bf16_bits(workloads.weights(512, cols, cfg.data_seed + 60, "cpu"))
+    qx, qw = oracle.quantize2d(xs, oracle.MODE_NEAREST), oracle.quantize2d(wbits, oracle.MODE_NEAREST)
+    t1 = time.perf_counter()
+    xd = oracle.dequantize2d(qx[0], qx[2], g_rows, cols)
+    wd = oracle.dequantize2d(qw[0], qw[2], 512, cols)
+    oracle.gemm_fwd(xd, wd)
+    g_dt = max(time.perf_counter() - t1, 1e-9)
     return {"value": rows * cols * BYTES_PER_ELEMENT / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
             "kind": "oracle", "seconds": dt,
+            "gemm": {"value": 2.0 * g_rows * 512 * cols / g_dt / 1e9, "unit": "GFLOP/s",
+                     "sample": "forward product oracle (dequantize + float64 matmul) on %d x 512 x %d" % (g_rows, cols)},
             "sample": "quantize+dual-pack (stochastic) of a %dx%d row slab of the %dx%d down-projection activation" %
                       (rows, cols, cfg.tokens, cols)}
 
