@@ -601,6 +601,37 @@ __device__ __forceinline__ void build_row_scale_images(const GemmParams &p, cons
 
 // ---------------------------------------------------------------------------------------- epilogue store
 
+// Transpose of a 32x32 matrix of nibbles held one row per lane (W[w] nibble n = column 8w + n of the lane's row): on
+// return lane c holds column c (W[w] nibble n = row 8w + n).  Five exchange steps, one per index bit: lanes that
+// differ in bit b swap the elements whose position bit b differs from their own lane bit b (whole words for the
+// two word-index bits, masked and shifted nibble groups for the three nibble-index bits).
+__device__ __forceinline__ void transpose32x32_nibbles(uint32_t W[4], int lane)
+{
+    {   // position bit 4 = word bit 1: words {2,3} <-> {0,1} between lanes 16 apart
+        const bool up = lane & 16;
+        const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, up ? W[0] : W[2], 16);
+        const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, up ? W[1] : W[3], 16);
+        if (up) { W[0] = r0; W[1] = r1; } else { W[2] = r0; W[3] = r1; }
+    }
+    {   // position bit 3 = word bit 0: words {1,3} <-> {0,2} between lanes 8 apart
+        const bool up = lane & 8;
+        const uint32_t r0 = __shfl_xor_sync(0xFFFFFFFFu, up ? W[0] : W[1], 8);
+        const uint32_t r1 = __shfl_xor_sync(0xFFFFFFFFu, up ? W[2] : W[3], 8);
+        if (up) { W[0] = r0; W[2] = r1; } else { W[1] = r0; W[3] = r1; }
+    }
+#pragma unroll
+    for (int b = 2; b >= 0; b--) {   // nibble-index bits: groups of 4, 2, 1 nibbles between lanes 4, 2, 1 apart
+        const uint32_t lo = b == 2 ? 0x0000FFFFu : b == 1 ? 0x00FF00FFu : 0x0F0F0F0Fu;
+        const int sh = 4 << b;
+        const bool up = lane & (1 << b);
+#pragma unroll
+        for (int w = 0; w < 4; w++) {
+            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, W[w], 1 << b);
+            W[w] = up ? ((W[w] & ~lo) | ((other & ~lo) >> sh)) : ((W[w] & lo) | ((other & lo) << sh));
+        }
+    }
+}
+
 // One round of the pair kernel's epilogue: 32 words per lane (this lane's row, 128 bytes) into the warp's swizzled
 // staging rows, then one TMA store (kind 0: BF16 bytes, 1: FP32 bytes, 2: FP32 add-reduction) of the 32 x 128 B box.
 __device__ __forceinline__ void stage_and_store(const CUtensorMap *map, const uint32_t *w, uint32_t stg_row, uint32_t swz,
@@ -690,7 +721,8 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
 template <int KIND, int CTAS, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                         const __grid_constant__ CUtensorMap tmC, const __grid_constant__ GemmParams p)
+                         const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
+                         const __grid_constant__ GemmParams p)
 {
     constexpr int kStageElems = KIND == KIND_MXF4 ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = KIND == KIND_MXF4 ? 64 : 32;           // contraction elements per MMA (32 B per row)
@@ -744,6 +776,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
         if (CTAS == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
+        if (EPI == EPI_QUANT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
     }
     if (warp == 1) {
         if (CTAS == 1) {
@@ -1105,11 +1138,19 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 // The output tile leaves as 2D-block FP4: each warp owns four 32x32 blocks (its 32 rows x 32 columns
                 // per chunk).  The accumulator is rounded to BF16 first, so the result equals fp4q_quantize2d applied
                 // to the BF16 output of the plain product: block maximum over the warp, truncation-free scale, E2M1
-                // codes by the same converts, row-major payload from the lane's own row, transposed payload gathered
-                // through the warp's staging rows.
-                uint32_t *stg = reinterpret_cast<uint32_t *>(smem_staging + (warp - 4) * kStagingWarpBytes);
+                // codes by the same converts, row-major payload from the lane's own row, transposed payload by a
+                // 32x32 nibble transpose across the warp's lanes; both leave through the staging rows and TMA stores.
                 const int64_t row_g = (int64_t)t.c_row0 + row_in_tile;
                 const int row0_blk = t.c_row0 + 32 * quarter;
+                // staging: 32 rows x 64 B of row-major payload (64-byte swizzle) and 128 rows x 16 B of transposed payload
+                uint8_t *stg = smem_staging + (warp - 4) * kStagingWarpBytes;
+                const uint32_t stg_rm = smem_u32(stg) + lane * 64, swz = (uint32_t)((lane >> 1) & 3);
+                const uint32_t stg_t = smem_u32(stg) + 2048 + lane * 16;
+                const bool any = row0_blk < p.M && t.c_col0 + 128 * half < p.N;   // warp-uniform: something to write
+                if (any) {
+                    if (lane == 0) bulk_wait_read_all();   // the previous tile's stores have read the staging rows
+                    __syncwarp();
+                }
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const int col0 = t.c_col0 + 128 * half + 32 * j;
@@ -1150,21 +1191,23 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             round_segment<FP4Q_ROUND_NEAREST>(raw + 8 * sg, inv_scale(code), R, W + 2 * sg);
                         }
                     }
-                    if (row_ok) *reinterpret_cast<uint4 *>(p.q_rm + row_g * p.q_ld_rm + (col0 >> 1)) = make_uint4(W[0], W[1], W[2], W[3]);
                     if (lane == 0) p.q_scale[(int64_t)(row0_blk >> 5) * p.q_ld_s + (col0 >> 5)] = (uint8_t)code;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg_rm + (((uint32_t)j ^ swz) << 4)), "r"(W[0]), "r"(W[1]),
+                                 "r"(W[2]), "r"(W[3]) : "memory");
                     if (p.q_t != nullptr) {
-                        // lane r parks its row's 32 nibbles; lane c then collects nibble c of every row
-                        __syncwarp();
-                        *reinterpret_cast<uint4 *>(stg + 4 * lane) = make_uint4(W[0], W[1], W[2], W[3]);
-                        __syncwarp();
-                        uint32_t T4[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                        for (int r = 0; r < 32; r++) {
-                            const uint32_t word = stg[4 * r + (lane >> 3)];
-                            T4[r >> 3] |= ((word >> (4 * (lane & 7))) & 0xFu) << (4 * (r & 7));
-                        }
-                        if (col0 + lane < p.N)
-                            *reinterpret_cast<uint4 *>(p.q_t + (int64_t)(col0 + lane) * p.q_ld_t + (row0_blk >> 1)) = make_uint4(T4[0], T4[1], T4[2], T4[3]);
+                        transpose32x32_nibbles(W, lane);   // lane c now holds column c: nibble r = row r of the block
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg_t + 512u * j), "r"(W[0]), "r"(W[1]), "r"(W[2]),
+                                     "r"(W[3]) : "memory");
+                    }
+                }
+                if (any) {
+                    // both payloads leave by TMA stores, which clip at the tensors' edges (rows past T, columns past N)
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmC, (t.c_col0 + 128 * half) >> 1, row0_blk, smem_u32(stg));
+                        if (p.q_t != nullptr) tma_store_2d(&tmD, row0_blk >> 1, t.c_col0 + 128 * half, smem_u32(stg) + 2048);
+                        bulk_commit();
                     }
                 }
             } else if (CTAS == 2) {
@@ -1208,7 +1251,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
-        if (CTAS == 2 && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
+        if ((CTAS == 2 || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
         if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
@@ -1277,6 +1320,20 @@ static bool make_output_map(CUtensorMap *map, void *base, int64_t rows, int64_t 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Plain byte matrix [rows, row_bytes] with pitch ld_bytes as a store target.
+static bool make_byte_map(CUtensorMap *map, void *base, int64_t rows, int64_t row_bytes, int64_t ld_bytes, int box_bytes,
+                          int box_rows, CUtensorMapSwizzle swizzle)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Operand {
     const uint8_t *payload;
     int64_t rows, row_bytes, ld_bytes;
@@ -1300,8 +1357,13 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     CUtensorMap tmA, tmB, tmC;
     const int64_t out_rows = p.mode == MODE_GROUPED_K ? (int64_t)p.n_groups * p.M : p.M;
     if (!make_operand_map(&tmA, A.payload, A.rows, A.row_bytes, A.ld_bytes, BM)) return FP4Q_ERR_CUDA;
-    if (EPI == EPI_QUANT) tmC = tmA;   // unused by the quantizing epilogue
-    else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
+    CUtensorMap tmD = tmA;   // second output map: only the quantizing epilogue has one
+    if (EPI == EPI_QUANT) {
+        // row-major payload [T, ceil32(N)/2] bytes, box 64 B x 32 rows (64-byte swizzle); transposed payload
+        // [N, ceil32(T)/2] bytes, box 16 B x 128 rows
+        if (!make_byte_map(&tmC, p.q_rm, p.M, round_up(p.N, 32) / 2, p.q_ld_rm, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return FP4Q_ERR_CUDA;
+        if (p.q_t && !make_byte_map(&tmD, p.q_t, p.N, round_up(p.M, 32) / 2, p.q_ld_t, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) return FP4Q_ERR_CUDA;
+    } else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
 #ifdef FP4Q_SPLIT_B
     if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, 128)) return FP4Q_ERR_CUDA;
 #else
@@ -1339,7 +1401,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = CTAS == 2 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS, EPI>, tmA, tmB, tmC, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS, EPI>, tmA, tmB, tmC, tmD, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }
 
 template <int KIND>
