@@ -403,7 +403,20 @@ def run_extras(torch, binding, workloads, dev, ws):
     out["mxfp8_qk"] = {"workload": "Q and K projections, %d tokens, %dx%d each" % (T, H, H),
                        "quantize_gbs": T * H * (3.0 + 1 / 32) / (ms_q * 1e-3) / 1e9,
                        "gemm_tflops": 2 * 2.0 * T * H * H / (ms_g * 1e-3) / 1e12, "gemm_ms": ms_g}
-    del xq, xs, wqq, wqs, wkq, wks
+    # backward of the same projections: operands re-quantized along the new contraction axis
+    dYq = workloads.gradients_rowscaled(T, H, cfg.data_seed + 2, dev)
+    ms_qt = timed(lambda: binding.fp4q_mxfp8_quantize1d_t(X))
+    dyq, dys = binding.fp4q_mxfp8_quantize1d(dYq)
+    wtq, wts = binding.fp4q_mxfp8_quantize1d_t(Wq)
+    dytq, dyts = binding.fp4q_mxfp8_quantize1d_t(dYq)
+    xtq, xts = binding.fp4q_mxfp8_quantize1d_t(X)
+    ms_dg = timed(lambda: binding.fp4q_mxfp8_gemm(dyq, dys, wtq, wts, T, H, H, ws=ws))
+    ms_wg = timed(lambda: binding.fp4q_mxfp8_gemm(dytq, dyts, xtq, xts, H, H, T, dt=binding.OUT_F32, ws=ws))
+    out["mxfp8_backward"] = {"workload": "dX = dY Wq and dWq = dY^T X of one projection, %d tokens, %dx%d" % (T, H, H),
+                             "transposing_quantize_gbs": T * H * (3.0 + 1 / 32) / (ms_qt * 1e-3) / 1e9,
+                             "dgrad_tflops": 2.0 * T * H * H / (ms_dg * 1e-3) / 1e12,
+                             "wgrad_tflops": 2.0 * T * H * H / (ms_wg * 1e-3) / 1e12}
+    del xq, xs, wqq, wqs, wkq, wks, dYq, dyq, dys, wtq, wts, dytq, dyts, xtq, xts
 
     # --- forward product with the output quantization fused into the epilogue, against product + separate quantize
     qx4, qw4 = binding.fp4q_quantize2d(X), binding.fp4q_quantize2d(Wq)

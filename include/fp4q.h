@@ -177,6 +177,32 @@ fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, i
                           void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * fp4q_mxfp8_quantize1d_t -- the same MXFP8 encoding of the TRANSPOSE of x[rows, cols]: payload q[cols, ld_q]
+ * (q[j, i] encodes x[i, j]; ld_q >= ceil32(rows), multiple of 16; q 16-byte aligned) with one UE8M0 scale per
+ * column j and 32 consecutive rows i, scale[cols, ld_s], ld_s >= ceil(rows/32).  The paper applies MXFP8 to the
+ * query/key projections (Section 3.2) and does not describe their backward pass; the reading taken here is that the
+ * backward products re-quantize their operands along the new contraction axis with the same rule, which is what
+ * this call produces without a separate transposition.  Payload bytes from rows to ceil32(rows) are written as 0.
+ */
+fp4q_status fp4q_mxfp8_quantize1d_t(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                    uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s,
+                                    void *stream);
+
+/*
+ * fp4q_mxfp8_gemm -- C[M,N] = A^ B^^T, FP32 accumulation, on two MXFP8 operands whose rows run along the
+ * contraction axis: aq [M, ld_aq] / as [M, ld_as], bq [N, ld_bq] / bs [N, ld_bs], contraction length Kdim
+ * (payload pitch >= ceil32(Kdim), scale pitch >= ceil(Kdim/32)).  C is BF16 or FP32 with leading dimension ldc.
+ * With the two quantizers above it gives the backward products of an MXFP8 projection Y = X W^T:
+ *   dX[T,K] = dY W      : A = quantize1d(dY)   [T, N],  B = quantize1d_t(W)  [K, N],  Kdim = N
+ *   dW[N,K] = dY^T X    : A = quantize1d_t(dY) [N, T],  B = quantize1d_t(X)  [K, T],  Kdim = T
+ * fp4q_mxfp8_qk is this call applied to the two forward projections.  ws/ws_bytes/stream as for fp4q_gemm_fwd.
+ */
+fp4q_status fp4q_mxfp8_gemm(const uint8_t *aq, int64_t ld_aq, const uint8_t *as, int64_t ld_as, int64_t M,
+                            const uint8_t *bq, int64_t ld_bq, const uint8_t *bs, int64_t ld_bs, int64_t N,
+                            int64_t Kdim, void *C, int64_t ldc, fp4q_out dt,
+                            void *ws, size_t ws_bytes, void *stream);
+
+/*
  * fp4q_gemm_fwd_quantized -- the dense forward product with the output quantization fused into the GEMM's epilogue
  * (Section 3.1 feeds each layer's BF16 output to the next layer's quantizer; here the tile is quantized while it is
  * still in registers):

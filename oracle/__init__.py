@@ -186,6 +186,13 @@ def mxfp8_quantize1d(x_bits):
     return q, s
 
 
+def mxfp8_quantize1d_t(x_bits):
+    """MXFP8 operand of the transpose (the backward products of an MXFP8 projection contract over the other axis;
+    Section 3.2 names the format only, the reading is: same rule, blocks along the new contraction axis)."""
+    x = _as_bf16_bits(x_bits)
+    return mxfp8_quantize1d(np.ascontiguousarray(x.T))
+
+
 def mxfp8_dequantize(q, scale):
     q = np.ascontiguousarray(q, dtype=np.uint8)
     s = np.ascontiguousarray(scale, dtype=np.uint8)

@@ -86,6 +86,12 @@ def lib() -> ctypes.CDLL:
             L.fp4q_gemm_fwd_static_workspace.restype = ci
             L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
                                                          ci, vp, vp]
+        if hasattr(L, "fp4q_mxfp8_gemm"):
+            L.fp4q_mxfp8_quantize1d_t.restype = ci
+            L.fp4q_mxfp8_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
+            L.fp4q_mxfp8_gemm.restype = ci
+            L.fp4q_mxfp8_gemm.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp, i64, i64, i64, vp, i64, ci, vp,
+                                          ctypes.c_size_t, vp]
         if hasattr(L, "fp4q_gemm_fwd_quantized"):
             L.fp4q_gemm_fwd_quantized.restype = ci
             L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
@@ -175,6 +181,36 @@ def fp4q_mxfp8_quantize1d(x: torch.Tensor, stream=None):
                                      scale.data_ptr(), scale.stride(0), _stream(stream))
     _check(st, "fp4q_mxfp8_quantize1d")
     return q, scale
+
+
+def fp4q_mxfp8_quantize1d_t(x: torch.Tensor, stream=None):
+    """MXFP8 encoding of x^T.  x: BF16 [rows, cols].  Returns (q uint8 [cols, ld_q], scale uint8 [cols, ceil(rows/32)])."""
+    _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+        raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
+    rows, cols = x.shape
+    ld_q = max((rows + 31) // 32 * 32, 32)
+    q = torch.empty((cols, ld_q), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((cols, max((rows + 31) // 32, 1)), dtype=torch.uint8, device=x.device)
+    st = lib().fp4q_mxfp8_quantize1d_t(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, q.data_ptr(), ld_q,
+                                       scale.data_ptr(), scale.stride(0), _stream(stream))
+    _check(st, "fp4q_mxfp8_quantize1d_t")
+    return q, scale
+
+
+def fp4q_mxfp8_gemm(aq, a_s, bq, b_s, M: int, N: int, Kdim: int, dt: int = OUT_BF16, ws=None, stream=None):
+    """C[M,N] = A^ B^^T on MXFP8 operands (rows along the contraction axis) from the two MXFP8 quantizers."""
+    dev = aq.device
+    per16 = 8 if dt == OUT_BF16 else 4
+    ldc = max((N + per16 - 1) // per16 * per16, per16)
+    out = torch.empty((M, ldc), dtype=_out_dtype(dt), device=dev)[:, :N]
+    if ws is None:
+        ws = alloc_workspace(dev)
+    st = lib().fp4q_mxfp8_gemm(aq.data_ptr(), aq.stride(0), a_s.data_ptr(), a_s.stride(0), M,
+                               bq.data_ptr(), bq.stride(0), b_s.data_ptr(), b_s.stride(0), N, Kdim,
+                               out.data_ptr(), ldc, dt, ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "fp4q_mxfp8_gemm")
+    return out
 
 
 def fp4q_workspace_bytes() -> int:

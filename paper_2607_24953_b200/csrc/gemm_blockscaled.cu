@@ -1612,6 +1612,30 @@ extern "C" fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uin
     return FP4Q_OK;
 }
 
+extern "C" fp4q_status fp4q_mxfp8_gemm(const uint8_t *aq, int64_t ld_aq, const uint8_t *as, int64_t ld_as, int64_t M,
+                                       const uint8_t *bq, int64_t ld_bq, const uint8_t *bs, int64_t ld_bs, int64_t N,
+                                       int64_t Kdim, void *C, int64_t ldc, fp4q_out dt, void *ws, size_t ws_bytes,
+                                       void *stream)
+{
+    if (M < 0 || N < 0 || Kdim < 0) return FP4Q_ERR_SHAPE;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (M > kMaxDim || N > kMaxDim || Kdim > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (M == 0 || N == 0) return FP4Q_OK;
+    if (!aq || !as || !bq || !bs || !C) return FP4Q_ERR_NULL;
+    const int64_t kpad = round_up(Kdim, 32), nkb = ceil_div(Kdim, 32);
+    if (ld_aq < kpad || ld_bq < kpad || ld_as < nkb || ld_bs < nkb || ldc < N) return FP4Q_ERR_SHAPE;
+    Operand A, B;
+    A.payload = aq; A.rows = M; A.row_bytes = kpad; A.ld_bytes = ld_aq;
+    A.sf = ScaleView{as, ld_as, 1, (int32_t)M, (int32_t)nkb};
+    B.payload = bq; B.rows = N; B.row_bytes = kpad; B.ld_bytes = ld_bq;
+    B.sf = ScaleView{bs, ld_bs, 1, (int32_t)N, (int32_t)nkb};
+    GemmParams p = {};
+    p.C = C; p.ldc = ldc; p.M = (int32_t)M; p.N = (int32_t)N; p.K = (int32_t)Kdim;
+    p.out_f32 = dt == FP4Q_OUT_F32;
+    dense_tiles(p);
+    return launch_gemm<KIND_MXF8>(A, B, p, ws, ws_bytes, stream);
+}
+
 // ------------------------------------------------------------------------------------------------------
 // Forward product for callers that cannot allocate device memory.
 //

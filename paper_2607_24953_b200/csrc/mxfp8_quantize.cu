@@ -92,6 +92,72 @@ __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_cons
     *reinterpret_cast<uint4 *>(p.q + i * p.ld_q + j0) = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
+// The transpose of the same operand: q_t[j, i] = E4M3 of x[i, j] with one scale per column j and 32 consecutive rows i
+// (the contraction axis of the backward products).  A warp owns 32 rows x 64 columns: each row is one coalesced
+// 128-byte load, a lane keeps its two columns' 32 values in registers, and writes 32 contiguous payload bytes per
+// column (one whole sector each).
+__global__ void __launch_bounds__(128) mxfp8_quantize1d_t_kernel(const __grid_constant__ Mxfp8QuantParams p)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t rb = (int64_t)blockIdx.y * 4 + warp;            // block of 32 rows
+    const int64_t i0 = rb * 32, c0 = (int64_t)blockIdx.x * 64 + 2 * lane;
+    if (i0 >= p.rows || c0 >= p.cols) return;
+    const bool two = c0 + 1 < p.cols;
+    uint32_t raw[32];
+#pragma unroll
+    for (int r = 0; r < 32; r++) {
+        raw[r] = 0u;
+        if (i0 + r < p.rows) {
+            const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
+            if (p.x_vec_ok && two) raw[r] = __ldg(reinterpret_cast<const uint32_t *>(src));
+            else raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+        }
+    }
+    uint32_t m0 = 0, m1 = 0;   // maxima over finite magnitudes
+#pragma unroll
+    for (int r = 0; r < 32; r++) {
+        const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
+        if (lo < 0x7F80u && lo > m0) m0 = lo;
+        if (hi < 0x7F80u && hi > m1) m1 = hi;
+    }
+    int code[2];
+    float inv[2];
+#pragma unroll
+    for (int k = 0; k < 2; k++) {
+        const uint32_t fm = k ? m1 : m0;
+        const int be = (int)(fm >> 7), m7 = (int)(fm & 0x7F);
+        int c = be == 0 ? 0 : be - 8 + (m7 > 0x60 ? 1 : 0);
+        code[k] = c < 0 ? 0 : c;
+        inv[k] = __uint_as_float((uint32_t)(254 - code[k]) << 23);
+    }
+    uint32_t A[8], B[8];   // the two columns' 32 payload bytes
+#pragma unroll
+    for (int w = 0; w < 8; w++) {
+        uint32_t res[4];
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            const uint32_t word = raw[4 * w + k];
+            const uint32_t lo = word << 16, hi = word & 0xFFFF0000u;
+            const float v0 = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv[0];
+            const float v1 = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv[1];
+            res[k] = cvt_rn_e4m3x2(v1, v0);   // byte 0: column c0, byte 1: column c0 + 1
+        }
+        const uint32_t t01 = res[0] | (res[1] << 16), t23 = res[2] | (res[3] << 16);
+        A[w] = __byte_perm(t01, t23, 0x6420);
+        B[w] = __byte_perm(t01, t23, 0x7531);
+    }
+    uint8_t *dst = p.q + c0 * p.ld_q + i0;
+    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(A[0], A[1], A[2], A[3]);
+    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(A[4], A[5], A[6], A[7]);
+    p.scale[c0 * p.ld_s + rb] = (uint8_t)code[0];
+    if (two) {
+        dst += p.ld_q;
+        reinterpret_cast<uint4 *>(dst)[0] = make_uint4(B[0], B[1], B[2], B[3]);
+        reinterpret_cast<uint4 *>(dst)[1] = make_uint4(B[4], B[5], B[6], B[7]);
+        p.scale[(c0 + 1) * p.ld_s + rb] = (uint8_t)code[1];
+    }
+}
+
 }  // namespace fp4q
 
 using namespace fp4q;
@@ -116,5 +182,27 @@ extern "C" fp4q_status fp4q_mxfp8_quantize1d(const void *x_bf16, int64_t rows, i
     const int64_t n_cta = ceil_div(total, 256);
     if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
     mxfp8_quantize1d_kernel<<<(unsigned)n_cta, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
+
+extern "C" fp4q_status fp4q_mxfp8_quantize1d_t(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                               uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s,
+                                               void *stream)
+{
+    if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return FP4Q_OK;
+    if (!x_bf16 || !q || !scale) return FP4Q_ERR_NULL;
+    if (ld_x < cols || ld_q < round_up(rows, 32) || ld_s < ceil_div(rows, 32)) return FP4Q_ERR_SHAPE;
+    if (!aligned(x_bf16, 2) || !aligned(q, 16) || ld_q % 16 != 0) return FP4Q_ERR_ALIGN;
+
+    Mxfp8QuantParams p;
+    p.x = static_cast<const uint16_t *>(x_bf16);
+    p.rows = rows; p.cols = cols; p.ld_x = ld_x;
+    p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
+    p.segs_per_row = 0;
+    p.x_vec_ok = aligned(x_bf16, 4) && ld_x % 2 == 0;
+    const int64_t gx = ceil_div(cols, 64), gy = ceil_div(ceil_div(rows, 32), 4);
+    if (gx > 0x7FFFFFFF || gy > 65535) return FP4Q_ERR_UNSUPPORTED;
+    mxfp8_quantize1d_t_kernel<<<dim3((unsigned)gx, (unsigned)gy), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
     return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }

@@ -126,3 +126,24 @@ def test_mxfp8_products_use_per_row_block_scales():
     x = oracle.mxfp8_dequantize(*oracle.mxfp8_quantize1d(_rand_bits(21, 6, 64)))
     w = oracle.mxfp8_dequantize(*oracle.mxfp8_quantize1d(_rand_bits(22, 10, 64)))
     assert np.allclose(oracle.gemm_fwd(x, w), oracle.gemm_nt_definition(x, w), rtol=1e-13, atol=0)
+
+
+def test_mxfp8_transposed_operand_is_the_operand_of_the_transpose():
+    """Blocks along the other axis: the transposing form must be the plain form applied to x^T, and decoding it
+    must give x^T back within the E4M3 rounding error (relative 2^-4 of the block maximum)."""
+    import numpy as np
+    from paper_2607_24953_b200 import workloads
+    import oracle
+    x = workloads.activations_student_t(70, 45, 5, "cpu")
+    bits = workloads.bf16_bits(x)
+    q, s = oracle.mxfp8_quantize1d_t(bits)
+    assert q.shape == (45, 70) and s.shape == (45, 3)
+    q2, s2 = oracle.mxfp8_quantize1d(np.ascontiguousarray(bits.T))
+    assert np.array_equal(q, q2) and np.array_equal(s, s2)
+    back = oracle.mxfp8_dequantize(q, s)
+    ref = x.double().numpy().T
+    for j in range(45):
+        for b in range(3):
+            seg = slice(32 * b, min(32 * b + 32, 70))
+            m = np.abs(ref[j, seg]).max()
+            assert np.abs(back[j, seg] - ref[j, seg]).max() <= m * 2.0 ** -4 + 1e-300
