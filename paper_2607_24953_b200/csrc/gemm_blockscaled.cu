@@ -78,12 +78,7 @@ constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
 constexpr uint32_t kWaitLimit = 1u << 22;
-#ifndef FP4Q_RELAXED_NS
-#define FP4Q_RELAXED_NS 64
-#endif
-#ifndef FP4Q_LAZY_NS
-#define FP4Q_LAZY_NS 256
-#endif
+constexpr int kRelaxedNs = 64, kLazyNs = 256;   // back-off between polls of roles with slack
 // Developer diagnostic (off by default): -DFP4Q_TRACE makes CTA 0 add up clock64() intervals of its roles in
 // registers and leave them in the workspace's padding words (status[16 + 2*slot], 64-bit each).
 #ifdef FP4Q_TRACE
@@ -216,12 +211,12 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile u
 __device__ __noinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
                                                uint32_t where)
 {
-    return mbar_wait_impl<FP4Q_RELAXED_NS>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kRelaxedNs>(bar, parity, abort_flag, status, where);
 }
 __device__ __noinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
                                             uint32_t where)
 {
-    return mbar_wait_impl<FP4Q_LAZY_NS>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kLazyNs>(bar, parity, abort_flag, status, where);
 }
 // For barriers that another CTA of the cluster completes (a multicast tcgen05.commit): probe instead of try_wait,
 // whose suspended thread is not reliably woken early by a remote arrival.
@@ -232,7 +227,7 @@ __device__ __noinline__ bool mbar_poll(uint32_t bar, uint32_t parity, volatile u
 __device__ __noinline__ bool mbar_poll_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
                                                uint32_t where)
 {
-    return mbar_wait_impl<FP4Q_RELAXED_NS, true>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kRelaxedNs, true>(bar, parity, abort_flag, status, where);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
@@ -885,7 +880,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
                 if (issuer) {
-#ifndef FP4Q_SKIP_MMA   // development only: leave the tensor pipe idle to time the load path alone
                     const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
                     if (KIND == KIND_MXF4) {
                         const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
@@ -915,7 +909,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                                                                  sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
                         }
                     }
-#endif
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
                     if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
                     if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
@@ -1131,9 +1124,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
                     for (int q = 0; q < 32; q++) v[j][q] = 0u;
             }
-#ifdef FP4Q_SKIP_STORE   // development only: results are dropped
-            if (row_ok && p.M < 0) {
-#else
             if (EPI == EPI_QUANT) {
                 // The output tile leaves as 2D-block FP4: each warp owns four 32x32 blocks (its 32 rows x 32 columns
                 // per chunk).  The accumulator is rounded to BF16 first, so the result equals fp4q_quantize2d applied
@@ -1242,7 +1232,6 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     }
                 }
             } else if (row_ok) {
-#endif
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const int col_in_tile = 128 * half + 32 * j;
@@ -1364,11 +1353,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
         if (!make_byte_map(&tmC, p.q_rm, p.M, round_up(p.N, 32) / 2, p.q_ld_rm, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return FP4Q_ERR_CUDA;
         if (p.q_t && !make_byte_map(&tmD, p.q_t, p.N, round_up(p.M, 32) / 2, p.q_ld_t, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) return FP4Q_ERR_CUDA;
     } else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
-#ifdef FP4Q_SPLIT_B
-    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, 128)) return FP4Q_ERR_CUDA;
-#else
     if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<CTAS>::kBRows)) return FP4Q_ERR_CUDA;
-#endif
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
