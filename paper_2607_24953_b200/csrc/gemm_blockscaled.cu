@@ -316,6 +316,11 @@ __device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64
                      " tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
                      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
                      : "memory");
+    } else if (CTAS == 2) {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
     } else {
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                      " tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%5], [%6], p;\n}"
@@ -1402,12 +1407,12 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     p.sfa = A.sf;
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
-    // Dense FP4 products with more than one row tile run as cta_group::2 pairs: 256x256 tiles, each CTA loads half of
-    // the B rows, which leaves room for a six-stage ring.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the
+    // Dense products (FP4 and MXFP8) with more than one row tile run as cta_group::2 pairs: 256x256 tiles, each CTA
+    // loads half of the B rows.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the
     // first GEMM call) selects the one-CTA kernel instead; grouped products (token groups are only 128-row aligned)
-    // and the MXFP8 path always use one CTA per 128x256 tile.
+    // always use one CTA per 128x256 tile.
     static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return !(e && e[0] == '0'); }();
-    if (use_pairs && KIND == KIND_MXF4 && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND_MXF4, 2>(A, B, p, stream);
+    if (use_pairs && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND, 2>(A, B, p, stream);
     return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
 
