@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
                                             i64, i64, i64, i64, u8p, i64, u8p, i64, u8p, i64]
         L.orc_dequantize2d.restype = None
         L.orc_dequantize2d.argtypes = [u8p, i64, u8p, i64, i64, i64, u8p, i64]
+        L.orc_quantize1d.restype = ctypes.c_int
+        L.orc_quantize1d.argtypes = [u8p, i64, i64, i64, ctypes.c_int, u64, u32, u32, u8p, i64, u8p, i64]
+        L.orc_dequantize1d.restype = None
+        L.orc_dequantize1d.argtypes = [u8p, i64, u8p, i64, i64, i64, u8p, i64]
         L.orc_mxfp8_quantize1d.restype = ctypes.c_int
         L.orc_mxfp8_quantize1d.argtypes = [u8p, i64, i64, i64, u8p, i64, u8p, i64]
         L.orc_mxfp8_dequantize.restype = None
@@ -95,6 +99,12 @@ def _as_bf16_bits(x) -> np.ndarray:
     if a.dtype != np.uint16 or a.ndim != 2:
         raise TypeError("expected a 2-D uint16 array of BF16 bit patterns")
     return a
+
+
+def bits_to_double(x_bits) -> np.ndarray:
+    """BF16 bit patterns -> float64 values (exact)."""
+    x = _as_bf16_bits(x_bits)
+    return (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
 def e2m1_value(code: int) -> float:
@@ -171,6 +181,62 @@ def dequantize2d(q_rm, scale, rows, cols):
     if rows and cols:
         lib().orc_dequantize2d(_ptr(q), q.shape[1], _ptr(s), s.shape[1], rows, cols, _ptr(out), cols)
     return out
+
+
+def quantize1d(x_bits, mode=MODE_NEAREST, seed=0, tensor_id=0, flags=0):
+    """1D-block (1 x 32) FP4 quantization along the rows of a BF16 matrix (the paper's activation layout).
+    Returns (q [rows, ceil(cols/2)], scale [rows, ceil(cols/32)]) as uint8."""
+    x = _as_bf16_bits(x_bits)
+    rows, cols = x.shape
+    q = np.zeros((rows, (cols + 1) // 2), dtype=np.uint8)
+    s = np.zeros((rows, -(-cols // BLOCK)), dtype=np.uint8)
+    if rows and cols:
+        rc = lib().orc_quantize1d(_ptr(x), rows, cols, cols, int(mode), seed, tensor_id, flags,
+                                  _ptr(q), q.shape[1], _ptr(s), s.shape[1])
+        if rc != 0:
+            raise ValueError("orc_quantize1d rejected its arguments")
+    return q, s
+
+
+def quantize1d_t(x_bits, mode=MODE_NEAREST, seed=0, tensor_id=0):
+    """The same encoding of the transpose (blocks along the rows of x, i.e. along the token axis when x is an
+    activation [tokens, channels]); the rounding stream stays keyed on the element's index in x."""
+    x = _as_bf16_bits(x_bits)
+    return quantize1d(np.ascontiguousarray(x.T), mode, seed, tensor_id, FLAG_INDEX_TRANSPOSED)
+
+
+def dequantize1d(q, scale, rows, cols):
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    s = np.ascontiguousarray(scale, dtype=np.uint8)
+    out = np.zeros((rows, cols), dtype=np.float64)
+    if rows and cols:
+        lib().orc_dequantize1d(_ptr(q), q.shape[1], _ptr(s), s.shape[1], rows, cols, _ptr(out), cols)
+    return out
+
+
+def transposition_diagnostic(x_bits):
+    """Figure 1 (c), (d) of the paper on one tensor, nearest rounding: per element the difference of the scale
+    exponents the element gets when the tensor is quantized as stored and when its transpose is quantized, and
+    the relative Frobenius deviation between the two dequantized tensors - for 1D blocks and for 2D blocks.
+    Returns a dict with the two exponent-difference maps and the two deviations."""
+    x = _as_bf16_bits(x_bits)
+    rows, cols = x.shape
+    ref = bits_to_double(x)
+    q1, s1 = quantize1d(x)
+    q1t, s1t = quantize1d(np.ascontiguousarray(x.T))
+    e_fwd = np.repeat(s1.astype(np.int32), BLOCK, axis=1)[:, :cols]
+    e_bwd = np.repeat(s1t.astype(np.int32), BLOCK, axis=1)[:, :rows].T
+    d1 = dequantize1d(q1, s1, rows, cols)
+    d1t = dequantize1d(q1t, s1t, cols, rows).T
+    q2, _, s2 = quantize2d(x, want_t=False)
+    q2t, _, s2t = quantize2d(np.ascontiguousarray(x.T), want_t=False)
+    f_fwd = np.repeat(np.repeat(s2.astype(np.int32), BLOCK, axis=0), BLOCK, axis=1)[:rows, :cols]
+    f_bwd = np.repeat(np.repeat(s2t.astype(np.int32), BLOCK, axis=0), BLOCK, axis=1)[:cols, :rows].T
+    d2 = dequantize2d(q2, s2, rows, cols)
+    d2t = dequantize2d(q2t, s2t, cols, rows).T
+    nrm = np.linalg.norm(ref)
+    return {"scale_exponent_difference_1d": e_fwd - e_bwd, "scale_exponent_difference_2d": f_fwd - f_bwd,
+            "deviation_1d": np.linalg.norm(d1 - d1t) / nrm, "deviation_2d": np.linalg.norm(d2 - d2t) / nrm}
 
 
 def mxfp8_quantize1d(x_bits):

@@ -298,6 +298,78 @@ void orc_dequantize2d(const uint8_t *q_rm, int64_t ld_rm, const uint8_t *scale, 
     }
 }
 
+/* ------------------------------------------------------- 1D (1 x 32) FP4 blocks */
+
+/*
+ * The activation layout the paper keeps (Section 3.1, "We retain a 1D layout for activations"; appendix
+ * "Quantization Placement", paragraph Activations): one scale per 32 consecutive elements of a row, everything
+ * else as in the 2D scheme - truncation-free power-of-two scale, E2M1 codes, nearest-even or stochastic rounding
+ * with the random byte of the element's row-major index i*cols + j (j*rows + i with the transposed-index flag).
+ * q[rows, ld_q] packed two codes per byte (low nibble = even column), scale[rows, ld_s], ld_s >= ceil(cols/32).
+ * +-Inf -> +-6, NaN -> +0, block maximum over finite entries.  Payload bytes up to ld_q are written as 0.
+ */
+int orc_quantize1d(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld_x, int mode, uint64_t seed,
+                   uint32_t tensor_id, uint32_t flags, uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s)
+{
+    int64_t nb = (cols + ORC_BLOCK - 1) / ORC_BLOCK, i;
+    if (rows < 0 || cols < 0 || (mode != ORC_MODE_NEAREST && mode != ORC_MODE_STOCHASTIC)) return -1;
+    if (rows == 0 || cols == 0) return 0;
+    if (!x || !q || !scale || ld_x < cols || ld_q < (cols + 1) / 2 || ld_s < nb) return -1;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < rows; i++) {
+        int64_t b;
+        memset(q + i * ld_q, 0, (size_t)ld_q);
+        for (b = 0; b < nb; b++) {
+            int64_t j0 = b * ORC_BLOCK, j1 = j0 + ORC_BLOCK < cols ? j0 + ORC_BLOCK : cols, j;
+            double M = 0.0, S;
+            int e;
+            for (j = j0; j < j1; j++) {
+                double a = fabs(orc_bf16_to_double(x[i * ld_x + j]));
+                if (isfinite(a) && a > M) M = a;
+            }
+            e = orc_scale_exponent(M);
+            S = ldexp(1.0, e);
+            scale[i * ld_s + b] = (uint8_t)(e + 127);
+            for (j = j0; j < j1; j++) {
+                uint16_t bits = x[i * ld_x + j];
+                double a = orc_bf16_to_double(bits);
+                int sign = (bits >> 15) & 1, mag, code;
+                if (isnan(a)) {
+                    code = 0;
+                } else {
+                    if (isinf(a)) {
+                        mag = 7;
+                    } else if (mode == ORC_MODE_NEAREST) {
+                        mag = orc_round_nearest(fabs(a) / S);
+                    } else {
+                        uint64_t idx = (flags & ORC_FLAG_INDEX_TRANSPOSED) ? (uint64_t)j * (uint64_t)rows + (uint64_t)i
+                                                                           : (uint64_t)i * (uint64_t)cols + (uint64_t)j;
+                        mag = orc_round_stochastic(fabs(a) / S, orc_random_byte(seed, tensor_id, idx));
+                    }
+                    code = (sign << 3) | mag;
+                }
+                orc_put_nibble(q + i * ld_q, j, code);
+            }
+        }
+    }
+    return 0;
+}
+
+/* Dequantized values of a 1D-block tensor, exact in double. */
+void orc_dequantize1d(const uint8_t *q, int64_t ld_q, const uint8_t *scale, int64_t ld_s, int64_t rows, int64_t cols,
+                      double *out, int64_t ld_out)
+{
+    int64_t i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < rows; i++) {
+        int64_t j;
+        for (j = 0; j < cols; j++) {
+            int e = (int)scale[i * ld_s + j / ORC_BLOCK] - 127;
+            out[i * ld_out + j] = ldexp(orc_e2m1_value(orc_get_nibble(q + i * ld_q, j)), e);
+        }
+    }
+}
+
 /* -------------------------------------------------------------------- MXFP8 */
 
 /* Nearest E4M3 magnitude code (0x00..0x7E) for v in [0, 448], ties to the even
