@@ -177,6 +177,29 @@ fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, i
                           void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * fp4q_quantize1d -- 1D-block FP4 quantization, the layout the paper keeps for activations (Section 3.1, "We retain a
+ * 1D layout for activations"; appendix "Quantization Placement"): one UE8M0 scale per 32 consecutive elements of a
+ * row of x[rows, cols], otherwise the arithmetic of fp4q_quantize2d (truncation-free scale with bound 6, E2M1 codes,
+ * nearest-even or stochastic rounding with the random byte of element index i*cols + j, non-finite inputs as there).
+ * q [rows, ld_q] packed two codes per byte (low nibble = even column; ld_q >= ceil32(cols)/2, multiple of 16, q
+ * 16-byte aligned; bytes up to ceil32(cols)/2 are written, padding codes are 0), scale [rows, ld_s],
+ * ld_s >= ceil(cols/32).  Stochastic rounding needs cols % 16 == 0 (FP4Q_ERR_UNSUPPORTED otherwise).
+ */
+fp4q_status fp4q_quantize1d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                            uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s,
+                            fp4q_round mode, uint64_t seed, uint32_t tensor_id, void *stream);
+
+/*
+ * fp4q_quantize1d_t -- the same encoding of the TRANSPOSE: q [cols, ld_q] (q[j, i/2] nibble i&1 encodes x[i, j];
+ * ld_q >= ceil32(rows)/2), scale [cols, ld_s] with one scale per column j and 32 consecutive rows i,
+ * ld_s >= ceil(rows/32).  Nearest-even rounding (activations are quantized in the forward pass).  This is the operand
+ * of the weight-gradient product, which contracts over the rows of x; with 1D blocks it is a second quantization of x
+ * whose scales differ from those of fp4q_quantize1d - the inconsistency Figure 1 of the paper illustrates.
+ */
+fp4q_status fp4q_quantize1d_t(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                              uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s, void *stream);
+
+/*
  * fp4q_mxfp8_quantize1d_t -- the same MXFP8 encoding of the TRANSPOSE of x[rows, cols]: payload q[cols, ld_q]
  * (q[j, i] encodes x[i, j]; ld_q >= ceil32(rows), multiple of 16; q 16-byte aligned) with one UE8M0 scale per
  * column j and 32 consecutive rows i, scale[cols, ld_s], ld_s >= ceil(rows/32).  The paper applies MXFP8 to the

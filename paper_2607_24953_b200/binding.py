@@ -86,6 +86,11 @@ def lib() -> ctypes.CDLL:
             L.fp4q_gemm_fwd_static_workspace.restype = ci
             L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
                                                          ci, vp, vp]
+        if hasattr(L, "fp4q_quantize1d"):
+            L.fp4q_quantize1d.restype = ci
+            L.fp4q_quantize1d.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, ci, u64, u32, vp]
+            L.fp4q_quantize1d_t.restype = ci
+            L.fp4q_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
         if hasattr(L, "fp4q_mxfp8_gemm"):
             L.fp4q_mxfp8_quantize1d_t.restype = ci
             L.fp4q_mxfp8_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
@@ -180,6 +185,36 @@ def fp4q_mxfp8_quantize1d(x: torch.Tensor, stream=None):
     st = lib().fp4q_mxfp8_quantize1d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, q.data_ptr(), ld_q,
                                      scale.data_ptr(), scale.stride(0), _stream(stream))
     _check(st, "fp4q_mxfp8_quantize1d")
+    return q, scale
+
+
+def fp4q_quantize1d(x: torch.Tensor, mode: int = ROUND_NEAREST, seed: int = 0, tensor_id: int = 0, stream=None):
+    """1D-block FP4 of x (blocks along its rows).  Returns (q uint8 [rows, ld_q], scale uint8 [rows, ceil(cols/32)])."""
+    _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+        raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
+    rows, cols = x.shape
+    ld_q = max(_pad16((cols + 31) // 32 * 16), 16)
+    q = torch.empty((rows, ld_q), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((rows, max((cols + 31) // 32, 1)), dtype=torch.uint8, device=x.device)
+    st = lib().fp4q_quantize1d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, q.data_ptr(), ld_q,
+                               scale.data_ptr(), scale.stride(0), mode, seed, tensor_id, _stream(stream))
+    _check(st, "fp4q_quantize1d")
+    return q, scale
+
+
+def fp4q_quantize1d_t(x: torch.Tensor, stream=None):
+    """1D-block FP4 of x^T (blocks along the rows of x), nearest rounding.  Returns (q [cols, ld_q], scale [cols, ceil(rows/32)])."""
+    _dev(x, "x")
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+        raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
+    rows, cols = x.shape
+    ld_q = max(_pad16((rows + 31) // 32 * 16), 16)
+    q = torch.empty((cols, ld_q), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((cols, max((rows + 31) // 32, 1)), dtype=torch.uint8, device=x.device)
+    st = lib().fp4q_quantize1d_t(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, q.data_ptr(), ld_q,
+                                 scale.data_ptr(), scale.stride(0), _stream(stream))
+    _check(st, "fp4q_quantize1d_t")
     return q, scale
 
 

@@ -1,0 +1,189 @@
+// fp4q_quantize1d / fp4q_quantize1d_t: 1D-block (1 x 32) FP4 quantization, the layout the paper keeps for
+// activations (Section 3.1), in both orientations the layer's products need:
+//   fp4q_quantize1d    blocks along the rows of x (the channel axis of an activation [tokens, channels]):
+//                      the A operand of the forward product;
+//   fp4q_quantize1d_t  the encoding of x^T with blocks along the rows of x (the token axis): the B operand of the
+//                      weight-gradient product, which contracts over tokens.
+// Same arithmetic as the 2D quantizer (shared device functions): truncation-free power-of-two scale from the block
+// maximum, E2M1 codes through the hardware converts, nearest-even or (row-wise form only) stochastic rounding
+// keyed on the element's index i*cols + j.  Streaming kernels: one coalesced pass over x.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "quant_device.cuh"
+
+namespace fp4q {
+
+struct Quant1dParams {
+    const uint16_t *x;
+    int64_t rows, cols, ld_x;
+    uint8_t *q;
+    int64_t ld_q;
+    uint8_t *scale;
+    int64_t ld_s;
+    int64_t segs_per_row;   // 16-element segments per row, even
+    int x_vec_ok;
+    uint32_t tensor_id;
+    PhiloxRoundKeys keys;
+};
+
+// Each thread owns 16 consecutive elements of a row (two 128-bit loads, one 64-bit store); two neighbouring lanes
+// own one 32-element block and exchange their maxima with one shuffle.
+template <int MODE>
+__global__ void __launch_bounds__(256) quantize1d_kernel(const __grid_constant__ Quant1dParams p)
+{
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t total = p.rows * p.segs_per_row;
+    const bool active = gid < total;   // whole warps stay in the shuffle below (total is even, lanes pair up)
+    const int64_t i = active ? gid / p.segs_per_row : 0;
+    const int64_t seg = active ? gid % p.segs_per_row : 0;
+    const int64_t j0 = seg * 16;
+
+    uint32_t raw[8];
+#pragma unroll
+    for (int k = 0; k < 8; k++) raw[k] = 0u;
+    if (active && j0 < p.cols) {
+        const uint16_t *src = p.x + i * p.ld_x + j0;
+        if (p.x_vec_ok && j0 + 16 <= p.cols) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
+            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
+            raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
+            raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
+                const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
+                raw[k] = lo | (hi << 16);
+            }
+        }
+    }
+    uint32_t fm = 0;
+    bool nonfinite = false;
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
+        nonfinite |= lo >= 0x7F80u || hi >= 0x7F80u;
+        if (lo < 0x7F80u && lo > fm) fm = lo;
+        if (hi < 0x7F80u && hi > fm) fm = hi;
+    }
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, 1);
+    fm = other > fm ? other : fm;
+    nonfinite |= __shfl_xor_sync(0xFFFFFFFFu, (int)nonfinite, 1) != 0;
+    const int code = scale_code_from_max(fm);
+    if (!active) return;
+    if ((seg & 1) == 0) p.scale[i * p.ld_s + (seg >> 1)] = (uint8_t)code;
+
+    uint32_t R[4] = {0u, 0u, 0u, 0u};
+    if (MODE == FP4Q_ROUND_STOCHASTIC) {   // cols % 16 == 0: the segment is one Philox block
+        const uint64_t blk = (uint64_t)(i * p.cols + j0) >> 4;
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, R);
+    }
+    uint32_t W[2];
+    if (!nonfinite) {
+        round_segment<MODE>(raw, inv_scale(code), R, W);
+    } else {
+        const uint2 w = round_segment_scalar<MODE>(make_uint4(raw[0], raw[1], raw[2], raw[3]), make_uint4(raw[4], raw[5], raw[6], raw[7]),
+                                                   make_uint4(R[0], R[1], R[2], R[3]), inv_scale_f16_aligned(code));
+        W[0] = w.x;
+        W[1] = w.y;
+    }
+    *reinterpret_cast<uint2 *>(p.q + i * p.ld_q + (j0 >> 1)) = make_uint2(W[0], W[1]);
+}
+
+// The encoding of x^T, nearest rounding.  A warp owns 32 rows x 64 columns: each row is one coalesced 128-byte load,
+// a lane keeps its two columns' 32 values in registers, and writes the 16 payload bytes of each column's block.
+__global__ void __launch_bounds__(128) quantize1d_t_kernel(const __grid_constant__ Quant1dParams p)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t rb = (int64_t)blockIdx.y * 4 + warp;   // block of 32 rows
+    const int64_t i0 = rb * 32, c0 = (int64_t)blockIdx.x * 64 + 2 * lane;
+    if (i0 >= p.rows || c0 >= p.cols) return;
+    const bool two = c0 + 1 < p.cols;
+    uint32_t raw[32];
+#pragma unroll
+    for (int r = 0; r < 32; r++) {
+        raw[r] = 0u;
+        if (i0 + r < p.rows) {
+            const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
+            if (p.x_vec_ok && two) raw[r] = __ldg(reinterpret_cast<const uint32_t *>(src));
+            else raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+        }
+    }
+    uint32_t m0 = 0, m1 = 0;
+#pragma unroll
+    for (int r = 0; r < 32; r++) {
+        const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
+        if (lo < 0x7F80u && lo > m0) m0 = lo;
+        if (hi < 0x7F80u && hi > m1) m1 = hi;
+    }
+    const int code0 = scale_code_from_max(m0), code1 = scale_code_from_max(m1);
+    const float inv0 = inv_scale(code0), inv1 = inv_scale(code1);
+    uint32_t A[4] = {0u, 0u, 0u, 0u}, B[4] = {0u, 0u, 0u, 0u};   // the two columns' 32 nibbles
+#pragma unroll
+    for (int r = 0; r < 32; r++) {
+        const uint32_t lo = raw[r] << 16, hi = raw[r] & 0xFFFF0000u;
+        // NaN -> +0; +-Inf saturates to +-6 in the conversion
+        const float v0 = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv0;
+        const float v1 = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv1;
+        const uint32_t res = cvt_rn_e2m1x2(v1, v0);   // nibble 0: column c0, nibble 1: column c0 + 1
+        A[r >> 3] |= (res & 0xFu) << (4 * (r & 7));
+        B[r >> 3] |= ((res >> 4) & 0xFu) << (4 * (r & 7));
+    }
+    *reinterpret_cast<uint4 *>(p.q + c0 * p.ld_q + (i0 >> 1)) = make_uint4(A[0], A[1], A[2], A[3]);
+    p.scale[c0 * p.ld_s + rb] = (uint8_t)code0;
+    if (two) {
+        *reinterpret_cast<uint4 *>(p.q + (c0 + 1) * p.ld_q + (i0 >> 1)) = make_uint4(B[0], B[1], B[2], B[3]);
+        p.scale[(c0 + 1) * p.ld_s + rb] = (uint8_t)code1;
+    }
+}
+
+}  // namespace fp4q
+
+using namespace fp4q;
+
+extern "C" fp4q_status fp4q_quantize1d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x, uint8_t *q, int64_t ld_q,
+                                       uint8_t *scale, int64_t ld_s, fp4q_round mode, uint64_t seed, uint32_t tensor_id,
+                                       void *stream)
+{
+    if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
+    if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
+    if (mode == FP4Q_ROUND_STOCHASTIC && cols % 16 != 0) return FP4Q_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return FP4Q_OK;
+    if (!x_bf16 || !q || !scale) return FP4Q_ERR_NULL;
+    if (ld_x < cols || ld_q < round_up(cols, 32) / 2 || ld_s < ceil_div(cols, 32)) return FP4Q_ERR_SHAPE;
+    if (!aligned(x_bf16, 2) || !aligned(q, 16) || ld_q % 16 != 0) return FP4Q_ERR_ALIGN;
+    Quant1dParams p;
+    p.x = static_cast<const uint16_t *>(x_bf16);
+    p.rows = rows; p.cols = cols; p.ld_x = ld_x;
+    p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
+    p.segs_per_row = round_up(cols, 32) / 16;
+    p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
+    p.tensor_id = tensor_id;
+    philox_round_keys(seed, p.keys);
+    const int64_t n_cta = ceil_div(rows * p.segs_per_row, 256);
+    if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (mode == FP4Q_ROUND_STOCHASTIC) quantize1d_kernel<FP4Q_ROUND_STOCHASTIC><<<(unsigned)n_cta, 256, 0, s>>>(p);
+    else quantize1d_kernel<FP4Q_ROUND_NEAREST><<<(unsigned)n_cta, 256, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
+
+extern "C" fp4q_status fp4q_quantize1d_t(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x, uint8_t *q, int64_t ld_q,
+                                         uint8_t *scale, int64_t ld_s, void *stream)
+{
+    if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return FP4Q_OK;
+    if (!x_bf16 || !q || !scale) return FP4Q_ERR_NULL;
+    if (ld_x < cols || ld_q < round_up(rows, 32) / 2 || ld_s < ceil_div(rows, 32)) return FP4Q_ERR_SHAPE;
+    if (!aligned(x_bf16, 2) || !aligned(q, 16) || ld_q % 16 != 0) return FP4Q_ERR_ALIGN;
+    Quant1dParams p = {};
+    p.x = static_cast<const uint16_t *>(x_bf16);
+    p.rows = rows; p.cols = cols; p.ld_x = ld_x;
+    p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
+    p.x_vec_ok = aligned(x_bf16, 4) && ld_x % 2 == 0;
+    const int64_t gx = ceil_div(cols, 64), gy = ceil_div(ceil_div(rows, 32), 4);
+    if (gx > 0x7FFFFFFF || gy > 65535) return FP4Q_ERR_UNSUPPORTED;
+    quantize1d_t_kernel<<<dim3((unsigned)gx, (unsigned)gy), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
