@@ -200,6 +200,27 @@ fp4q_status fp4q_quantize1d_t(const void *x_bf16, int64_t rows, int64_t cols, in
                               uint8_t *q, int64_t ld_q, uint8_t *scale, int64_t ld_s, void *stream);
 
 /*
+ * fp4q_gemm_fwd_act1d -- the forward product with the paper's mixed layout (Section 3.1: 2D blocks for weights, 1D
+ * blocks for activations): Y[T, N] = X^ W^T, X given by its 1D-block encoding along the contraction axis as written
+ * by fp4q_quantize1d (xq [T, ld_xq] packed payload, xs [T, ld_xs] per-row scales; K = W->cols), W a 2D-block tensor
+ * (row-major payload used).  Dense only.  Output, workspace, alignment and error behaviour as fp4q_gemm_fwd.
+ */
+fp4q_status fp4q_gemm_fwd_act1d(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, int64_t ld_xs, int64_t T,
+                                const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt,
+                                void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * fp4q_gemm_wgrad_act1d -- the weight-gradient product with a 1D-block activation: dW[N, K] (+)= dY^^T X^_t, dY a
+ * 2D-block tensor (transposed payload used; T = dY->rows, N = dY->cols), X given by the 1D-block encoding of its
+ * transpose as written by fp4q_quantize1d_t (xtq [K, ld_xtq], xts [K, ld_xts], blocks along the token axis).  This is
+ * the product in which 1D blocks force the activation to be quantized a second time with different scales
+ * (Figure 1 of the paper).  Dense only.  Output, accumulate, workspace and errors as fp4q_gemm_wgrad.
+ */
+fp4q_status fp4q_gemm_wgrad_act1d(const fp4q_tensor *dY, const uint8_t *xtq, int64_t ld_xtq, const uint8_t *xts,
+                                  int64_t ld_xts, int64_t K, void *dW, int64_t ldw, fp4q_out dt, int accumulate,
+                                  void *ws, size_t ws_bytes, void *stream);
+
+/*
  * fp4q_mxfp8_quantize1d_t -- the same MXFP8 encoding of the TRANSPOSE of x[rows, cols]: payload q[cols, ld_q]
  * (q[j, i] encodes x[i, j]; ld_q >= ceil32(rows), multiple of 16; q 16-byte aligned) with one UE8M0 scale per
  * column j and 32 consecutive rows i, scale[cols, ld_s], ld_s >= ceil(rows/32).  The paper applies MXFP8 to the

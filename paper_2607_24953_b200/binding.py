@@ -91,6 +91,11 @@ def lib() -> ctypes.CDLL:
             L.fp4q_quantize1d.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, ci, u64, u32, vp]
             L.fp4q_quantize1d_t.restype = ci
             L.fp4q_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
+        if hasattr(L, "fp4q_gemm_fwd_act1d"):
+            L.fp4q_gemm_fwd_act1d.restype = ci
+            L.fp4q_gemm_fwd_act1d.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, ci, vp, ctypes.c_size_t, vp]
+            L.fp4q_gemm_wgrad_act1d.restype = ci
+            L.fp4q_gemm_wgrad_act1d.argtypes = [vp, vp, i64, vp, i64, i64, vp, i64, ci, ci, vp, ctypes.c_size_t, vp]
         if hasattr(L, "fp4q_mxfp8_gemm"):
             L.fp4q_mxfp8_quantize1d_t.restype = ci
             L.fp4q_mxfp8_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
@@ -245,6 +250,44 @@ def fp4q_mxfp8_gemm(aq, a_s, bq, b_s, M: int, N: int, Kdim: int, dt: int = OUT_B
                                bq.data_ptr(), bq.stride(0), b_s.data_ptr(), b_s.stride(0), N, Kdim,
                                out.data_ptr(), ldc, dt, ws.data_ptr(), ws.numel(), _stream(stream))
     _check(st, "fp4q_mxfp8_gemm")
+    return out
+
+
+def _out_buffer(rows: int, cols: int, dt: int, device):
+    per16 = 8 if dt == OUT_BF16 else 4
+    ld = max((cols + per16 - 1) // per16 * per16, per16)
+    return torch.empty((rows, ld), dtype=_out_dtype(dt), device=device)[:, :cols]
+
+
+def fp4q_gemm_fwd_act1d(xq, xs, T: int, W: QTensor, out=None, dt: int = OUT_BF16, ws=None, stream=None):
+    """Y[T,N] = X^ W^^T with X in 1D blocks along the contraction axis (fp4q_quantize1d) and W in 2D blocks."""
+    dev = xq.device
+    if out is None:
+        out = _out_buffer(T, W.rows, dt, dev)
+    if ws is None:
+        ws = alloc_workspace(dev)
+    cw = W.c_struct()
+    st = lib().fp4q_gemm_fwd_act1d(xq.data_ptr(), xq.stride(0), xs.data_ptr(), xs.stride(0), T, ctypes.byref(cw),
+                                   out.data_ptr(), out.stride(0), dt, ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "fp4q_gemm_fwd_act1d")
+    return out
+
+
+def fp4q_gemm_wgrad_act1d(dY: QTensor, xtq, xts, K: int, out=None, dt: int = OUT_F32, accumulate: bool = False,
+                          ws=None, stream=None):
+    """dW[N,K] (+)= dY^^T X^_t with X^_t the 1D-block encoding of X^T (fp4q_quantize1d_t) and dY in 2D blocks."""
+    dev = xtq.device
+    if out is None:
+        out = _out_buffer(dY.cols, K, dt, dev)
+        if accumulate:
+            out.zero_()
+    if ws is None:
+        ws = alloc_workspace(dev)
+    cd = dY.c_struct()
+    st = lib().fp4q_gemm_wgrad_act1d(ctypes.byref(cd), xtq.data_ptr(), xtq.stride(0), xts.data_ptr(), xts.stride(0), K,
+                                     out.data_ptr(), out.stride(0), dt, 1 if accumulate else 0, ws.data_ptr(),
+                                     ws.numel(), _stream(stream))
+    _check(st, "fp4q_gemm_wgrad_act1d")
     return out
 
 

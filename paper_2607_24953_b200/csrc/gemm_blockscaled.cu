@@ -54,6 +54,10 @@ constexpr int kCompactBytes = kCacheChunks * 48;
 constexpr int kImageStageBytes = 768;        // A chunk 0, A chunk 1, B chunk 0 (rows 0..127, 128..255), B chunk 1 (same)
 constexpr int kCacheBufBytes = kUnitStagesMxf4 * kImageStageBytes;
 static_assert(kUnitStagesMxf8 * kImageStageBytesMxf8 == kCacheBufBytes, "both kinds share the image buffers");
+// mxf4 with per-row scales: a stage has two chunks of four blocks; A 2 x 512 B, B (256 rows) 4 x 512 B per stage
+constexpr int kUnitStagesMxf4R = 4;
+constexpr int kImageStageBytesMxf4R = 3072;
+static_assert(kUnitStagesMxf4R * kImageStageBytesMxf4R == kCacheBufBytes, "all kinds share the image buffers");
 constexpr int kSmemCache = kCompactBytes + 2 * kCacheBufBytes;
 // Epilogue staging of the pair kernel: each of the 8 epilogue warps owns 32 rows x 128 bytes, written from registers
 // (128-byte swizzle: the 16-byte pieces of 8 rows fall into different banks) and drained by a TMA store, which keeps
@@ -103,7 +107,11 @@ extern "C" int fp4q_debug_events(void *host) { return (int)cudaMemcpyFromSymbol(
 #endif
 constexpr uint8_t kScalePad = 127;           // UE8M0 code of 1.0 for scale slots beyond the tensor (their payload is 0)
 
-enum { KIND_MXF4 = 0, KIND_MXF8 = 1 };
+// KIND_MXF4: FP4 payloads, 2D-block scales on both operands (replicated scale images).  KIND_MXF8: E4M3 payloads,
+// per-row scales.  KIND_MXF4R: FP4 payloads with per-row scale images - an operand quantized in 1D blocks (the
+// paper's activation layout) next to a 2D-block operand, whose tile scale is then expanded to its 32 rows.
+enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2 };
+__host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8; }
 enum { MODE_DENSE = 0, MODE_GROUPED_ROWS = 1, MODE_GROUPED_K = 2 };
 
 struct ScaleView {
@@ -112,6 +120,7 @@ struct ScaleView {
     int64_t stride_kb;    // bytes between consecutive contraction blocks of 32
     int32_t n_row;        // mxf4: number of row tiles; mxf8: number of rows
     int32_t n_kb;         // number of contraction blocks
+    int32_t row_shift;    // per-row images only: operand row r reads scale row r >> row_shift (5: a 2D-block operand, n_row counts tiles)
 };
 
 struct GemmParams {
@@ -306,12 +315,12 @@ template <int KIND, int CTAS>
 __device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
 {
-    if (KIND == KIND_MXF4 && CTAS == 2) {
+    if (kind_fp4(KIND) && CTAS == 2) {
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                      " tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
                      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
                      : "memory");
-    } else if (KIND == KIND_MXF4) {
+    } else if (kind_fp4(KIND)) {
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                      " tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
                      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
@@ -351,7 +360,7 @@ __device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
 template <int KIND, int CTAS>
 __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_id)
 {
-    const uint32_t fmt = KIND == KIND_MXF4 ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
+    const uint32_t fmt = kind_fp4(KIND) ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
     return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) |
            ((uint32_t)((BM * CTAS) >> 4) << 24) | (a_sf_id << 29);
 }
@@ -568,16 +577,42 @@ __device__ __forceinline__ void ldg_v4(const uint8_t *ptr, uint32_t *w)
     asm volatile("ld.global.nc.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(ptr));
 }
 
-// Builds the scale images of one unit (up to 8 stages = 32 contraction blocks from k0) for per-row scales.  Lane l
-// takes operand rows l, l+32, ... (4 of A, 8 of B); the 32 scale bytes of a row for the whole unit are contiguous
-// in the scale matrix, so the common case is two 16-byte loads per row, all 24 issued before any use.
-__device__ __forceinline__ void build_row_scale_images(const GemmParams &p, const Tile &t, int k0, int n_stages, uint8_t *images, int lane)
+// Builds the scale images of one unit (32 contraction blocks from k0: 8 MXFP8 stages, or 4 FP4 stages of two chunks)
+// for per-row scales.  Lane l takes operand rows l, l+32, ... (4 of A, 8 of B); the 32 scale bytes of a row for the
+// whole unit are contiguous in the scale matrix, so the common case is two 16-byte loads per row, all 24 issued
+// before any use.  An operand with 2D-block scales (row_shift 5) reads its tile's scale row instead (every lane the
+// same bytes); if that view is transposed (consecutive blocks stride_kb apart) each lane fetches one block's byte
+// and the 32 bytes are regrouped through `scratch` (12 x 32 bytes).
+template <int KIND>
+__device__ __forceinline__ void build_row_scale_images(const GemmParams &p, const Tile &t, int k0, int n_stages, uint8_t *images,
+                                                       uint8_t *scratch, int lane)
 {
     uint32_t w[12][8];
+    const bool a_tr = p.sfa.row_shift != 0 && p.sfa.stride_kb != 1, b_tr = p.sfb.row_shift != 0 && p.sfb.stride_kb != 1;
+    if (a_tr || b_tr) {
+#pragma unroll
+        for (int q = 0; q < 12; q++) {
+            if (q < 4 ? a_tr : b_tr) {
+                const ScaleView &v = q < 4 ? p.sfa : p.sfb;
+                const int row = (q < 4 ? t.a_row0 + 32 * q : t.b_row0 + 32 * (q - 4)) >> v.row_shift;
+                const int kb0 = ((q < 4 ? t.a_k0 : t.b_k0) + k0) >> 5;
+                uint32_t b;
+                load_scale(v, row, kb0 + lane, b);
+                scratch[q * 32 + lane] = (uint8_t)b;
+            }
+        }
+        __syncwarp();
+    }
 #pragma unroll
     for (int q = 0; q < 12; q++) {
         const ScaleView &v = q < 4 ? p.sfa : p.sfb;
-        const int row = q < 4 ? t.a_row0 + lane + 32 * q : t.b_row0 + lane + 32 * (q - 4);
+        if (q < 4 ? a_tr : b_tr) {
+            const uint4 lo = reinterpret_cast<const uint4 *>(scratch + q * 32)[0], hi = reinterpret_cast<const uint4 *>(scratch + q * 32)[1];
+            w[q][0] = lo.x; w[q][1] = lo.y; w[q][2] = lo.z; w[q][3] = lo.w;
+            w[q][4] = hi.x; w[q][5] = hi.y; w[q][6] = hi.z; w[q][7] = hi.w;
+            continue;
+        }
+        const int row = (q < 4 ? t.a_row0 + lane + 32 * q : t.b_row0 + lane + 32 * (q - 4)) >> v.row_shift;
         const int kb0 = ((q < 4 ? t.a_k0 : t.b_k0) + k0) >> 5;
         const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
         if (row < v.n_row && kb0 + 32 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 15) == 0) {
@@ -588,15 +623,32 @@ __device__ __forceinline__ void build_row_scale_images(const GemmParams &p, cons
             for (int st = 0; st < 8; st++) load_scale_word(v, row, kb0 + 4 * st, w[q][st]);
         }
     }
+    if (KIND == KIND_MXF8) {
 #pragma unroll
-    for (int st = 0; st < 8; st++) {
-        if (st < n_stages) {
-            uint4 *img = reinterpret_cast<uint4 *>(images + st * kImageStageBytesMxf8);
-            img[lane] = make_uint4(w[0][st], w[1][st], w[2][st], w[3][st]);           // A
-            img[32 + lane] = make_uint4(w[4][st], w[5][st], w[6][st], w[7][st]);      // B rows 0..127
-            img[64 + lane] = make_uint4(w[8][st], w[9][st], w[10][st], w[11][st]);    // B rows 128..255
+        for (int st = 0; st < 8; st++) {
+            if (st < n_stages) {
+                uint4 *img = reinterpret_cast<uint4 *>(images + st * kImageStageBytesMxf8);
+                img[lane] = make_uint4(w[0][st], w[1][st], w[2][st], w[3][st]);           // A
+                img[32 + lane] = make_uint4(w[4][st], w[5][st], w[6][st], w[7][st]);      // B rows 0..127
+                img[64 + lane] = make_uint4(w[8][st], w[9][st], w[10][st], w[11][st]);    // B rows 128..255
+            }
+        }
+    } else {
+#pragma unroll
+        for (int st = 0; st < 4; st++) {
+            if (st < n_stages) {
+                uint4 *img = reinterpret_cast<uint4 *>(images + st * kImageStageBytesMxf4R);
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    const int j = 2 * st + c;
+                    img[32 * c + lane] = make_uint4(w[0][j], w[1][j], w[2][j], w[3][j]);                 // A, chunk c
+                    img[64 + 64 * c + lane] = make_uint4(w[4][j], w[5][j], w[6][j], w[7][j]);            // B rows 0..127
+                    img[96 + 64 * c + lane] = make_uint4(w[8][j], w[9][j], w[10][j], w[11][j]);          // B rows 128..255
+                }
+            }
         }
     }
+    if (a_tr || b_tr) __syncwarp();   // scratch is rewritten for the next unit
 }
 
 // ---------------------------------------------------------------------------------------- epilogue store
@@ -724,12 +776,12 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                          const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
                          const __grid_constant__ GemmParams p)
 {
-    constexpr int kStageElems = KIND == KIND_MXF4 ? 256 : 128;   // contraction elements per stage (128 B per row)
-    constexpr int kMmaK = KIND == KIND_MXF4 ? 64 : 32;           // contraction elements per MMA (32 B per row)
-    constexpr int kElemsPerByte = KIND == KIND_MXF4 ? 2 : 1;
+    constexpr int kStageElems = kind_fp4(KIND) ? 256 : 128;   // contraction elements per stage (128 B per row)
+    constexpr int kMmaK = kind_fp4(KIND) ? 64 : 32;           // contraction elements per MMA (32 B per row)
+    constexpr int kElemsPerByte = kind_fp4(KIND) ? 2 : 1;
     constexpr int kStages = Cfg<CTAS>::kStages;
     constexpr int kBStageBytes = Cfg<CTAS>::kBStageBytes;
-    constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : kUnitStagesMxf8;   // stages whose scale images are built together
+    constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8 : kUnitStagesMxf4R;   // stages whose scale images are built together
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -894,6 +946,14 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image_rep(img + 256 + 256 * c));
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
                         }
+                    } else if (KIND == KIND_MXF4R) {
+                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
+#pragma unroll
+                        for (int c = 0; c < 2; c++) {
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image(img + 512 * c));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image(img + 1024 + 1024 * c));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image(img + 1536 + 1024 * c));
+                        }
                     } else {
                         const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(img));
@@ -907,8 +967,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
                     for (int i = 0; i < 4; i++) {
                         if (i < n_mma) {
-                            const int chunk = KIND == KIND_MXF4 ? (i >> 1) : 0;
-                            const uint32_t sf_id = KIND == KIND_MXF4 ? 2u * (i & 1) : (uint32_t)i;
+                            const int chunk = kind_fp4(KIND) ? (i >> 1) : 0;
+                            const uint32_t sf_id = kind_fp4(KIND) ? 2u * (i & 1) : (uint32_t)i;
                             tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
                                                                  instr_desc<KIND, CTAS>(sf_id, sf_id), sf_tmem + 4 * chunk,
                                                                  sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
@@ -952,13 +1012,14 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, unit++) {
                 const int buf = unit & 1;
                 uint8_t *images = smem_images + buf * kCacheBufBytes;
-                if (KIND == KIND_MXF8) {
+                if (KIND != KIND_MXF4) {
                     // per-row scales: straight from global memory into the images
                     if (lane == 0)
                         ok = mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     if (!ok) break;
-                    build_row_scale_images(p, t, k0, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images, lane);
+                    build_row_scale_images<KIND>(p, t, k0, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images,
+                                                 smem_compact, lane);
                 } else {
                     const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
                     uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
@@ -1624,6 +1685,53 @@ extern "C" fp4q_status fp4q_mxfp8_gemm(const uint8_t *aq, int64_t ld_aq, const u
     p.out_f32 = dt == FP4Q_OUT_F32;
     dense_tiles(p);
     return launch_gemm<KIND_MXF8>(A, B, p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_fwd_act1d(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, int64_t ld_xs, int64_t T,
+                                           const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt, void *ws, size_t ws_bytes,
+                                           void *stream)
+{
+    if (!tensor_ok(W)) return W ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (T < 0) return FP4Q_ERR_SHAPE;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    const int64_t N = W->rows, K = W->cols;
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (T == 0 || N == 0) return FP4Q_OK;
+    if (!Y || !xq || !xs || !W->q_rm || !W->scale) return FP4Q_ERR_NULL;
+    if (ldy < N || ld_xq < round_up(K, 32) / 2 || ld_xs < ceil_div(K, 32)) return FP4Q_ERR_SHAPE;
+    Operand A, B = operand_rm(W);
+    A.payload = xq; A.rows = T; A.row_bytes = round_up(K, 32) / 2; A.ld_bytes = ld_xq;
+    A.sf = ScaleView{xs, ld_xs, 1, (int32_t)T, (int32_t)ceil_div(K, 32), 0};
+    B.sf.row_shift = 5;
+    GemmParams p = {};
+    p.C = Y; p.ldc = ldy; p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)K;
+    p.out_f32 = dt == FP4Q_OUT_F32;
+    dense_tiles(p);
+    return launch_gemm<KIND_MXF4R>(A, B, p, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_wgrad_act1d(const fp4q_tensor *dY, const uint8_t *xtq, int64_t ld_xtq, const uint8_t *xts,
+                                             int64_t ld_xts, int64_t K, void *dW, int64_t ldw, fp4q_out dt, int accumulate,
+                                             void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(dY)) return dY ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (K < 0) return FP4Q_ERR_SHAPE;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (accumulate && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    const int64_t T = dY->rows, N = dY->cols;
+    if (T > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (N == 0 || K == 0) return FP4Q_OK;
+    if (!dW || !dY->q_t || !dY->scale || !xtq || !xts) return FP4Q_ERR_NULL;
+    if (ldw < K || ld_xtq < round_up(T, 32) / 2 || ld_xts < ceil_div(T, 32)) return FP4Q_ERR_SHAPE;
+    Operand A = operand_t(dY), B;
+    A.sf.row_shift = 5;
+    B.payload = xtq; B.rows = K; B.row_bytes = round_up(T, 32) / 2; B.ld_bytes = ld_xtq;
+    B.sf = ScaleView{xts, ld_xts, 1, (int32_t)K, (int32_t)ceil_div(T, 32), 0};
+    GemmParams p = {};
+    p.C = dW; p.ldc = ldw; p.M = (int32_t)N; p.N = (int32_t)K; p.K = (int32_t)T;
+    p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = accumulate ? 1 : 0;
+    dense_tiles(p);
+    return launch_gemm<KIND_MXF4R>(A, B, p, ws, ws_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------------------

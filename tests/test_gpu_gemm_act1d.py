@@ -1,0 +1,95 @@
+"""GPU parity of the products with the paper's mixed layout (Section 3.1: 2D blocks for weights and gradients, 1D
+blocks for activations): Y = X^ W^^T with X in 1D blocks along the channels, and dW = dY^^T X^_t with X re-quantized
+in 1D blocks along the tokens.  Operands are quantized on the GPU (bit-exactness is covered elsewhere and re-checked
+here), the expected products come from the oracle's dequantized operands in float64."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_24953_b200 import binding, workloads
+from tests.gpu_util import assert_matches_oracle, dequant_from_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def check(got, ref, what):
+    g = got.double().cpu().numpy()
+    if got.dtype == torch.bfloat16:
+        ref = oracle.bf16_round(ref)
+    rel = np.linalg.norm(g - ref) / np.linalg.norm(ref)
+    assert rel <= 1e-3, "%s: relative Frobenius error %.3e" % (what, rel)
+    row_inf = np.abs(ref).max(axis=1, keepdims=True)
+    assert (np.abs(g - ref) <= 1e-2 * row_inf + 1e-300).all(), "%s: per-row max-abs bound violated" % what
+
+
+def act1d(x):
+    """Row-wise 1D encoding from the GPU, checked against the oracle; returns (q, s, dequantized [T, K])."""
+    rows, cols = x.shape
+    q, s = binding.fp4q_quantize1d(x)
+    torch.cuda.synchronize()
+    oq, os_ = oracle.quantize1d(workloads.bf16_bits(x))
+    assert np.array_equal(q.cpu().numpy()[:, :oq.shape[1]], oq) and np.array_equal(s.cpu().numpy()[:, :os_.shape[1]], os_)
+    return q, s, oracle.dequantize1d(oq, os_, rows, cols)
+
+
+def act1d_t(x):
+    """Transposed 1D encoding from the GPU, checked; returns (q, s, dequantized as [T, K])."""
+    rows, cols = x.shape
+    q, s = binding.fp4q_quantize1d_t(x)
+    torch.cuda.synchronize()
+    oq, os_ = oracle.quantize1d_t(workloads.bf16_bits(x))
+    assert np.array_equal(q.cpu().numpy()[:, :oq.shape[1]], oq) and np.array_equal(s.cpu().numpy()[:, :os_.shape[1]], os_)
+    return q, s, oracle.dequantize1d(oq, os_, cols, rows).T
+
+
+SHAPES = [(128, 256, 256),      # one tile (one-CTA kernel)
+          (384, 512, 1280),     # pairs, several units of four stages, ragged last unit
+          (200, 300, 416),      # ragged in every dimension (K tail inside an MMA)
+          (1024, 768, 2048)]    # several tiles per CTA
+
+
+@pytest.mark.parametrize("T,N,K", SHAPES)
+@pytest.mark.parametrize("dt", [binding.OUT_BF16, binding.OUT_F32])
+def test_forward_with_1d_activations(T, N, K, dt):
+    x = workloads.activations_gauss_outliers(T, K, seed=1, device="cuda")
+    w = workloads.weights(N, K, seed=2, device="cuda")
+    xq, xs, x_hat = act1d(x)
+    W = assert_matches_oracle(w, binding.ROUND_NEAREST, seed=0, tensor_id=0)
+    y = binding.fp4q_gemm_fwd_act1d(xq, xs, T, W, dt=dt)
+    torch.cuda.synchronize()
+    check(y, oracle.gemm_fwd(x_hat, dequant_from_gpu(W)), "forward, 1D activations")
+
+
+@pytest.mark.parametrize("T,N,K", SHAPES)
+def test_wgrad_with_1d_activations(T, N, K):
+    x = workloads.activations_gauss_outliers(T, K, seed=3, device="cuda")
+    dy = workloads.gradients_rowscaled(T, N, seed=4, device="cuda")
+    xtq, xts, x_hat_t = act1d_t(x)
+    dY = assert_matches_oracle(dy, binding.ROUND_STOCHASTIC, seed=7, tensor_id=2)
+    dw = binding.fp4q_gemm_wgrad_act1d(dY, xtq, xts, K, dt=binding.OUT_F32)
+    torch.cuda.synchronize()
+    ref = oracle.gemm_wgrad(dequant_from_gpu(dY), x_hat_t)
+    check(dw, ref, "wgrad, 1D activations")
+    # accumulation into an FP32 gradient buffer
+    acc = torch.full((N, K), 0.25, dtype=torch.float32, device="cuda")
+    binding.fp4q_gemm_wgrad_act1d(dY, xtq, xts, K, out=acc, dt=binding.OUT_F32, accumulate=True)
+    torch.cuda.synchronize()
+    check(acc, ref + 0.25, "wgrad, 1D activations, accumulate")
+
+
+def test_mixed_layout_differs_from_all_2d_and_shows_the_inconsistency():
+    """The two 1D encodings of one activation dequantize to different tensors (Figure 1), the 2D ones do not; and the
+    1D forward product is not the all-2D product (the kernel really reads per-row scales)."""
+    T, N, K = 256, 256, 512
+    x = workloads.activations_gauss_outliers(T, K, seed=5, device="cuda")
+    w = workloads.weights(N, K, seed=6, device="cuda")
+    xq, xs, x_fwd = act1d(x)
+    _, _, x_bwd = act1d_t(x)
+    assert np.linalg.norm(x_fwd - x_bwd) / np.linalg.norm(x_fwd) > 1e-2
+    W = binding.fp4q_quantize2d(w)
+    X2 = binding.fp4q_quantize2d(x)
+    y1 = binding.fp4q_gemm_fwd_act1d(xq, xs, T, W, dt=binding.OUT_F32)
+    y2 = binding.fp4q_gemm_fwd(X2, W, dt=binding.OUT_F32)
+    torch.cuda.synchronize()
+    assert (y1 - y2).norm() / y2.norm() > 1e-3
