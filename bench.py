@@ -430,7 +430,24 @@ def run_extras(torch, binding, workloads, dev, ws):
         "workload": "Y = X W^T, %d x %d x %d, output as 2D-block FP4 (stochastic rounding)" % (T, H, H),
         "fused_ms": ms_f, "product_ms": ms_p, "separate_quantize_ms": ms_s,
         "fused_tflops": 2.0 * T * H * H / (ms_f * 1e-3) / 1e12, "speedup_vs_unfused": (ms_p + ms_s) / ms_f}
-    del X, Wq, Wk, qx4, qw4, y, qy
+    # --- the paper's mixed layout: activations in 1D blocks (two encodings of X), weights and gradients in 2D blocks
+    dY4 = binding.fp4q_quantize2d(workloads.gradients_rowscaled(T, H, cfg.data_seed + 2, dev), mode=SR, seed=1, tensor_id=3)
+    x1q, x1s = binding.fp4q_quantize1d(X)
+    x1tq, x1ts = binding.fp4q_quantize1d_t(X)
+    dw = torch.empty(H, H, dtype=torch.float32, device=dev)
+    ms_q1 = timed(lambda: binding.fp4q_quantize1d(X))
+    ms_q1t = timed(lambda: binding.fp4q_quantize1d_t(X))
+    ms_f1 = timed(lambda: binding.fp4q_gemm_fwd_act1d(x1q, x1s, T, qw4, out=y, ws=ws))
+    ms_w1 = timed(lambda: binding.fp4q_gemm_wgrad_act1d(dY4, x1tq, x1ts, H, out=dw, ws=ws))
+    ms_w2 = timed(lambda: binding.fp4q_gemm_wgrad(dY4, qx4, out=dw, ws=ws))
+    out["mixed_layout_1d_activations"] = {
+        "workload": "X %d x %d in 1 x 32 blocks (row-wise for the forward product, transposed for the weight gradient), "
+                    "W and dY %d x %d in 32 x 32 blocks" % (T, H, H, H),
+        "quantize1d_gbs": T * H * (2.5 + 1 / 32) / (ms_q1 * 1e-3) / 1e9,
+        "quantize1d_t_gbs": T * H * (2.5 + 1 / 32) / (ms_q1t * 1e-3) / 1e9,
+        "fwd_tflops": 2.0 * T * H * H / (ms_f1 * 1e-3) / 1e12, "wgrad_tflops": 2.0 * T * H * H / (ms_w1 * 1e-3) / 1e12,
+        "all_2d_fwd_tflops": 2.0 * T * H * H / (ms_p * 1e-3) / 1e12, "all_2d_wgrad_tflops": 2.0 * T * H * H / (ms_w2 * 1e-3) / 1e12}
+    del X, Wq, Wk, qx4, qw4, y, qy, dY4, x1q, x1s, x1tq, x1ts, dw
 
     # --- grouped MoE expert layer: 128 experts, hidden 2048, expert FFN 768, top-8 of 16384 tokens
     moe = workloads.CONFIG_MOE

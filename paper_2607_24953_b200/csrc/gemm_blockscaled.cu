@@ -58,7 +58,6 @@ static_assert(kUnitStagesMxf8 * kImageStageBytesMxf8 == kCacheBufBytes, "both ki
 constexpr int kUnitStagesMxf4R = 4;
 constexpr int kImageStageBytesMxf4R = 3072;
 static_assert(kUnitStagesMxf4R * kImageStageBytesMxf4R == kCacheBufBytes, "all kinds share the image buffers");
-constexpr int kSmemCache = kCompactBytes + 2 * kCacheBufBytes;
 // Epilogue staging of the pair kernel: each of the 8 epilogue warps owns 32 rows x 128 bytes, written from registers
 // (128-byte swizzle: the 16-byte pieces of 8 rows fall into different banks) and drained by a TMA store, which keeps
 // the output off the load/store unit that the MMA warp's instructions also pass through.
@@ -67,9 +66,22 @@ constexpr int kStagingWarpBytes = 32 * 128;
 // CTAS = 1: one CTA per 128x256 tile, it loads all 256 B rows.  CTAS = 2: a cluster of two CTAs shares a 256x256
 // tile through cta_group::2 MMAs; each CTA loads its own 128 A rows and half of the B rows, which halves the
 // B-operand shared-memory and L2 traffic per CTA and leaves room for two more ring stages.
-template <int CTAS>
+// KIND_MXF4: FP4 payloads, 2D-block scales on both operands (replicated scale images).  KIND_MXF8: E4M3 payloads,
+// per-row scales.  KIND_MXF4R: FP4 payloads with per-row scale images - an operand quantized in 1D blocks (the
+// paper's activation layout) next to a 2D-block operand, whose tile scale is then expanded to its 32 rows.
+enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2 };
+__host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8; }
+
+// Per-row scale images are rebuilt every 4 (FP4) or 8 (MXFP8) stages, and the way from "the MMAs have finished with
+// a buffer" to "the leader may copy the next unit out of it" (commit to both CTAs, build, report to the leader)
+// takes longer than one such unit runs.  The pair kernel for those kinds therefore keeps four image buffers
+// (three units of slack) and pays for them with one ring stage.
+template <int KIND, int CTAS>
 struct Cfg {
-    static constexpr int kStages = CTAS == 2 ? 5 : 4;
+    static constexpr int kImageBufs = (CTAS == 2 && KIND != KIND_MXF4) ? 4 : 2;
+    static constexpr int kLog2ImageBufs = kImageBufs == 4 ? 2 : 1;
+    static constexpr int kStages = CTAS == 2 ? (KIND == KIND_MXF4 ? 5 : 4) : 4;
+    static constexpr int kSmemCache = kCompactBytes + kImageBufs * kCacheBufBytes;
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
@@ -107,11 +119,6 @@ extern "C" int fp4q_debug_events(void *host) { return (int)cudaMemcpyFromSymbol(
 #endif
 constexpr uint8_t kScalePad = 127;           // UE8M0 code of 1.0 for scale slots beyond the tensor (their payload is 0)
 
-// KIND_MXF4: FP4 payloads, 2D-block scales on both operands (replicated scale images).  KIND_MXF8: E4M3 payloads,
-// per-row scales.  KIND_MXF4R: FP4 payloads with per-row scale images - an operand quantized in 1D blocks (the
-// paper's activation layout) next to a 2D-block operand, whose tile scale is then expanded to its 32 rows.
-enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2 };
-__host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8; }
 enum { MODE_DENSE = 0, MODE_GROUPED_ROWS = 1, MODE_GROUPED_K = 2 };
 
 struct ScaleView {
@@ -583,11 +590,9 @@ __device__ __forceinline__ void ldg_v4(const uint8_t *ptr, uint32_t *w)
 // before any use.  An operand with 2D-block scales (row_shift 5) reads its tile's scale row instead (every lane the
 // same bytes); if that view is transposed (consecutive blocks stride_kb apart) each lane fetches one block's byte
 // and the 32 bytes are regrouped through `scratch` (12 x 32 bytes).
-template <int KIND>
-__device__ __forceinline__ void build_row_scale_images(const GemmParams &p, const Tile &t, int k0, int n_stages, uint8_t *images,
-                                                       uint8_t *scratch, int lane)
+// Two steps, so that the loads are in flight while the builder waits for the image buffer to be free.
+__device__ __forceinline__ void load_row_scales(const GemmParams &p, const Tile &t, int k0, uint8_t *scratch, int lane, uint32_t (&w)[12][8])
 {
-    uint32_t w[12][8];
     const bool a_tr = p.sfa.row_shift != 0 && p.sfa.stride_kb != 1, b_tr = p.sfb.row_shift != 0 && p.sfb.stride_kb != 1;
     if (a_tr || b_tr) {
 #pragma unroll
@@ -623,6 +628,12 @@ __device__ __forceinline__ void build_row_scale_images(const GemmParams &p, cons
             for (int st = 0; st < 8; st++) load_scale_word(v, row, kb0 + 4 * st, w[q][st]);
         }
     }
+    if (a_tr || b_tr) __syncwarp();   // scratch is rewritten for the next unit
+}
+
+template <int KIND>
+__device__ __forceinline__ void store_row_scale_images(const uint32_t (&w)[12][8], int n_stages, uint8_t *images, int lane)
+{
     if (KIND == KIND_MXF8) {
 #pragma unroll
         for (int st = 0; st < 8; st++) {
@@ -648,7 +659,6 @@ __device__ __forceinline__ void build_row_scale_images(const GemmParams &p, cons
             }
         }
     }
-    if (a_tr || b_tr) __syncwarp();   // scratch is rewritten for the next unit
 }
 
 // ---------------------------------------------------------------------------------------- epilogue store
@@ -779,29 +789,30 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kStageElems = kind_fp4(KIND) ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = kind_fp4(KIND) ? 64 : 32;           // contraction elements per MMA (32 B per row)
     constexpr int kElemsPerByte = kind_fp4(KIND) ? 2 : 1;
-    constexpr int kStages = Cfg<CTAS>::kStages;
-    constexpr int kBStageBytes = Cfg<CTAS>::kBStageBytes;
+    constexpr int kStages = Cfg<KIND, CTAS>::kStages;
+    constexpr int kBStageBytes = Cfg<KIND, CTAS>::kBStageBytes;
     constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8 : kUnitStagesMxf4R;   // stages whose scale images are built together
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_compact = smem + Cfg<CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
-    uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and two buffers of ready scale images (either kind)
-    uint8_t *smem_staging = smem_compact + Cfg<CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<CTAS>::kSmemStaging);
+    uint8_t *smem_compact = smem + Cfg<KIND, CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
+    uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and the buffers of ready scale images (any kind)
+    uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS>::kSmemStaging);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
-    // bars[14..15] scale images full, bars[16..17] scale images empty, bars[18] tensor pipe drained (abort path),
-    // bars[19..20] (leader of a pair) the second CTA's scale images full
+    // bars[18] tensor pipe drained (abort path), bars[24..27] scale images full, bars[28..31] scale images empty,
+    // bars[32..35] (leader of a pair) the second CTA's scale images full - one of each per image buffer
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 21);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 21) + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
-    const uint32_t bar_cache_full = smem_u32(bars + 14), bar_cache_empty = smem_u32(bars + 16);
-    const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 19);
+    const uint32_t bar_cache_full = smem_u32(bars + 24), bar_cache_empty = smem_u32(bars + 28);
+    const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 32);
+    constexpr uint32_t kBufMask = Cfg<KIND, CTAS>::kImageBufs - 1, kBufShift = Cfg<KIND, CTAS>::kLog2ImageBufs;
 
     // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
     const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
@@ -818,7 +829,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         mbar_init(bar_acc_full, 1);
         mbar_init(bar_drain, 1);
         mbar_init(bar_acc_empty, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
-        for (int b = 0; b < 2; b++) {
+        for (int b = 0; b < Cfg<KIND, CTAS>::kImageBufs; b++) {
             mbar_init(bar_cache_full + 8 * b, 1);
             mbar_init(bar_cache_empty + 8 * b, 1);
             mbar_init(bar_peer_cache_full + 8 * b, 1);
@@ -939,7 +950,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (issuer) {
                     const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
                     if (KIND == KIND_MXF4) {
-                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
+                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
                         for (int c = 0; c < 2; c++) {
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image_rep(img + 128 * c));
@@ -947,7 +958,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
                         }
                     } else if (KIND == KIND_MXF4R) {
-                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
+                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
 #pragma unroll
                         for (int c = 0; c < 2; c++) {
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image(img + 512 * c));
@@ -955,7 +966,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image(img + 1536 + 1024 * c));
                         }
                     } else {
-                        const uint32_t img = smem_u32(smem_images + (unit & 1u) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
+                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(img));
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8, smem_desc_scale_image(img + 512));
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12, smem_desc_scale_image(img + 1024));
@@ -977,7 +988,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
                     if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
                     if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
-                        tcgen05_commit<CTAS>(bar_cache_empty + 8 * (unit & 1u));   // the unit's images have been copied
+                        tcgen05_commit<CTAS>(bar_cache_empty + 8 * (unit & kBufMask));   // the unit's images have been copied
                 }
                 if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1) unit++;
                 TRACE_ADD(c_issue, tt);
@@ -1010,16 +1021,19 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             Tile t;
             decode_tile(p, tile, rank, t);
             for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, unit++) {
-                const int buf = unit & 1;
+                const int buf = unit & kBufMask;
                 uint8_t *images = smem_images + buf * kCacheBufBytes;
                 if (KIND != KIND_MXF4) {
-                    // per-row scales: straight from global memory into the images
+                    // per-row scales: from global memory into registers, and once the buffer is free into the images.
+                    // In a pair the buffer is released by the leader's multicast commit: probe (a suspended try_wait
+                    // is not reliably woken early by a remote arrival).
+                    uint32_t w[12][8];
+                    load_row_scales(p, t, k0, smem_compact, lane, w);
                     if (lane == 0)
-                        ok = mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                        ok = mbar_wait_impl<kRelaxedNs, CTAS == 2>(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     if (!ok) break;
-                    build_row_scale_images<KIND>(p, t, k0, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images,
-                                                 smem_compact, lane);
+                    store_row_scale_images<KIND>(w, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images, lane);
                 } else {
                     const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
                     uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
@@ -1027,8 +1041,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
                     __syncwarp();
                     if (lane == 0)
-                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
-                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
+                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     if (!ok) break;
                     const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
@@ -1049,10 +1063,9 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
-                if (lane == 0) {
-                    if (CTAS == 1 || leader) mbar_arrive(bar_cache_full + 8 * buf);
-                    else mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * buf, 0));   // the leader copies both CTAs' images
-                }
+                // In the second CTA of a pair the arrival is forwarded to the leader by warp 2: the remote arrival
+                // stalls its issuing thread for about a thousand cycles, which this warp spends on the next unit.
+                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);
             }
         }
     } else if (warp == 2) {
@@ -1079,17 +1092,17 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             } else {
                 if (ok && lane == 0) {
                     if ((sg.it & (kUnitStages - 1)) == 0 && !unit_seen) {
-                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x510u + (unit & 1u));
+                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * (unit & kBufMask), (unit >> kBufShift) & 1u, abort_flag, p.status, 0x510u + (unit & kBufMask));
                         if (ok && CTAS == 2)
-                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * (unit & 1u), (unit >> 1) & 1u, abort_flag, p.status, 0x520u + (unit & 1u));
+                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * (unit & kBufMask), (unit >> kBufShift) & 1u, abort_flag, p.status, 0x520u + (unit & kBufMask));
                     }
                     if ((sg.it & (kUnitStages - 1)) == 0) unit_seen = false;
                     if (ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen) {
                         // second half of a unit: look whether the next unit's images are in place already, so that
                         // the unit boundary costs no extra probes on the critical path
                         const uint32_t nu = unit + 1;
-                        unit_seen = mbar_test_wait(bar_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u) &&
-                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * (nu & 1u), (nu >> 1) & 1u));
+                        unit_seen = mbar_test_wait(bar_cache_full + 8 * (nu & kBufMask), (nu >> kBufShift) & 1u) &&
+                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * (nu & kBufMask), (nu >> kBufShift) & 1u));
                     }
                     if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
                     if (ok) {
@@ -1142,6 +1155,21 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
             sg.next(p, kStageElems);
         }
+        if (CTAS == 2 && !leader && lane == 0) {
+            // Second CTA of a pair: report each unit of scale images the builder has finished to the leader, which
+            // issues the scale copies of both CTAs.
+            bool fwd_ok = true;
+            uint32_t u = 0;
+            for (int tile = first_tile; fwd_ok && tile < p.n_tile_total; tile += tile_step) {
+                Tile t;
+                decode_tile(p, tile, rank, t);
+                for (int k0 = 0; fwd_ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, u++) {
+                    fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * (u & kBufMask), (u >> kBufShift) & 1u, abort_flag, p.status, 0x530u + (u & kBufMask));
+                    if (fwd_ok) mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * (u & kBufMask), 0));
+                }
+            }
+        }
+        __syncwarp();
         if (lane == 0) { TRACE_OUT(p, 6, c_meet); TRACE_OUT(p, 7, c_poll); }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
@@ -1419,7 +1447,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
         if (!make_byte_map(&tmC, p.q_rm, p.M, round_up(p.N, 32) / 2, p.q_ld_rm, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return FP4Q_ERR_CUDA;
         if (p.q_t && !make_byte_map(&tmD, p.q_t, p.N, round_up(p.M, 32) / 2, p.q_ld_t, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) return FP4Q_ERR_CUDA;
     } else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
-    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<CTAS>::kBRows)) return FP4Q_ERR_CUDA;
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<KIND, CTAS>::kBRows)) return FP4Q_ERR_CUDA;
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
@@ -1431,7 +1459,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<CTAS>::kSmemBytes) != cudaSuccess)
+                                 Cfg<KIND, CTAS>::kSmemBytes) != cudaSuccess)
             return FP4Q_ERR_CUDA;
         attr_set = true;
     }
@@ -1443,7 +1471,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = Cfg<CTAS>::kSmemBytes;
+    cfg.dynamicSmemBytes = Cfg<KIND, CTAS>::kSmemBytes;
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
