@@ -72,16 +72,19 @@ constexpr int kStagingWarpBytes = 32 * 128;
 enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2 };
 __host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8; }
 
-// Per-row scale images are rebuilt every 4 (FP4) or 8 (MXFP8) stages, and the way from "the MMAs have finished with
-// a buffer" to "the leader may copy the next unit out of it" (commit to both CTAs, build, report to the leader)
-// takes longer than one such unit runs.  The pair kernel for those kinds therefore keeps four image buffers
-// (three units of slack) and pays for them with one ring stage.
+// Per-row scale images are rebuilt every 4 (FP4) or 8 (MXFP8) stages from 12 KB of scale bytes, whose global-memory
+// latency under the operand traffic (about 3000 cycles) exceeds the time such a unit runs.  The kernels for those
+// kinds therefore fetch the bytes two units ahead with cp.async into raw buffers (no registers are held meanwhile)
+// and pay for the buffers with one ring stage; the pair kernel also keeps a third image buffer, because the way
+// from "the MMAs have finished with a buffer" to "the leader may copy the next unit out of it" (commit to both
+// CTAs, build, report to the leader) is longer than one unit as well.
 template <int KIND, int CTAS>
 struct Cfg {
-    static constexpr int kImageBufs = (CTAS == 2 && KIND != KIND_MXF4) ? 4 : 2;
-    static constexpr int kLog2ImageBufs = kImageBufs == 4 ? 2 : 1;
-    static constexpr int kStages = CTAS == 2 ? (KIND == KIND_MXF4 ? 5 : 4) : 4;
-    static constexpr int kSmemCache = kCompactBytes + kImageBufs * kCacheBufBytes;
+    static constexpr bool kRowImages = KIND != KIND_MXF4;
+    static constexpr int kImageBufs = (CTAS == 2 && kRowImages) ? 3 : 2;
+    static constexpr int kRawBufs = kRowImages ? 2 : 0;
+    static constexpr int kStages = (CTAS == 2 ? 5 : 4) - (kRowImages ? 1 : 0);
+    static constexpr int kSmemCache = kCompactBytes + (kImageBufs + kRawBufs) * kCacheBufBytes;
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
@@ -778,6 +781,146 @@ __device__ __forceinline__ void store_row_chunk(const GemmParams &p, int64_t row
     }
 }
 
+// Position in a ring of image buffers: buffer index and the parity of the barrier phase that goes with it.
+struct BufRing {
+    uint32_t buf = 0, phase = 0;
+    __device__ __forceinline__ void next(uint32_t n) { if (++buf == n) { buf = 0; phase ^= 1u; } }
+};
+
+// The stream of scale units (kUnitStages stages of one tile) a CTA works through.
+struct UnitIter {
+    int tile, step, rank, k0;
+    Tile t;
+    __device__ __forceinline__ void seek(const GemmParams &p)
+    {
+        while (tile < p.n_tile_total) {
+            decode_tile(p, tile, rank, t);
+            if (k0 < t.k_len) return;
+            tile += step;
+            k0 = 0;
+        }
+    }
+    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_) { tile = first; step = step_; rank = rank_; k0 = 0; seek(p); }
+    __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
+    __device__ __forceinline__ void next(const GemmParams &p, int unit_elems) { k0 += unit_elems; seek(p); }
+};
+
+__device__ __forceinline__ void cp_async(uint32_t dst, const void *src, int bytes, int src_bytes)
+{
+    if (bytes == 16) asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+    else if (bytes == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+// Raw scale bytes of one unit (32 contraction blocks from k0), asynchronously into `raw` (12 KB): slot q (1 KB,
+// q < 4: A rows 32q.., q >= 4: B rows 32(q-4)..) holds 32 bytes per lane, the scale bytes of the lane's operand row.
+// A 2D-block operand (row_shift 5) needs only 32 bytes per row tile: they are packed at the start of the operand's
+// first slot; if its view is transposed (blocks stride_kb apart, row tiles contiguous) lane l fetches block l's
+// bytes for the operand's 4 or 8 row tiles into the first 8 bytes of its entry of that slot.  Bytes beyond the tensor arrive as zero.  Every lane commits
+// exactly one cp.async group per call.
+__device__ __forceinline__ void issue_raw_scales(const GemmParams &p, const Tile &t, int k0, uint8_t *raw, int lane)
+{
+#pragma unroll
+    for (int op = 0; op < 2; op++) {
+        const ScaleView &v = op == 0 ? p.sfa : p.sfb;
+        const int nq = op == 0 ? 4 : 8, q0 = op == 0 ? 0 : 4;
+        const int row0 = op == 0 ? t.a_row0 : t.b_row0;
+        const int kb0 = ((op == 0 ? t.a_k0 : t.b_k0) + k0) >> 5;
+        if (v.row_shift != 0 && v.stride_kb != 1) {
+            const int rt0 = row0 >> 5, kb = kb0 + lane, nbytes = nq;   // 4 or 8 row tiles, one byte each
+            uint8_t *dst = raw + q0 * 1024 + lane * 32;
+            const uint8_t *src = v.ptr + (int64_t)kb * v.stride_kb + rt0;
+            const int valid = kb < v.n_kb ? max(0, min(nbytes, v.n_row - rt0)) : 0;
+            if (v.stride_row == 1 && (reinterpret_cast<uintptr_t>(src) & (nbytes - 1)) == 0) {
+                cp_async(smem_u32(dst), valid > 0 ? src : v.ptr - (reinterpret_cast<uintptr_t>(v.ptr) & 7), nbytes, valid);
+            } else {
+                for (int r = 0; r < nbytes; r++) {
+                    uint32_t b;
+                    load_scale(v, rt0 + r, kb, b);
+                    dst[r] = (uint8_t)b;
+                }
+            }
+            continue;
+        }
+        if (v.row_shift != 0) {
+            // 2D-block operand, blocks contiguous: the 32 bytes of each of the operand's row tiles once (lanes
+            // 0 .. 2 nq - 1 copy 16 bytes each), packed at the start of the operand's first slot
+            if (lane < 2 * nq) {
+                const int rt = (row0 >> 5) + (lane >> 1), kb = kb0 + 16 * (lane & 1);
+                uint8_t *dst = raw + q0 * 1024 + lane * 16;
+                const uint8_t *src = v.ptr + (int64_t)rt * v.stride_row + kb;
+                if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+                    const int valid = rt < v.n_row ? max(0, min(16, v.n_kb - kb)) : 0;
+                    cp_async(smem_u32(dst), valid > 0 ? src : v.ptr - (reinterpret_cast<uintptr_t>(v.ptr) & 15), 16, valid);
+                } else {
+#pragma unroll
+                    for (int st = 0; st < 4; st++) {
+                        uint32_t word;
+                        load_scale_word(v, rt, kb + 4 * st, word);
+                        reinterpret_cast<uint32_t *>(dst)[st] = word;
+                    }
+                }
+            }
+            continue;
+        }
+#pragma unroll
+        for (int q = 0; q < nq; q++) {
+            const int row = row0 + lane + 32 * q;
+            uint8_t *dst = raw + (q0 + q) * 1024 + lane * 32;
+            const uint8_t *src = v.ptr + (int64_t)row * v.stride_row + kb0;
+            if (v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+                const int valid = row < v.n_row ? max(0, min(32, v.n_kb - kb0)) : 0;
+                const uint8_t *safe = v.ptr - (reinterpret_cast<uintptr_t>(v.ptr) & 15);
+                cp_async(smem_u32(dst), valid > 0 ? src : safe, 16, min(valid, 16));
+                cp_async(smem_u32(dst + 16), valid > 16 ? src + 16 : safe, 16, max(valid - 16, 0));
+            } else {
+#pragma unroll
+                for (int st = 0; st < 8; st++) {
+                    uint32_t word;
+                    load_scale_word(v, row, kb0 + 4 * st, word);
+                    reinterpret_cast<uint32_t *>(dst)[st] = word;
+                }
+            }
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// The unit's scale words from a raw buffer whose copies have completed: w[q][j] = the four scale bytes of the
+// lane's row of slot q for blocks 4j..4j+3.  Lanes read bytes other lanes copied: the caller synchronizes the warp
+// after its cp.async wait.
+__device__ __forceinline__ void read_raw_scales(const GemmParams &p, const uint8_t *raw, int lane, uint32_t (&w)[12][8])
+{
+#pragma unroll
+    for (int op = 0; op < 2; op++) {
+        const ScaleView &v = op == 0 ? p.sfa : p.sfb;
+        const int nq = op == 0 ? 4 : 8, q0 = op == 0 ? 0 : 4;
+        if (v.row_shift != 0 && v.stride_kb != 1) {
+            // lane l holds block l's bytes [row tile 0..]: words of four consecutive lanes, transposed as 4x4 bytes,
+            // are the four row tiles' words of one chunk
+            const uint2 mine = *reinterpret_cast<const uint2 *>(raw + q0 * 1024 + lane * 32);
+#pragma unroll
+            for (int h = 0; h < (op == 0 ? 1 : 2); h++) {
+                const uint32_t m = h == 0 ? mine.x : mine.y;
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    const uint4 tr = transpose4x4_bytes(__shfl_sync(0xFFFFFFFFu, m, 4 * j), __shfl_sync(0xFFFFFFFFu, m, 4 * j + 1),
+                                                        __shfl_sync(0xFFFFFFFFu, m, 4 * j + 2), __shfl_sync(0xFFFFFFFFu, m, 4 * j + 3));
+                    w[q0 + 4 * h + 0][j] = tr.x; w[q0 + 4 * h + 1][j] = tr.y; w[q0 + 4 * h + 2][j] = tr.z; w[q0 + 4 * h + 3][j] = tr.w;
+                }
+            }
+            continue;
+        }
+#pragma unroll
+        for (int q = 0; q < nq; q++) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(v.row_shift != 0 ? raw + q0 * 1024 + q * 32 : raw + (q0 + q) * 1024 + lane * 32);
+            const uint4 lo = src[0], hi = src[1];
+            w[q0 + q][0] = lo.x; w[q0 + q][1] = lo.y; w[q0 + q][2] = lo.z; w[q0 + q][3] = lo.w;
+            w[q0 + q][4] = hi.x; w[q0 + q][5] = hi.y; w[q0 + q][6] = hi.z; w[q0 + q][7] = hi.w;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------- kernel
 
 template <int KIND, int CTAS, int EPI>
@@ -799,6 +942,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     uint8_t *smem_b = smem + kStages * kAStageBytes;
     uint8_t *smem_compact = smem + Cfg<KIND, CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
     uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and the buffers of ready scale images (any kind)
+    uint8_t *smem_raw_scales = smem_images + Cfg<KIND, CTAS>::kImageBufs * kCacheBufBytes;   // per-row scales: bytes in flight
     uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS>::kSmemStaging);
     // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
@@ -812,7 +956,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
     const uint32_t bar_cache_full = smem_u32(bars + 24), bar_cache_empty = smem_u32(bars + 28);
     const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 32);
-    constexpr uint32_t kBufMask = Cfg<KIND, CTAS>::kImageBufs - 1, kBufShift = Cfg<KIND, CTAS>::kLog2ImageBufs;
+    constexpr int kImageBufs = Cfg<KIND, CTAS>::kImageBufs;
 
     // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
     const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
@@ -931,7 +1075,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0, unit = 0;
+        uint32_t stage = 0;
+        BufRing ring;   // image buffer of the current unit
         const bool issuer = elect_one();
         int ev_j = 0;
         TRACE_DECL(c_acc); TRACE_DECL(c_sync); TRACE_DECL(c_issue);
@@ -950,7 +1095,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (issuer) {
                     const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
                     if (KIND == KIND_MXF4) {
-                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
+                        const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
                         for (int c = 0; c < 2; c++) {
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image_rep(img + 128 * c));
@@ -958,7 +1103,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
                         }
                     } else if (KIND == KIND_MXF4R) {
-                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
+                        const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
 #pragma unroll
                         for (int c = 0; c < 2; c++) {
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image(img + 512 * c));
@@ -966,7 +1111,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image(img + 1536 + 1024 * c));
                         }
                     } else {
-                        const uint32_t img = smem_u32(smem_images + (unit & kBufMask) * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
+                        const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf8);
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem, smem_desc_scale_image(img));
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8, smem_desc_scale_image(img + 512));
                         tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12, smem_desc_scale_image(img + 1024));
@@ -988,9 +1133,9 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
                     if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
                     if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
-                        tcgen05_commit<CTAS>(bar_cache_empty + 8 * (unit & kBufMask));   // the unit's images have been copied
+                        tcgen05_commit<CTAS>(bar_cache_empty + 8 * ring.buf);   // the unit's images have been copied
                 }
-                if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1) unit++;
+                if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1) ring.next(kImageBufs);
                 TRACE_ADD(c_issue, tt);
                 if (lane == 0) TRACE_EV(3, ev_j);
                 ev_j++;
@@ -1015,34 +1160,70 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // critical path, and nothing has to be written per stage.  A buffer is free again once the MMA warp's
         // commit reports that the last scale copy out of it has completed.  In a pair each CTA builds the images
         // of its own 128 A rows and of all 256 B rows.
-        uint32_t unit = 0;
+        BufRing ring;
         bool ok = true;
-        for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
+        if (KIND != KIND_MXF4) {
+            // per-row scales: the raw bytes of the next kRawBufs units are in flight (cp.async) while a unit is
+            // turned into images.  In a pair an image buffer is released by the leader's multicast commit: probe
+            // (a suspended try_wait is not reliably woken early by a remote arrival).
+            constexpr int kRawBufs = Cfg<KIND, CTAS>::kRawBufs > 0 ? Cfg<KIND, CTAS>::kRawBufs : 1;
+            UnitIter ahead, cur;
+            ahead.init(p, first_tile, tile_step, rank);
+            cur.init(p, first_tile, tile_step, rank);
+            uint32_t raw_fill = 0, raw_read = 0;
+            for (int i = 0; i < kRawBufs; i++) {
+                if (ahead.valid(p)) {
+                    issue_raw_scales(p, ahead.t, ahead.k0, smem_raw_scales + raw_fill * kCacheBufBytes, lane);
+                    ahead.next(p, kUnitStages * kStageElems);
+                } else {
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                }
+                if (++raw_fill == kRawBufs) raw_fill = 0;
+            }
+            while (cur.valid(p)) {
+                asm volatile("cp.async.wait_group %0;" ::"n"(kRawBufs - 1) : "memory");   // this unit's bytes have landed
+                __syncwarp();
+                uint32_t w[12][8];
+                read_raw_scales(p, smem_raw_scales + raw_read * kCacheBufBytes, lane, w);
+                if (lane == 0)
+                    ok = mbar_wait_impl<kRelaxedNs, CTAS == 2>(bar_cache_empty + 8 * ring.buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + ring.buf);
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                store_row_scale_images<KIND>(w, min(kUnitStages, (cur.t.k_len - cur.k0 + kStageElems - 1) / kStageElems),
+                                             smem_images + ring.buf * kCacheBufBytes, lane);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
+                __syncwarp();
+                // In the second CTA of a pair the arrival is forwarded to the leader by warp 2: the remote arrival
+                // stalls its issuing thread for about a thousand cycles, which this warp spends on the next unit.
+                if (lane == 0) mbar_arrive(bar_cache_full + 8 * ring.buf);
+                ring.next(kImageBufs);
+                cur.next(p, kUnitStages * kStageElems);
+                // the raw buffer just read is free: fetch the unit kRawBufs ahead into it
+                if (ahead.valid(p)) {
+                    issue_raw_scales(p, ahead.t, ahead.k0, smem_raw_scales + raw_read * kCacheBufBytes, lane);
+                    ahead.next(p, kUnitStages * kStageElems);
+                } else {
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                }
+                if (++raw_read == kRawBufs) raw_read = 0;
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+        }
+        for (int tile = first_tile; KIND == KIND_MXF4 && ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
             decode_tile(p, tile, rank, t);
-            for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, unit++) {
-                const int buf = unit & kBufMask;
+            for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, ring.next(kImageBufs)) {
+                const int buf = ring.buf;
                 uint8_t *images = smem_images + buf * kCacheBufBytes;
-                if (KIND != KIND_MXF4) {
-                    // per-row scales: from global memory into registers, and once the buffer is free into the images.
-                    // In a pair the buffer is released by the leader's multicast commit: probe (a suspended try_wait
-                    // is not reliably woken early by a remote arrival).
-                    uint32_t w[12][8];
-                    load_row_scales(p, t, k0, smem_compact, lane, w);
-                    if (lane == 0)
-                        ok = mbar_wait_impl<kRelaxedNs, CTAS == 2>(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
-                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-                    if (!ok) break;
-                    store_row_scale_images<KIND>(w, min(kUnitStages, (t.k_len - k0 + kStageElems - 1) / kStageElems), images, lane);
-                } else {
+                {
                     const int n_chunks = min(kCacheChunks, (((t.k_len - k0 + 127) >> 7) + 1) & ~1);   // whole stages; pad rows beyond the tensor
                     uint32_t *compact = reinterpret_cast<uint32_t *>(smem_compact);
                     build_scale_cache(p.sfa, t.a_row0 >> 5, ((t.a_k0 + k0) >> 5), n_chunks, 2, compact, lane);
                     build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
                     __syncwarp();
                     if (lane == 0)
-                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf)
-                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ((unit >> kBufShift) & 1u) ^ 1u, abort_flag, p.status, 0x500u + buf);
+                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + buf)
+                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + buf);
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     if (!ok) break;
                     const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
@@ -1063,9 +1244,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
-                // In the second CTA of a pair the arrival is forwarded to the leader by warp 2: the remote arrival
-                // stalls its issuing thread for about a thousand cycles, which this warp spends on the next unit.
-                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);
+                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);   // forwarded to the leader by warp 2 in a pair's second CTA
             }
         }
     } else if (warp == 2) {
@@ -1078,7 +1257,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // to its end.
         StageIter sg;
         sg.init(p, first_tile, tile_step, rank, kStageElems);
-        uint32_t stage = 0, phase = 0, acc_phase = 0, unit = 0;
+        uint32_t stage = 0, phase = 0, acc_phase = 0;
+        BufRing ring;   // image buffer of the current unit
         bool ok = true;
         TRACE_DECL(c_meet); TRACE_DECL(c_poll);
         TRACE_T0(tt);
@@ -1092,17 +1272,18 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             } else {
                 if (ok && lane == 0) {
                     if ((sg.it & (kUnitStages - 1)) == 0 && !unit_seen) {
-                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * (unit & kBufMask), (unit >> kBufShift) & 1u, abort_flag, p.status, 0x510u + (unit & kBufMask));
+                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * ring.buf, ring.phase, abort_flag, p.status, 0x510u + ring.buf);
                         if (ok && CTAS == 2)
-                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * (unit & kBufMask), (unit >> kBufShift) & 1u, abort_flag, p.status, 0x520u + (unit & kBufMask));
+                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * ring.buf, ring.phase, abort_flag, p.status, 0x520u + ring.buf);
                     }
                     if ((sg.it & (kUnitStages - 1)) == 0) unit_seen = false;
                     if (ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen) {
                         // second half of a unit: look whether the next unit's images are in place already, so that
                         // the unit boundary costs no extra probes on the critical path
-                        const uint32_t nu = unit + 1;
-                        unit_seen = mbar_test_wait(bar_cache_full + 8 * (nu & kBufMask), (nu >> kBufShift) & 1u) &&
-                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * (nu & kBufMask), (nu >> kBufShift) & 1u));
+                        BufRing nu = ring;
+                        nu.next(kImageBufs);
+                        unit_seen = mbar_test_wait(bar_cache_full + 8 * nu.buf, nu.phase) &&
+                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * nu.buf, nu.phase));
                     }
                     if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
                     if (ok) {
@@ -1151,7 +1332,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
             TRACE_ADD(c_meet, tt);
             if (sg.it == 0) acc_phase ^= 1u;
-            if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) unit++;
+            if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) ring.next(kImageBufs);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
             sg.next(p, kStageElems);
         }
@@ -1159,14 +1340,11 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             // Second CTA of a pair: report each unit of scale images the builder has finished to the leader, which
             // issues the scale copies of both CTAs.
             bool fwd_ok = true;
-            uint32_t u = 0;
-            for (int tile = first_tile; fwd_ok && tile < p.n_tile_total; tile += tile_step) {
-                Tile t;
-                decode_tile(p, tile, rank, t);
-                for (int k0 = 0; fwd_ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, u++) {
-                    fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * (u & kBufMask), (u >> kBufShift) & 1u, abort_flag, p.status, 0x530u + (u & kBufMask));
-                    if (fwd_ok) mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * (u & kBufMask), 0));
-                }
+            BufRing fr;
+            UnitIter un;
+            for (un.init(p, first_tile, tile_step, rank); fwd_ok && un.valid(p); un.next(p, kUnitStages * kStageElems), fr.next(kImageBufs)) {
+                fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * fr.buf, fr.phase, abort_flag, p.status, 0x530u + fr.buf);
+                if (fwd_ok) mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * fr.buf, 0));
             }
         }
         __syncwarp();
