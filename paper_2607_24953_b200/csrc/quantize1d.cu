@@ -35,8 +35,16 @@ __global__ void __launch_bounds__(256) quantize1d_kernel(const __grid_constant__
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t total = p.rows * p.segs_per_row;
     const bool active = gid < total;   // whole warps stay in the shuffle below (total is even, lanes pair up)
-    const int64_t i = active ? gid / p.segs_per_row : 0;
-    const int64_t seg = active ? gid % p.segs_per_row : 0;
+    int64_t i = 0, seg = 0;
+    if (active) {
+        if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
+            i = (uint32_t)gid / (uint32_t)p.segs_per_row;
+            seg = (uint32_t)gid - (uint32_t)i * (uint32_t)p.segs_per_row;
+        } else {
+            i = gid / p.segs_per_row;
+            seg = gid - i * p.segs_per_row;
+        }
+    }
     const int64_t j0 = seg * 16;
 
     uint32_t raw[8];
@@ -58,18 +66,30 @@ __global__ void __launch_bounds__(256) quantize1d_kernel(const __grid_constant__
             }
         }
     }
-    uint32_t fm = 0;
-    bool nonfinite = false;
+    // block maximum: packed BF16 |.| max with NaN propagation, so that any non-finite entry shows up in the
+    // result and routes the block to the scalar path
+    __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int k = 0; k < 8; k++) {
-        const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
-        nonfinite |= lo >= 0x7F80u || hi >= 0x7F80u;
-        if (lo < 0x7F80u && lo > fm) fm = lo;
-        if (hi < 0x7F80u && hi > fm) fm = hi;
+    for (int k = 0; k < 8; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
+    {
+        uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), 1);
+        m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
     }
-    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, 1);
-    fm = other > fm ? other : fm;
-    nonfinite |= __shfl_xor_sync(0xFFFFFFFFu, (int)nonfinite, 1) != 0;
+    const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
+    uint32_t fm = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
+    const bool nonfinite = fm >= 0x7F80u;
+    if (__any_sync(0xFFFFFFFFu, nonfinite)) {   // maximum over the finite entries only
+        uint32_t f = 0;
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
+            if (lo < 0x7F80u && lo > f) f = lo;
+            if (hi < 0x7F80u && hi > f) f = hi;
+        }
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, f, 1);
+        f = other > f ? other : f;
+        if (nonfinite) fm = f;
+    }
     const int code = scale_code_from_max(fm);
     if (!active) return;
     if ((seg & 1) == 0) p.scale[i * p.ld_s + (seg >> 1)] = (uint8_t)code;
@@ -101,34 +121,60 @@ __global__ void __launch_bounds__(128) quantize1d_t_kernel(const __grid_constant
     if (i0 >= p.rows || c0 >= p.cols) return;
     const bool two = c0 + 1 < p.cols;
     uint32_t raw[32];
+    if (p.x_vec_ok && two && i0 + 32 <= p.rows) {   // interior: 32 unconditional word loads, one address step each
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(p.x + i0 * p.ld_x + c0);
+        const int64_t step = p.ld_x >> 1;
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-        raw[r] = 0u;
-        if (i0 + r < p.rows) {
-            const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
-            if (p.x_vec_ok && two) raw[r] = __ldg(reinterpret_cast<const uint32_t *>(src));
-            else raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+        for (int r = 0; r < 32; r++) raw[r] = __ldg(src + r * step);
+    } else {
+#pragma unroll
+        for (int r = 0; r < 32; r++) {
+            raw[r] = 0u;
+            if (i0 + r < p.rows) {
+                const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
+                raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+            }
         }
     }
-    uint32_t m0 = 0, m1 = 0;
+    // both columns' maxima at once: packed |.| max with NaN propagation; a non-finite entry routes the lane to the
+    // careful path
+    __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-        const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
-        if (lo < 0x7F80u && lo > m0) m0 = lo;
-        if (hi < 0x7F80u && hi > m1) m1 = hi;
+    for (int r = 0; r < 32; r++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r])));
+    uint32_t m0 = *reinterpret_cast<const uint32_t *>(&m2) & 0x7FFFu, m1 = (*reinterpret_cast<const uint32_t *>(&m2) >> 16) & 0x7FFFu;
+    const bool nonfinite = m0 >= 0x7F80u || m1 >= 0x7F80u;
+    if (nonfinite) {
+        m0 = m1 = 0;
+#pragma unroll
+        for (int r = 0; r < 32; r++) {
+            const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
+            if (lo < 0x7F80u && lo > m0) m0 = lo;
+            if (hi < 0x7F80u && hi > m1) m1 = hi;
+        }
     }
     const int code0 = scale_code_from_max(m0), code1 = scale_code_from_max(m1);
     const float inv0 = inv_scale(code0), inv1 = inv_scale(code1);
-    uint32_t A[4] = {0u, 0u, 0u, 0u}, B[4] = {0u, 0u, 0u, 0u};   // the two columns' 32 nibbles
+    // One convert takes the same column of two consecutive rows: its result byte (row r in the low nibble, row r + 1
+    // in the high one) is a payload byte of that column as it stands.
+    uint32_t A[4], B[4];   // the two columns' 32 nibbles
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-        const uint32_t lo = raw[r] << 16, hi = raw[r] & 0xFFFF0000u;
-        // NaN -> +0; +-Inf saturates to +-6 in the conversion
-        const float v0 = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv0;
-        const float v1 = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv1;
-        const uint32_t res = cvt_rn_e2m1x2(v1, v0);   // nibble 0: column c0, nibble 1: column c0 + 1
-        A[r >> 3] |= (res & 0xFu) << (4 * (r & 7));
-        B[r >> 3] |= ((res >> 4) & 0xFu) << (4 * (r & 7));
+    for (int g = 0; g < 4; g++) {
+        uint32_t a = 0, b = 0;
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+            uint32_t w0 = raw[8 * g + 2 * e], w1 = raw[8 * g + 2 * e + 1];
+            uint32_t lo0 = w0 << 16, hi0 = w0 & 0xFFFF0000u, lo1 = w1 << 16, hi1 = w1 & 0xFFFF0000u;
+            if (nonfinite) {   // NaN -> +0; +-Inf saturates to +-6 in the conversion
+                if ((lo0 & 0x7FFFFFFFu) > 0x7F800000u) lo0 = 0u;
+                if ((hi0 & 0x7FFFFFFFu) > 0x7F800000u) hi0 = 0u;
+                if ((lo1 & 0x7FFFFFFFu) > 0x7F800000u) lo1 = 0u;
+                if ((hi1 & 0x7FFFFFFFu) > 0x7F800000u) hi1 = 0u;
+            }
+            a |= cvt_rn_e2m1x2(__uint_as_float(lo1) * inv0, __uint_as_float(lo0) * inv0) << (8 * e);
+            b |= cvt_rn_e2m1x2(__uint_as_float(hi1) * inv1, __uint_as_float(hi0) * inv1) << (8 * e);
+        }
+        A[g] = a;
+        B[g] = b;
     }
     *reinterpret_cast<uint4 *>(p.q + c0 * p.ld_q + (i0 >> 1)) = make_uint4(A[0], A[1], A[2], A[3]);
     p.scale[c0 * p.ld_s + rb] = (uint8_t)code0;
