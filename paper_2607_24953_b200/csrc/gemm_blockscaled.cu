@@ -1272,19 +1272,35 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             } else {
                 if (ok && lane == 0) {
                     if ((sg.it & (kUnitStages - 1)) == 0 && !unit_seen) {
-                        ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * ring.buf, ring.phase, abort_flag, p.status, 0x510u + ring.buf);
-                        if (ok && CTAS == 2)
-                            ok = mbar_wait_impl<0, true>(bar_peer_cache_full + 8 * ring.buf, ring.phase, abort_flag, p.status, 0x520u + ring.buf);
+                        // both CTAs' images of this unit: the two barriers probed together (the latencies overlap)
+                        const uint32_t b0 = bar_cache_full + 8 * ring.buf, b1 = (CTAS == 2 ? bar_peer_cache_full : bar_cache_full) + 8 * ring.buf;
+                        for (uint32_t spin = 0; ; spin++) {
+                            uint32_t q0, q1;
+                            asm volatile("{\n .reg .pred p0, p1;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p0, [%2], %4;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p1, [%3], %4;\n"
+                                         " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n}"
+                                         : "=r"(q0), "=r"(q1) : "r"(b0), "r"(b1), "r"(ring.phase) : "memory");
+                            if (q0 && q1) break;
+                            if (spin >= kWaitLimit) {
+                                ok = false;
+                                *abort_flag = 1u;
+                                if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = (q0 ? 0x520u : 0x510u) + ring.buf;
+                                break;
+                            }
+                            if ((spin & 255u) == 255u && *abort_flag) { ok = false; break; }
+                        }
                     }
                     if ((sg.it & (kUnitStages - 1)) == 0) unit_seen = false;
-                    if (ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen) {
-                        // second half of a unit: look whether the next unit's images are in place already, so that
-                        // the unit boundary costs no extra probes on the critical path
-                        BufRing nu = ring;
-                        nu.next(kImageBufs);
-                        unit_seen = mbar_test_wait(bar_cache_full + 8 * nu.buf, nu.phase) &&
-                                    (CTAS == 1 || mbar_test_wait(bar_peer_cache_full + 8 * nu.buf, nu.phase));
-                    }
+                    // Whether the next unit's images are in place is looked up ahead of time, so that a unit boundary
+                    // costs no extra probe on the critical path: with short units (per-row scales) the two barriers
+                    // ride along with every probe of the ring slots below; with 16-stage units one look in the second
+                    // half of the unit is enough, and the slot probes stay as light as they can be.
+                    BufRing nu = ring;
+                    nu.next(kImageBufs);
+                    const uint32_t nb0 = bar_cache_full + 8 * nu.buf, nb1 = (CTAS == 2 ? bar_peer_cache_full : bar_cache_full) + 8 * nu.buf;
+                    if (KIND == KIND_MXF4 && ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen)
+                        unit_seen = mbar_test_wait(nb0, nu.phase) && (CTAS == 1 || mbar_test_wait(nb1, nu.phase));
                     if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
                     if (ok) {
                         // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long
@@ -1300,17 +1316,32 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             sl[q] = sl[q - 1] + 1 == kStages ? 0u : sl[q - 1] + 1;
                             ph[q] = sl[q] == 0 ? ph[q - 1] ^ 1u : ph[q - 1];
                         }
-                        uint32_t r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+                        uint32_t r0 = 0, r1 = 0, r2 = 0, r3 = 0, r4 = 0, r5 = 0;
                         for (uint32_t spin = 0; ; spin++) {
-                            asm volatile("{\n .reg .pred p0, p1, p2, p3;\n"
-                                         " mbarrier.test_wait.parity.shared::cta.b64 p0, [%4], %5;\n"
-                                         " mbarrier.test_wait.parity.shared::cta.b64 p1, [%6], %7;\n"
-                                         " mbarrier.test_wait.parity.shared::cta.b64 p2, [%8], %9;\n"
-                                         " mbarrier.test_wait.parity.shared::cta.b64 p3, [%10], %11;\n"
-                                         " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n selp.b32 %2, 1, 0, p2;\n selp.b32 %3, 1, 0, p3;\n}"
-                                         : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                            if (KIND == KIND_MXF4)
+                                asm volatile("{\n .reg .pred p0, p1, p2, p3;\n"
+                                             " mbarrier.test_wait.parity.shared::cta.b64 p0, [%4], %5;\n"
+                                             " mbarrier.test_wait.parity.shared::cta.b64 p1, [%6], %7;\n"
+                                             " mbarrier.test_wait.parity.shared::cta.b64 p2, [%8], %9;\n"
+                                             " mbarrier.test_wait.parity.shared::cta.b64 p3, [%10], %11;\n"
+                                             " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n selp.b32 %2, 1, 0, p2;\n selp.b32 %3, 1, 0, p3;\n}"
+                                             : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                                             : "r"(bar_full + 8 * sl[0]), "r"(ph[0]), "r"(bar_full + 8 * sl[1]), "r"(ph[1]),
+                                               "r"(bar_full + 8 * sl[2]), "r"(ph[2]), "r"(bar_full + 8 * sl[3]), "r"(ph[3]) : "memory");
+                            else
+                            asm volatile("{\n .reg .pred p0, p1, p2, p3, p4, p5;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p0, [%6], %7;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p1, [%8], %9;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p2, [%10], %11;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p3, [%12], %13;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p4, [%14], %16;\n"
+                                         " mbarrier.test_wait.parity.shared::cta.b64 p5, [%15], %16;\n"
+                                         " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n selp.b32 %2, 1, 0, p2;\n selp.b32 %3, 1, 0, p3;\n"
+                                         " selp.b32 %4, 1, 0, p4;\n selp.b32 %5, 1, 0, p5;\n}"
+                                         : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3), "=r"(r4), "=r"(r5)
                                          : "r"(bar_full + 8 * sl[0]), "r"(ph[0]), "r"(bar_full + 8 * sl[1]), "r"(ph[1]),
-                                           "r"(bar_full + 8 * sl[2]), "r"(ph[2]), "r"(bar_full + 8 * sl[3]), "r"(ph[3]) : "memory");
+                                           "r"(bar_full + 8 * sl[2]), "r"(ph[2]), "r"(bar_full + 8 * sl[3]), "r"(ph[3]),
+                                           "r"(nb0), "r"(nb1), "r"(nu.phase) : "memory");
                             if (r0) break;
                             if (spin >= kWaitLimit) {
                                 ok = false;
@@ -1321,6 +1352,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             if ((spin & 255u) == 255u && *abort_flag) { ok = false; break; }
                         }
                         ahead = !ok ? 0u : (left >= 1 && r1) ? ((left >= 2 && r2) ? ((left >= 3 && r3) ? 3u : 2u) : 1u) : 0u;
+                        if (r4 && r5) unit_seen = true;
                     }
                 }
                 ahead = __shfl_sync(0xFFFFFFFFu, ahead, 0);
