@@ -2,6 +2,8 @@
 // elements of a row), the operand format of the query/key projections.  Streaming kernel: each
 // thread owns 16 consecutive elements (two 128-bit loads, one 128-bit store); two neighbouring
 // lanes own one 32-element block and exchange their maxima with one shuffle.
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace fp4q {
@@ -104,21 +106,36 @@ __global__ void __launch_bounds__(128) mxfp8_quantize1d_t_kernel(const __grid_co
     if (i0 >= p.rows || c0 >= p.cols) return;
     const bool two = c0 + 1 < p.cols;
     uint32_t raw[32];
+    if (p.x_vec_ok && two && i0 + 32 <= p.rows) {   // interior: 32 unconditional word loads, one address step each
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(p.x + i0 * p.ld_x + c0);
+        const int64_t step = p.ld_x >> 1;
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-        raw[r] = 0u;
-        if (i0 + r < p.rows) {
-            const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
-            if (p.x_vec_ok && two) raw[r] = __ldg(reinterpret_cast<const uint32_t *>(src));
-            else raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+        for (int r = 0; r < 32; r++) raw[r] = __ldg(src + r * step);
+    } else {
+#pragma unroll
+        for (int r = 0; r < 32; r++) {
+            raw[r] = 0u;
+            if (i0 + r < p.rows) {
+                const uint16_t *src = p.x + (i0 + r) * p.ld_x + c0;
+                raw[r] = (uint32_t)__ldg(src) | (two ? (uint32_t)__ldg(src + 1) << 16 : 0u);
+            }
         }
     }
-    uint32_t m0 = 0, m1 = 0;   // maxima over finite magnitudes
+    // both columns' maxima at once: packed |.| max with NaN propagation; a non-finite entry routes the lane to the
+    // careful path (maxima over finite magnitudes, NaN -> +0)
+    __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-        const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
-        if (lo < 0x7F80u && lo > m0) m0 = lo;
-        if (hi < 0x7F80u && hi > m1) m1 = hi;
+    for (int r = 0; r < 32; r++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r])));
+    uint32_t m0 = *reinterpret_cast<const uint32_t *>(&m2) & 0x7FFFu, m1 = (*reinterpret_cast<const uint32_t *>(&m2) >> 16) & 0x7FFFu;
+    const bool nonfinite = m0 >= 0x7F80u || m1 >= 0x7F80u;
+    if (nonfinite) {
+        m0 = m1 = 0;
+#pragma unroll
+        for (int r = 0; r < 32; r++) {
+            const uint32_t lo = raw[r] & 0x7FFFu, hi = (raw[r] >> 16) & 0x7FFFu;
+            if (lo < 0x7F80u && lo > m0) m0 = lo;
+            if (hi < 0x7F80u && hi > m1) m1 = hi;
+        }
     }
     int code[2];
     float inv[2];
@@ -130,21 +147,27 @@ __global__ void __launch_bounds__(128) mxfp8_quantize1d_t_kernel(const __grid_co
         code[k] = c < 0 ? 0 : c;
         inv[k] = __uint_as_float((uint32_t)(254 - code[k]) << 23);
     }
+    // One convert takes the same column of two consecutive rows: its two result bytes are consecutive payload bytes
+    // of that column.  +-Inf saturates to +-448 in the conversion.
     uint32_t A[8], B[8];   // the two columns' 32 payload bytes
 #pragma unroll
     for (int w = 0; w < 8; w++) {
-        uint32_t res[4];
+        uint32_t a = 0, b = 0;
 #pragma unroll
-        for (int k = 0; k < 4; k++) {
-            const uint32_t word = raw[4 * w + k];
-            const uint32_t lo = word << 16, hi = word & 0xFFFF0000u;
-            const float v0 = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv[0];
-            const float v1 = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv[1];
-            res[k] = cvt_rn_e4m3x2(v1, v0);   // byte 0: column c0, byte 1: column c0 + 1
+        for (int e = 0; e < 2; e++) {
+            const uint32_t w0 = raw[4 * w + 2 * e], w1 = raw[4 * w + 2 * e + 1];
+            uint32_t lo0 = w0 << 16, hi0 = w0 & 0xFFFF0000u, lo1 = w1 << 16, hi1 = w1 & 0xFFFF0000u;
+            if (nonfinite) {
+                if ((lo0 & 0x7FFFFFFFu) > 0x7F800000u) lo0 = 0u;
+                if ((hi0 & 0x7FFFFFFFu) > 0x7F800000u) hi0 = 0u;
+                if ((lo1 & 0x7FFFFFFFu) > 0x7F800000u) lo1 = 0u;
+                if ((hi1 & 0x7FFFFFFFu) > 0x7F800000u) hi1 = 0u;
+            }
+            a |= cvt_rn_e4m3x2(__uint_as_float(lo1) * inv[0], __uint_as_float(lo0) * inv[0]) << (16 * e);
+            b |= cvt_rn_e4m3x2(__uint_as_float(hi1) * inv[1], __uint_as_float(hi0) * inv[1]) << (16 * e);
         }
-        const uint32_t t01 = res[0] | (res[1] << 16), t23 = res[2] | (res[3] << 16);
-        A[w] = __byte_perm(t01, t23, 0x6420);
-        B[w] = __byte_perm(t01, t23, 0x7531);
+        A[w] = a;
+        B[w] = b;
     }
     uint8_t *dst = p.q + c0 * p.ld_q + i0;
     reinterpret_cast<uint4 *>(dst)[0] = make_uint4(A[0], A[1], A[2], A[3]);
