@@ -262,6 +262,18 @@ fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, 
                                     void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * fp4q_gemm_dgrad_quantized -- the dense input-gradient product with the same fused epilogue: dX = dY^ W^ with FP32
+ * accumulation, rounded to BF16, then dXq = 2D-block FP4 of dX exactly as fp4q_quantize2d computes it (element index
+ * i*K + j): the layer's dX is the previous layer's dY, which the backward pass quantizes with stochastic rounding
+ * (Section 3.1), so that quantization can happen here and dX never reaches memory in BF16.
+ * dY [T,N] (row-major payload used), W [N,K] (transposed payload used) as for fp4q_gemm_dgrad (dense form).
+ * dXq: rows = T, cols = K (multiple of 16), otherwise as Yq of fp4q_gemm_fwd_quantized; errors as there.
+ */
+fp4q_status fp4q_gemm_dgrad_quantized(const fp4q_tensor *dY, const fp4q_tensor *W, const fp4q_tensor *dXq,
+                                      fp4q_round mode, uint64_t seed, uint32_t tensor_id,
+                                      void *ws, size_t ws_bytes, void *stream);
+
+/*
  * fp4q_gemm_fwd_static_workspace -- no counterpart in the paper: the dense forward product of
  * fp4q_gemm_fwd for callers that cannot allocate device memory (code living inside an application that
  * owns the device heap, a loop that must stay out of the allocator, a sandbox restricted to buffers it was

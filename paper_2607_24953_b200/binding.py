@@ -102,6 +102,9 @@ def lib() -> ctypes.CDLL:
             L.fp4q_mxfp8_gemm.restype = ci
             L.fp4q_mxfp8_gemm.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp, i64, i64, i64, vp, i64, ci, vp,
                                           ctypes.c_size_t, vp]
+        if hasattr(L, "fp4q_gemm_dgrad_quantized"):
+            L.fp4q_gemm_dgrad_quantized.restype = ci
+            L.fp4q_gemm_dgrad_quantized.argtypes = [vp, vp, vp, ci, u64, u32, vp, ctypes.c_size_t, vp]
         if hasattr(L, "fp4q_gemm_fwd_quantized"):
             L.fp4q_gemm_fwd_quantized.restype = ci
             L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
@@ -355,6 +358,21 @@ def fp4q_gemm_fwd_quantized(X: QTensor, W: QTensor, out: Optional[QTensor] = Non
     st = lib().fp4q_gemm_fwd_quantized(ctypes.byref(cx), ctypes.byref(cw), ctypes.byref(cy), mode, seed, tensor_id,
                                        ws.data_ptr(), ws.numel(), _stream(stream))
     _check(st, "fp4q_gemm_fwd_quantized")
+    return out
+
+
+def fp4q_gemm_dgrad_quantized(dY: QTensor, W: QTensor, out: Optional[QTensor] = None, mode: int = ROUND_STOCHASTIC,
+                              seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None) -> QTensor:
+    """dXq = 2D-block FP4 of the BF16-rounded product dY^ W^, quantized in the GEMM's epilogue."""
+    dev = dY.q_rm.device
+    if out is None:
+        out = alloc_qtensor(dY.rows, W.cols, dev, want_t)
+    if ws is None:
+        ws = alloc_workspace(dev)
+    cd, cw, cx = dY.c_struct(), W.c_struct(), out.c_struct()
+    st = lib().fp4q_gemm_dgrad_quantized(ctypes.byref(cd), ctypes.byref(cw), ctypes.byref(cx), mode, seed, tensor_id,
+                                         ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "fp4q_gemm_dgrad_quantized")
     return out
 
 

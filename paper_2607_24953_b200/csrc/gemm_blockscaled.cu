@@ -1786,37 +1786,50 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
     return launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, ws_bytes, stream);
 }
 
+// C[M, N] = A B^T with the output leaving as the 2D-block FP4 tensor Cq (dense, pair kernel).
+static fp4q_status launch_gemm_quantized(const Operand &A, const Operand &B, int64_t M, int64_t N, int64_t K, const fp4q_tensor *Cq,
+                                         fp4q_round mode, uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+{
+    if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
+    if (Cq->rows != M || Cq->cols != N) return FP4Q_ERR_SHAPE;
+    if (M > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (N % 16 != 0) return FP4Q_ERR_UNSUPPORTED;   // one Philox block per 16-element row segment of the output
+    if (M == 0 || N == 0) return FP4Q_OK;
+    if (!A.payload || !B.payload || !A.sf.ptr || !B.sf.ptr || !Cq->q_rm || !Cq->scale) return FP4Q_ERR_NULL;
+    if (Cq->ld_rm < round_up(N, 32) / 2 || Cq->ld_s < ceil_div(N, 32)) return FP4Q_ERR_SHAPE;
+    if (Cq->q_t && Cq->ld_t < round_up(M, 32) / 2) return FP4Q_ERR_SHAPE;
+    if (!aligned(Cq->q_rm, 16) || Cq->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
+    if (Cq->q_t && (!aligned(Cq->q_t, 16) || Cq->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
+    if (!ws || ws_bytes < sizeof(Workspace)) return FP4Q_ERR_WORKSPACE;
+    if (!aligned(ws, 256)) return FP4Q_ERR_ALIGN;
+    if (!aligned(A.payload, 16) || !aligned(B.payload, 16) || A.ld_bytes % 16 || B.ld_bytes % 16) return FP4Q_ERR_ALIGN;
+    GemmParams p = {};
+    p.M = (int32_t)M; p.N = (int32_t)N; p.K = (int32_t)K;
+    dense_tiles(p);
+    p.sfa = A.sf; p.sfb = B.sf;
+    p.status = reinterpret_cast<uint32_t *>(ws);
+    p.q_rm = Cq->q_rm; p.q_ld_rm = Cq->ld_rm;
+    p.q_t = Cq->q_t; p.q_ld_t = Cq->ld_t;
+    p.q_scale = Cq->scale; p.q_ld_s = Cq->ld_s;
+    p.q_mode = (int32_t)mode; p.q_tensor_id = tensor_id;
+    philox_round_keys(seed, p.q_keys);
+    return launch_gemm_impl<KIND_MXF4, 2, EPI_QUANT>(A, B, p, stream);
+}
+
 extern "C" fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, const fp4q_tensor *Yq, fp4q_round mode,
                                                uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
 {
     if (!tensor_ok(X) || !tensor_ok(W) || !tensor_ok(Yq)) return X && W && Yq ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
-    if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
     if (X->cols != W->cols) return FP4Q_ERR_SHAPE;
-    const int64_t T = X->rows, K = X->cols, N = W->rows;
-    if (Yq->rows != T || Yq->cols != N) return FP4Q_ERR_SHAPE;
-    if (T > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
-    if (N % 16 != 0) return FP4Q_ERR_UNSUPPORTED;   // one Philox block per 16-element row segment of the output
-    if (T == 0 || N == 0) return FP4Q_OK;
-    if (!X->q_rm || !W->q_rm || !X->scale || !W->scale || !Yq->q_rm || !Yq->scale) return FP4Q_ERR_NULL;
-    if (Yq->ld_rm < round_up(N, 32) / 2 || Yq->ld_s < ceil_div(N, 32)) return FP4Q_ERR_SHAPE;
-    if (Yq->q_t && Yq->ld_t < round_up(T, 32) / 2) return FP4Q_ERR_SHAPE;
-    if (!aligned(Yq->q_rm, 16) || Yq->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
-    if (Yq->q_t && (!aligned(Yq->q_t, 16) || Yq->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
-    if (!ws || ws_bytes < sizeof(Workspace)) return FP4Q_ERR_WORKSPACE;
-    if (!aligned(ws, 256)) return FP4Q_ERR_ALIGN;
-    const Operand A = operand_rm(X), B = operand_rm(W);
-    if (!aligned(A.payload, 16) || !aligned(B.payload, 16) || A.ld_bytes % 16 || B.ld_bytes % 16) return FP4Q_ERR_ALIGN;
-    GemmParams p = {};
-    p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)K;
-    dense_tiles(p);
-    p.sfa = A.sf; p.sfb = B.sf;
-    p.status = reinterpret_cast<uint32_t *>(ws);
-    p.q_rm = Yq->q_rm; p.q_ld_rm = Yq->ld_rm;
-    p.q_t = Yq->q_t; p.q_ld_t = Yq->ld_t;
-    p.q_scale = Yq->scale; p.q_ld_s = Yq->ld_s;
-    p.q_mode = (int32_t)mode; p.q_tensor_id = tensor_id;
-    philox_round_keys(seed, p.q_keys);
-    return launch_gemm_impl<KIND_MXF4, 2, EPI_QUANT>(A, B, p, stream);
+    return launch_gemm_quantized(operand_rm(X), operand_rm(W), X->rows, W->rows, X->cols, Yq, mode, seed, tensor_id, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_dgrad_quantized(const fp4q_tensor *dY, const fp4q_tensor *W, const fp4q_tensor *dXq, fp4q_round mode,
+                                                 uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(dY) || !tensor_ok(W) || !tensor_ok(dXq)) return dY && W && dXq ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (dY->cols != W->rows) return FP4Q_ERR_SHAPE;
+    return launch_gemm_quantized(operand_rm(dY), operand_t(W), dY->rows, W->cols, dY->cols, dXq, mode, seed, tensor_id, ws, ws_bytes, stream);
 }
 
 extern "C" fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt,

@@ -77,3 +77,44 @@ def test_output_width_must_be_a_multiple_of_16():
     qx, qw = binding.fp4q_quantize2d(X), binding.fp4q_quantize2d(W)
     with pytest.raises(binding.Fp4qError):
         binding.fp4q_gemm_fwd_quantized(qx, qw)
+
+
+@pytest.mark.parametrize("T,N,K", [(256, 256, 256), (300, 1000, 272), (1000, 320, 1040), (97, 64, 48)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_fused_dgrad_equals_product_then_quantize(T, N, K, mode):
+    """dX = dY^ W^ quantized in the epilogue (the previous layer's dY) against fp4q_gemm_dgrad + fp4q_quantize2d."""
+    dY = workloads.gradients_rowscaled(T, N, 710, "cuda")
+    W = workloads.weights(N, K, 711, "cuda")
+    qdy = binding.fp4q_quantize2d(dY, mode=1, seed=2, tensor_id=5)
+    qw = binding.fp4q_quantize2d(W, mode=0)
+    ws = binding.alloc_workspace("cuda")
+    fused = binding.fp4q_gemm_dgrad_quantized(qdy, qw, mode=mode, seed=3, tensor_id=8, ws=ws)
+    dx = binding.fp4q_gemm_dgrad(qdy, qw, dt=binding.OUT_BF16, ws=ws)
+    chain = binding.fp4q_quantize2d(dx.contiguous(), mode=mode, seed=3, tensor_id=8)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    c_rm, c_t, c_s = logical(chain)
+    compare_logical(fused, c_rm, c_t, c_s, T, K)
+
+
+def test_fused_dgrad_exact_operands_match_the_oracle_bit_for_bit():
+    g = torch.Generator(device="cuda").manual_seed(6)
+    grid = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6], device="cuda")
+
+    def draw(r, c, e):
+        v = grid[torch.randint(0, 8, (r, c), generator=g, device="cuda")]
+        s = torch.randint(0, 2, (r, c), generator=g, device="cuda") * 2 - 1
+        return (v * s * 2.0 ** e).to(torch.bfloat16)
+
+    T, N, K = 200, 512, 400
+    dY, W = draw(T, N, -9), draw(N, K, 4)
+    qdy = assert_matches_oracle(dY, 0, seed=0, tensor_id=0)
+    qw = assert_matches_oracle(W, 0, seed=0, tensor_id=1)
+    ws = binding.alloc_workspace("cuda")
+    dxq = binding.fp4q_gemm_dgrad_quantized(qdy, qw, mode=oracle.MODE_STOCHASTIC, seed=9, tensor_id=4, ws=ws)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    dx = oracle.bf16_round(oracle.gemm_dgrad(dequant_from_gpu(qdy), dequant_from_gpu(qw)))
+    dx_bits = workloads.bf16_bits(torch.from_numpy(dx).to(torch.bfloat16))
+    o_rm, o_t, o_s = oracle.quantize2d(dx_bits, oracle.MODE_STOCHASTIC, 9, 4)
+    compare_logical(dxq, o_rm, o_t, o_s, T, K)
