@@ -69,6 +69,11 @@ def lib() -> ctypes.CDLL:
                                             i64, i64, i64, i64, u8p, i64, u8p, i64, u8p, i64]
         L.orc_dequantize2d.restype = None
         L.orc_dequantize2d.argtypes = [u8p, i64, u8p, i64, i64, i64, u8p, i64]
+        L.orc_quantize2d_block.restype = ctypes.c_int
+        L.orc_quantize2d_block.argtypes = [u8p, i64, i64, i64, ctypes.c_int, ctypes.c_int, u64, u32, u32, u8p, i64, u8p, i64,
+                                           u8p, i64]
+        L.orc_dequantize2d_block.restype = None
+        L.orc_dequantize2d_block.argtypes = [u8p, i64, u8p, i64, ctypes.c_int, i64, i64, u8p, i64]
         L.orc_quantize1d.restype = ctypes.c_int
         L.orc_quantize1d.argtypes = [u8p, i64, i64, i64, ctypes.c_int, u64, u32, u32, u8p, i64, u8p, i64]
         L.orc_dequantize1d.restype = None
@@ -180,6 +185,32 @@ def dequantize2d(q_rm, scale, rows, cols):
     out = np.zeros((rows, cols), dtype=np.float64)
     if rows and cols:
         lib().orc_dequantize2d(_ptr(q), q.shape[1], _ptr(s), s.shape[1], rows, cols, _ptr(out), cols)
+    return out
+
+
+def quantize2d_block(x_bits, block, mode=MODE_NEAREST, seed=0, tensor_id=0, flags=0, want_t=True):
+    """The 2D scheme with b x b blocks (block-size study, Table 4).  Returns (q_rm, q_t or None,
+    scale [ceil(rows/b), ceil(cols/b)]) as uint8."""
+    x = _as_bf16_bits(x_bits)
+    rows, cols = x.shape
+    q_rm = np.zeros((rows, (cols + 1) // 2), dtype=np.uint8)
+    q_t = np.zeros((cols, (rows + 1) // 2), dtype=np.uint8) if want_t else None
+    scale = np.zeros((-(-rows // block), -(-cols // block)), dtype=np.uint8)
+    if rows and cols:
+        rc = lib().orc_quantize2d_block(_ptr(x), rows, cols, cols, int(block), int(mode), seed, tensor_id, flags,
+                                        _ptr(q_rm), q_rm.shape[1], _ptr(q_t) if want_t else None,
+                                        q_t.shape[1] if want_t else 0, _ptr(scale), scale.shape[1])
+        if rc != 0:
+            raise ValueError("orc_quantize2d_block rejected its arguments")
+    return q_rm, q_t, scale
+
+
+def dequantize2d_block(q_rm, scale, block, rows, cols):
+    q = np.ascontiguousarray(q_rm, dtype=np.uint8)
+    s = np.ascontiguousarray(scale, dtype=np.uint8)
+    out = np.zeros((rows, cols), dtype=np.float64)
+    if rows and cols:
+        lib().orc_dequantize2d_block(_ptr(q), q.shape[1], _ptr(s), s.shape[1], int(block), rows, cols, _ptr(out), cols)
     return out
 
 

@@ -298,6 +298,83 @@ void orc_dequantize2d(const uint8_t *q_rm, int64_t ld_rm, const uint8_t *scale, 
     }
 }
 
+/* ------------------------------------------------------- block-size variants (b x b, b free) */
+
+/*
+ * The 2D scheme with another block size (the block-size study, Table 4: 8 / 16 / 32 / 64): the matrix is cut into
+ * b x b blocks, each with one truncation-free power-of-two scale; everything else as orc_quantize2d (E2M1 codes,
+ * nearest-even or stochastic rounding with the random byte of the element's index, +-Inf -> +-6, NaN -> +0, block
+ * maximum over finite entries, out-of-range entries excluded).  scale[ceil(rows/b), ld_s >= ceil(cols/b)].
+ * q_rm[rows, ld_rm >= ceil(cols/2)], q_t[cols, ld_t >= ceil(rows/2)] or NULL; payload rows are cleared first.
+ */
+int orc_quantize2d_block(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld_x, int block, int mode, uint64_t seed,
+                         uint32_t tensor_id, uint32_t flags, uint8_t *q_rm, int64_t ld_rm, uint8_t *q_t, int64_t ld_t,
+                         uint8_t *scale, int64_t ld_s)
+{
+    int64_t rt, ct, I, i;
+    if (block < 1 || rows < 0 || cols < 0 || (mode != ORC_MODE_NEAREST && mode != ORC_MODE_STOCHASTIC)) return -1;
+    if (rows == 0 || cols == 0) return 0;
+    rt = (rows + block - 1) / block;
+    ct = (cols + block - 1) / block;
+    if (!x || !q_rm || !scale || ld_x < cols || ld_rm < (cols + 1) / 2 || ld_s < ct) return -1;
+    if (q_t && ld_t < (rows + 1) / 2) return -1;
+    for (i = 0; i < rows; i++) memset(q_rm + i * ld_rm, 0, (size_t)ld_rm);
+    if (q_t)
+        for (i = 0; i < cols; i++) memset(q_t + i * ld_t, 0, (size_t)ld_t);
+    for (I = 0; I < rt; I++) {
+        int64_t J;
+        for (J = 0; J < ct; J++) {
+            int64_t i0 = I * block, j0 = J * block, j;
+            int64_t i1 = i0 + block < rows ? i0 + block : rows, j1 = j0 + block < cols ? j0 + block : cols;
+            double M = 0.0, S;
+            int e;
+            for (i = i0; i < i1; i++)
+                for (j = j0; j < j1; j++) {
+                    double a = fabs(orc_bf16_to_double(x[i * ld_x + j]));
+                    if (isfinite(a) && a > M) M = a;
+                }
+            e = orc_scale_exponent(M);
+            S = ldexp(1.0, e);
+            scale[I * ld_s + J] = (uint8_t)(e + 127);
+            for (i = i0; i < i1; i++)
+                for (j = j0; j < j1; j++) {
+                    uint16_t bits = x[i * ld_x + j];
+                    double a = orc_bf16_to_double(bits);
+                    int sign = (bits >> 15) & 1, mag, code;
+                    if (isnan(a)) {
+                        code = 0;
+                    } else {
+                        if (isinf(a)) {
+                            mag = 7;
+                        } else if (mode == ORC_MODE_NEAREST) {
+                            mag = orc_round_nearest(fabs(a) / S);
+                        } else {
+                            uint64_t idx = (flags & ORC_FLAG_INDEX_TRANSPOSED) ? (uint64_t)j * (uint64_t)rows + (uint64_t)i
+                                                                               : (uint64_t)i * (uint64_t)cols + (uint64_t)j;
+                            mag = orc_round_stochastic(fabs(a) / S, orc_random_byte(seed, tensor_id, idx));
+                        }
+                        code = (sign << 3) | mag;
+                    }
+                    orc_put_nibble(q_rm + i * ld_rm, j, code);
+                    if (q_t) orc_put_nibble(q_t + j * ld_t, i, code);
+                }
+        }
+    }
+    return 0;
+}
+
+/* Dequantized values of a b x b block tensor (row-major payload), exact in double. */
+void orc_dequantize2d_block(const uint8_t *q_rm, int64_t ld_rm, const uint8_t *scale, int64_t ld_s, int block,
+                            int64_t rows, int64_t cols, double *out, int64_t ld_out)
+{
+    int64_t i, j;
+    for (i = 0; i < rows; i++)
+        for (j = 0; j < cols; j++) {
+            int e = (int)scale[(i / block) * ld_s + j / block] - 127;
+            out[i * ld_out + j] = ldexp(orc_e2m1_value(orc_get_nibble(q_rm + i * ld_rm, j)), e);
+        }
+}
+
 /* ------------------------------------------------------- 1D (1 x 32) FP4 blocks */
 
 /*
