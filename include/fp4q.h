@@ -54,6 +54,12 @@ typedef enum { FP4Q_OUT_BF16 = 0, FP4Q_OUT_F32 = 1 } fp4q_out;
  * TRANSPOSED tensor (j*rows + i instead of i*cols + j), so that quantize(A^T) with this flag
  * reproduces quantize(A) transposed bit for bit. */
 #define FP4Q_INDEX_TRANSPOSED 1u
+/* Block-size study (Table 4 of the paper): quantize with 16 x 16 or 64 x 64 blocks instead of 32 x 32.
+ * FP4Q_BLOCK_64: the scale matrix keeps its 32-granular shape, each block's scale written to its four entries, so the
+ *   tensor is a valid operand of every GEMM entry point (the hardware's scale vectors are 32 wide).
+ * FP4Q_BLOCK_16: scale is [ceil(rows/16), ld_s >= ceil(cols/16)]; such a tensor cannot be passed to the GEMMs. */
+#define FP4Q_BLOCK_16 2u
+#define FP4Q_BLOCK_64 4u
 
 /*
  * A 2D-block-quantized tensor with logical source shape [rows, cols] (Section 3; appendix

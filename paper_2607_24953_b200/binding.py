@@ -22,6 +22,8 @@ ROUND_STOCHASTIC = 1
 OUT_BF16 = 0
 OUT_F32 = 1
 INDEX_TRANSPOSED = 1
+BLOCK_16 = 2   # fp4q_quantize2d flags: 16 x 16 or 64 x 64 blocks instead of 32 x 32 (block-size study)
+BLOCK_64 = 4
 
 EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgrad",
            "fp4q_mxfp8_quantize1d", "fp4q_mxfp8_qk", "fp4q_workspace_bytes", "fp4q_workspace_status",
@@ -141,9 +143,12 @@ class QTensor:
     cols: int
     q_rm: torch.Tensor               # uint8 [rows, ld_rm]
     q_t: Optional[torch.Tensor]      # uint8 [cols, ld_t] or None
-    scale: torch.Tensor              # uint8 [ceil(rows/32), ld_s]
+    scale: torch.Tensor              # uint8 [ceil(rows/32), ld_s] ([ceil(rows/16), ld_s] after BLOCK_16)
+    scale_granularity: int = 32      # 16 only for tensors quantized with BLOCK_16, which the GEMMs cannot take
 
     def c_struct(self) -> _CTensor:
+        if self.scale_granularity != 32 and not getattr(self, "_quantizing", False):
+            raise ValueError("a tensor quantized in 16 x 16 blocks is not a GEMM operand (the hardware's scale vectors are 32 wide)")
         return _CTensor(self.rows, self.cols,
                         self.q_rm.data_ptr(), self.q_rm.stride(0),
                         self.q_t.data_ptr() if self.q_t is not None else None,
@@ -155,14 +160,15 @@ def _pad16(n: int) -> int:
     return (n + 15) // 16 * 16
 
 
-def alloc_qtensor(rows: int, cols: int, device, want_t: bool = True) -> QTensor:
+def alloc_qtensor(rows: int, cols: int, device, want_t: bool = True, scale_granularity: int = 32) -> QTensor:
     """Allocate the output buffers of fp4q_quantize2d with the leading dimensions the ABI asks for."""
     ld_rm = max(_pad16((cols + 31) // 32 * 16), 16)
     ld_t = max(_pad16((rows + 31) // 32 * 16), 16)
     q_rm = torch.empty((rows, ld_rm), dtype=torch.uint8, device=device)
     q_t = torch.empty((cols, ld_t), dtype=torch.uint8, device=device) if want_t else None
-    scale = torch.empty(((rows + 31) // 32, max((cols + 31) // 32, 1)), dtype=torch.uint8, device=device)
-    return QTensor(rows, cols, q_rm, q_t, scale)
+    g = scale_granularity
+    scale = torch.empty(((rows + g - 1) // g, max((cols + g - 1) // g, 1)), dtype=torch.uint8, device=device)
+    return QTensor(rows, cols, q_rm, q_t, scale, g)
 
 
 def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = ROUND_NEAREST, seed: int = 0,
@@ -173,8 +179,12 @@ def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = 
         raise ValueError("x must be a 2-D BF16 tensor with contiguous rows")
     rows, cols = x.shape
     if out is None:
-        out = alloc_qtensor(rows, cols, x.device, want_t)
-    cs = out.c_struct()
+        out = alloc_qtensor(rows, cols, x.device, want_t, 16 if flags & BLOCK_16 else 32)
+    out._quantizing = True
+    try:
+        cs = out.c_struct()
+    finally:
+        out._quantizing = False
     st = lib().fp4q_quantize2d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, ctypes.byref(cs),
                                mode, seed, tensor_id, flags, _stream(stream))
     _check(st, "fp4q_quantize2d")

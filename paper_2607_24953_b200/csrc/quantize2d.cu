@@ -133,8 +133,12 @@ __device__ __forceinline__ void segment_random_bytes(const Quant2dParams &p, int
 
 // FAST = the CTA's 128x128 tile lies fully inside the tensor, rows are 32-byte aligned (256-bit loads) and
 // one Philox block covers each 16-element segment: no per-row bounds or path checks remain in the hot loop.
-template <int MODE, bool FAST>
-__device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_stage, uint4 *rnd_stage)
+// BLK = block size: 32 (the method), or 16 / 64 for the block-size study.  A 16x16 block is two lanes (8 rows x 16
+// columns each), a 64x64 block sixteen lanes in each of two neighbouring warps, which exchange their maxima through
+// `xchg`.  With BLK = 64 the scale is still written once per 32x32 tile (four equal entries per block), so that the
+// tensor feeds the GEMMs as it stands; with BLK = 16 the scale matrix has one entry per 16x16 block.
+template <int MODE, bool FAST, int BLK>
+__device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_stage, uint4 *rnd_stage, uint32_t *xchg)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = lane >> 3;          // which of the warp's four 32x32 blocks
@@ -181,16 +185,45 @@ __device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_
 #pragma unroll
         for (int k = 0; k < 8; k++)
             m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r][k])));
+    constexpr int kShflLo = BLK == 16 ? 2 : 1, kShflHi = BLK == 16 ? 2 : BLK == 32 ? 4 : 8;   // lanes of one block
 #pragma unroll
-    for (int s = 1; s <= 4; s <<= 1) {
+    for (int s = kShflLo; s <= kShflHi; s <<= 1) {
         uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), s);
         m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
     }
     const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
     uint32_t mbits = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
+    bool nonfinite64 = false;
+    if (BLK == 64) {
+        // the other 32 rows of the block belong to the neighbouring warp: both maxima (with NaN propagation, and over
+        // finite entries only) cross through shared memory, unconditionally, so that every thread reaches the barrier
+        uint32_t fm = 0;
+#pragma unroll
+        for (int r = 0; r < 8; r++)
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint32_t lo = raw[r][k] & 0x7FFFu, hi = (raw[r][k] >> 16) & 0x7FFFu;
+                if (lo < 0x7F80u && lo > fm) fm = lo;
+                if (hi < 0x7F80u && hi > fm) fm = hi;
+            }
+#pragma unroll
+        for (int s = 1; s <= 8; s <<= 1) {
+            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, s);
+            fm = other > fm ? other : fm;
+        }
+        if ((lane & 15) == 0) {
+            xchg[(warp * 2 + (t >> 1)) * 2] = mbits;
+            xchg[(warp * 2 + (t >> 1)) * 2 + 1] = fm;
+        }
+        __syncthreads();
+        const uint32_t om = xchg[((warp ^ 1) * 2 + (t >> 1)) * 2], of = xchg[((warp ^ 1) * 2 + (t >> 1)) * 2 + 1];
+        fm = of > fm ? of : fm;
+        nonfinite64 = mbits >= 0x7F80u || om >= 0x7F80u;
+        mbits = nonfinite64 ? fm : (om > mbits ? om : mbits);
+    }
 
-    const bool nonfinite = mbits >= 0x7F80u;
-    if (__any_sync(0xFFFFFFFFu, nonfinite)) {
+    const bool nonfinite = BLK == 64 ? nonfinite64 : mbits >= 0x7F80u;
+    if (BLK != 64 && __any_sync(0xFFFFFFFFu, nonfinite)) {
         // maximum over the finite entries only
         uint32_t fm = 0;
 #pragma unroll
@@ -202,7 +235,7 @@ __device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_
                 if (hi < 0x7F80u && hi > fm) fm = hi;
             }
 #pragma unroll
-        for (int s = 1; s <= 4; s <<= 1) {
+        for (int s = kShflLo; s <= kShflHi; s <<= 1) {
             const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, s);
             fm = other > fm ? other : fm;
         }
@@ -211,8 +244,11 @@ __device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_
 
     const int code = scale_code_from_max(mbits);
     const float inv = inv_scale(code);
-    if (tile_exists && (lane & 7) == 0)
+    if (BLK == 16) {
+        if ((lane & 2) == 0 && row0 < p.rows && col0 < p.cols) p.scale[(row0 >> 4) * p.ld_s + (col0 >> 4)] = (uint8_t)code;
+    } else if (tile_exists && (lane & 7) == 0) {
         p.scale[(tile_row0 >> 5) * p.ld_s + (tile_col0 >> 5)] = (uint8_t)code;
+    }
 
     uint32_t W[8][2];
     uint8_t *dst_rm = p.q_rm + row0 * p.ld_rm + (col0 >> 1);
@@ -289,15 +325,16 @@ __device__ __forceinline__ void quantize_tile(const Quant2dParams &p, uint4 *qt_
     }
 }
 
-template <int MODE>
+template <int MODE, int BLK = 32>
 __global__ void __launch_bounds__(128, FP4Q_QUANT_MIN_BLOCKS) quantize2d_kernel(const __grid_constant__ Quant2dParams p)
 {
     __shared__ uint4 qt_stage[128 * 4];   // 128 transposed rows x 64 B (four 16-byte chunks, XOR-swizzled)
     __shared__ uint4 rnd_stage[MODE == FP4Q_ROUND_STOCHASTIC ? 8 * 128 : 1];   // per thread: 8 rows x 16 random bytes
+    __shared__ uint32_t xchg[BLK == 64 ? 16 : 1];   // 64x64 blocks: maxima of the four warps' two half blocks
     const int64_t bx = (int64_t)blockIdx.x % p.grid_x, by = (int64_t)blockIdx.x / p.grid_x;
     const bool full = p.x_vec_ok == 2 && p.rng_aligned && (by + 1) * 128 <= p.rows && (bx + 1) * 128 <= p.cols;
-    if (full) quantize_tile<MODE, true>(p, qt_stage, rnd_stage);
-    else quantize_tile<MODE, false>(p, qt_stage, rnd_stage);
+    if (full) quantize_tile<MODE, true, BLK>(p, qt_stage, rnd_stage, xchg);
+    else quantize_tile<MODE, false, BLK>(p, qt_stage, rnd_stage, xchg);
 }
 
 }  // namespace fp4q
@@ -310,12 +347,14 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
 {
     if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
     if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
-    if (flags & ~FP4Q_INDEX_TRANSPOSED) return FP4Q_ERR_UNSUPPORTED;
+    if (flags & ~(FP4Q_INDEX_TRANSPOSED | FP4Q_BLOCK_16 | FP4Q_BLOCK_64)) return FP4Q_ERR_UNSUPPORTED;
+    if ((flags & FP4Q_BLOCK_16) && (flags & FP4Q_BLOCK_64)) return FP4Q_ERR_UNSUPPORTED;
+    const int sgran = (flags & FP4Q_BLOCK_16) ? 16 : 32;   // granularity of the scale matrix
     if (!out) return FP4Q_ERR_NULL;
     if (out->rows != rows || out->cols != cols) return FP4Q_ERR_SHAPE;
     if (rows == 0 || cols == 0) return FP4Q_OK;
     if (!x_bf16 || !out->q_rm || !out->scale) return FP4Q_ERR_NULL;
-    if (ld_x < cols || out->ld_rm < round_up(cols, 32) / 2 || out->ld_s < ceil_div(cols, 32)) return FP4Q_ERR_SHAPE;
+    if (ld_x < cols || out->ld_rm < round_up(cols, 32) / 2 || out->ld_s < ceil_div(cols, sgran)) return FP4Q_ERR_SHAPE;
     if (out->q_t && out->ld_t < round_up(rows, 32) / 2) return FP4Q_ERR_SHAPE;
     if (!aligned(x_bf16, 2) || !aligned(out->q_rm, 16) || out->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
     if (out->q_t && (!aligned(out->q_t, 16) || out->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
@@ -336,9 +375,17 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
     const int64_t n_cta = p.grid_x * ceil_div(rows, 128);
     if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (mode == FP4Q_ROUND_STOCHASTIC)
+    const bool sr = mode == FP4Q_ROUND_STOCHASTIC;
+    if (flags & FP4Q_BLOCK_16) {
+        if (sr) quantize2d_kernel<FP4Q_ROUND_STOCHASTIC, 16><<<(unsigned)n_cta, 128, 0, s>>>(p);
+        else quantize2d_kernel<FP4Q_ROUND_NEAREST, 16><<<(unsigned)n_cta, 128, 0, s>>>(p);
+    } else if (flags & FP4Q_BLOCK_64) {
+        if (sr) quantize2d_kernel<FP4Q_ROUND_STOCHASTIC, 64><<<(unsigned)n_cta, 128, 0, s>>>(p);
+        else quantize2d_kernel<FP4Q_ROUND_NEAREST, 64><<<(unsigned)n_cta, 128, 0, s>>>(p);
+    } else if (sr) {
         quantize2d_kernel<FP4Q_ROUND_STOCHASTIC><<<(unsigned)n_cta, 128, 0, s>>>(p);
-    else
+    } else {
         quantize2d_kernel<FP4Q_ROUND_NEAREST><<<(unsigned)n_cta, 128, 0, s>>>(p);
+    }
     return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }
