@@ -1244,7 +1244,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tcgen05.cp
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_cache_full + 8 * buf);   // forwarded to the leader by warp 2 in a pair's second CTA
+                if (lane == 0) {   // 16-stage units leave time for the second CTA's own (slow) remote arrival
+                    if (CTAS == 1 || leader) mbar_arrive(bar_cache_full + 8 * buf);
+                    else mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * buf, 0));
+                }
             }
         }
     } else if (warp == 2) {
@@ -1368,9 +1371,9 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
             sg.next(p, kStageElems);
         }
-        if (CTAS == 2 && !leader && lane == 0) {
-            // Second CTA of a pair: report each unit of scale images the builder has finished to the leader, which
-            // issues the scale copies of both CTAs.
+        if (KIND != KIND_MXF4 && CTAS == 2 && !leader && lane == 0) {
+            // Per-row scales, second CTA of a pair: report each unit of scale images the builder has finished to the
+            // leader, which issues the scale copies of both CTAs.
             bool fwd_ok = true;
             BufRing fr;
             UnitIter un;
