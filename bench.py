@@ -581,6 +581,30 @@ def run_kernel(args):
         out = binding.alloc_qtensor(rows, cols, dev)
         fn = lambda: binding.fp4q_quantize2d(x, out, mode=args.mode, seed=3, tensor_id=1)
         units, unit = rows * cols * BYTES_PER_ELEMENT / 1e9, "GB/s"
+    elif args.kernel in ("quantize1d", "quantize1d_t"):
+        rows, cols = dims
+        x = workloads.activations_student_t(rows, cols, 1, dev)
+        fn = (lambda: binding.fp4q_quantize1d(x)) if args.kernel == "quantize1d" else (lambda: binding.fp4q_quantize1d_t(x))
+        units, unit = rows * cols * (2.5 + 1 / 32) / 1e9, "GB/s"
+    elif args.kernel in ("gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm"):
+        T, N, K = dims
+        ws = binding.alloc_workspace(dev)
+        x = workloads.activations_student_t(T, K, 1, dev)
+        if args.kernel == "gemm_fwd_act1d":
+            xq, xs = binding.fp4q_quantize1d(x)
+            qw = binding.fp4q_quantize2d(workloads.weights(N, K, 2, dev))
+            out = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+            fn = lambda: binding.fp4q_gemm_fwd_act1d(xq, xs, T, qw, out=out, ws=ws)
+        elif args.kernel == "gemm_wgrad_act1d":
+            xtq, xts = binding.fp4q_quantize1d_t(x)
+            qdy = binding.fp4q_quantize2d(workloads.gradients_rowscaled(T, N, 3, dev), mode=1, seed=3, tensor_id=2)
+            out = torch.empty((N, K), dtype=torch.float32, device=dev)
+            fn = lambda: binding.fp4q_gemm_wgrad_act1d(qdy, xtq, xts, K, out=out, ws=ws)
+        else:
+            xq, xs = binding.fp4q_mxfp8_quantize1d(x)
+            wq, wsf = binding.fp4q_mxfp8_quantize1d(workloads.weights(N, K, 2, dev))
+            fn = lambda: binding.fp4q_mxfp8_gemm(xq, xs, wq, wsf, T, N, K, ws=ws)
+        units, unit = 2.0 * T * N * K / 1e12, "TFLOP/s"
     else:
         T, N, K = dims
         ws = binding.alloc_workspace(dev)
@@ -620,7 +644,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad"],
+    ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "quantize1d", "quantize1d_t",
+                                                        "gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm"],
                     help="run one kernel on --shape a few times (for profiler captures) instead of the benchmark")
     ap.add_argument("--shape", default="16384x4096", help="RxC for quantize, TxNxK for the GEMMs")
     ap.add_argument("--iters", type=int, default=3)
