@@ -196,19 +196,28 @@ def run_gpu(args):
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
-    def step(marks=None):
-        if marks: marks[0].record()
+    def phase_quantize():
         for x, q, tid in quant_jobs:
             binding.fp4q_quantize2d(x, q, mode=SR, seed=seed, tensor_id=tid)
-        if marks: marks[1].record()
+
+    def phase_fwd():
         for i, o in enumerate(ops):
             binding.fp4q_gemm_fwd(q_x[o["x_key"]], q_w[i], out=outputs(o)[0], dt=binding.OUT_BF16, ws=ws)
-        if marks: marks[2].record()
+
+    def phase_dgrad():
         for i, o in enumerate(ops):
             binding.fp4q_gemm_dgrad(q_dy[i], q_w[i], out=outputs(o)[1], dt=binding.OUT_BF16, ws=ws)
-        if marks: marks[3].record()
+
+    def phase_wgrad():
         for i, o in enumerate(ops):
             binding.fp4q_gemm_wgrad(q_dy[i], q_x[o["x_key"]], out=outputs(o)[2], dt=binding.OUT_F32, ws=ws)
+
+    phases = [phase_quantize, phase_fwd, phase_dgrad, phase_wgrad]
+
+    def step(marks=None):
+        for i, ph in enumerate(phases):
+            if marks: marks[i].record()
+            ph()
         if marks: marks[4].record()
 
     launches_per_step = len(quant_jobs) + 3 * len(ops)
@@ -229,6 +238,19 @@ def run_gpu(args):
     barrier()
     if binding.fp4q_workspace_status(ws) != 0:
         raise RuntimeError("a GEMM kernel reported a device-side timeout during warm-up")
+    if not args.no_graphs:
+        # The step's launches are short (8 us for a 4096 x 4096 weight) against the cost of issuing them one by one
+        # from Python: each phase is captured once into a CUDA graph (same kernels, same arguments, same order) and
+        # the timed steps replay the graphs.
+        graphs = []
+        for ph in list(phases):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                ph()
+            graphs.append(g)
+        phases[:] = [g.replay for g in graphs]
+        step()
+        barrier()
 
     marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
     barrier()
@@ -344,7 +366,8 @@ def run_gpu(args):
         "config": {"workload": cfg.name + ": hidden %d, FFN %d, %d tokens; quantize sweep over 7 W + %d X + 7 dY "
                                "(stochastic rounding) then fwd/dgrad/wgrad FP4 GEMMs of 7 linear layers" %
                                (cfg.hidden, cfg.ffn, cfg.tokens, len(xs)),
-                   "parallelism": "replicas only (x%d)" % world, "l2": "inputs larger than L2 (%.2f GB of BF16 operands per step)" %
+                   "parallelism": "replicas only (x%d)" % world,
+                   "launch": "per-launch calls from Python" if args.no_graphs else "one CUDA graph per phase (quantize, fwd, dgrad, wgrad), replayed", "l2": "inputs larger than L2 (%.2f GB of BF16 operands per step)" %
                    (quant_elems * 2 / 1e9), "quantize_bytes_per_step": quant_bytes, "gemm_flops_per_step": 3 * gemm_flops},
         "gemm_tflops": gemm_tflops,
         "phase_ms": {"quantize": q_ms, "fwd": f_ms, "dgrad": d_ms, "wgrad": w_ms},
@@ -643,6 +666,7 @@ def main():
     ap.add_argument("--workload", default="7b", choices=["7b", "1b", "tiny"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-graphs", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "quantize1d", "quantize1d_t",
                                                         "gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm"],
