@@ -93,3 +93,37 @@ def test_mixed_layout_differs_from_all_2d_and_shows_the_inconsistency():
     y2 = binding.fp4q_gemm_fwd(X2, W, dt=binding.OUT_F32)
     torch.cuda.synchronize()
     assert (y1 - y2).norm() / y2.norm() > 1e-3
+
+
+def test_full_size_attention_projection_sampled_rows():
+    """16384 tokens, 4096 x 4096 (the shape the benchmark times these products on), in the benchmark's launch
+    configuration: the oracle recomputes a deterministic sample of output rows from operands it dequantizes itself."""
+    T, N, K = 16384, 4096, 4096
+    x = workloads.activations_student_t(T, K, 21, "cuda")
+    w = workloads.weights(N, K, 22, "cuda")
+    dy = workloads.gradients_rowscaled(T, N, 23, "cuda")
+    W = binding.fp4q_quantize2d(w)
+    dY = binding.fp4q_quantize2d(dy, mode=1, seed=5, tensor_id=2)
+    xq, xs = binding.fp4q_quantize1d(x)
+    xtq, xts = binding.fp4q_quantize1d_t(x)
+    ws = binding.alloc_workspace("cuda")
+    y = binding.fp4q_gemm_fwd_act1d(xq, xs, T, W, dt=binding.OUT_F32, ws=ws)
+    dw = binding.fp4q_gemm_wgrad_act1d(dY, xtq, xts, K, dt=binding.OUT_F32, ws=ws)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    rng = np.random.default_rng(1)
+    rows = np.unique(np.concatenate([[0, T - 1], rng.integers(0, T, 30)]))
+    # forward: sampled token rows; the oracle quantizes those rows itself (1D blocks lie inside a row)
+    oq, os_ = oracle.quantize1d(workloads.bf16_bits(x[torch.from_numpy(rows).cuda()]))
+    g_q = xq[torch.from_numpy(rows).cuda()].cpu().numpy()
+    assert np.array_equal(g_q[:, :oq.shape[1]], oq)
+    x_hat = oracle.dequantize1d(oq, os_, len(rows), K)
+    check(y[torch.from_numpy(rows).cuda()], oracle.gemm_fwd(x_hat, dequant_from_gpu(W)), "forward sample, 1D activations")
+    # weight gradient: sampled output rows n need column n of dY over all tokens and the whole transposed encoding of X
+    ncols = np.unique(np.concatenate([[0, N - 1], rng.integers(0, N, 10)]))
+    dyd = dequant_from_gpu(dY)[:, ncols]
+    xt_hat = oracle.dequantize1d(np.ascontiguousarray(xtq.cpu().numpy()[:, :T // 2]), np.ascontiguousarray(xts.cpu().numpy()), K, T)
+    sample_cols = rng.integers(0, K, 16)           # the transposed encoding itself, on sampled columns of x
+    oq_t, os_t = oracle.quantize1d(np.ascontiguousarray(workloads.bf16_bits(x[:, torch.from_numpy(sample_cols).cuda()]).T))
+    assert np.array_equal(xtq.cpu().numpy()[sample_cols, :T // 2], oq_t) and np.array_equal(xts.cpu().numpy()[sample_cols], os_t)
+    check(dw[torch.from_numpy(ncols).cuda()], dyd.T @ xt_hat.T, "wgrad sample, 1D activations")
