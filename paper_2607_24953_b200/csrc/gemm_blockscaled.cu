@@ -37,6 +37,7 @@ namespace fp4q {
 constexpr int BM = 128, BN = 256;            // per-CTA accumulator: 128 rows x 256 columns (a CTA pair covers 256 x 256)
 constexpr int kMaxStages = 6;
 constexpr int kAStageBytes = BM * 128;
+constexpr int kMaxGroupsShared = 1023;       // grouped products: group boundaries kept in shared memory up to this many groups
 constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
 // 2D-block scales: the scale images of a whole unit (up to 16 stages = 4096 contraction elements of one tile) are
 // built once, ahead of time, and tcgen05.cp reads them in place.  Per 128-element chunk the compact form is one
@@ -90,7 +91,9 @@ struct Cfg {
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
     static constexpr int kSmemStaging = CTAS == 2 ? 8 * kStagingWarpBytes : 0;
-    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail;
+    static constexpr int kSmemGroups = CTAS == 1 ? (kMaxGroupsShared + 1) * 4 : 0;   // grouped products: group boundaries
+    static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail + kSmemGroups;
+    static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
 constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
@@ -388,17 +391,23 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_i
 
 // ---------------------------------------------------------------------------------------- tile decoding
 
-__device__ __forceinline__ int find_group(const int64_t *offs, int n_groups, int64_t row)
+// Grouped products look up their group boundaries once per tile and role.  From global memory that is a chain of
+// dependent loads (seven for 128 groups) of a few hundred cycles each - more than a tile with a short contraction
+// runs - so the one-CTA kernel keeps a 32-bit copy of the boundaries in shared memory (`goffs`, null when there are
+// more than kMaxGroupsShared groups or the kernel has no room for it).
+
+__device__ __forceinline__ int find_group(const int64_t *offs, const int32_t *goffs, int n_groups, int64_t row)
 {
     int lo = 0, hi = n_groups;      // largest g with offs[g] <= row
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (__ldg(offs + mid) <= row) lo = mid; else hi = mid;
+        const int64_t v = goffs ? (int64_t)goffs[mid] : __ldg(offs + mid);
+        if (v <= row) lo = mid; else hi = mid;
     }
     return lo;
 }
 
-__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int rank, Tile &t)
+__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int rank, Tile &t, const int32_t *goffs)
 {
     const int per_problem = p.m_tiles * p.n_tiles;
     const int g = p.mode == MODE_GROUPED_K ? tile / per_problem : 0;
@@ -420,12 +429,12 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int r
     t.m_valid = min(BM, p.M - t.a_row0);
     t.n_valid = min(BN, p.N - t.b_row0);
     if (p.mode == MODE_GROUPED_ROWS) {
-        const int grp = find_group(p.row_offsets, p.n_groups, (int64_t)t.a_row0);
+        const int grp = find_group(p.row_offsets, goffs, p.n_groups, (int64_t)t.a_row0);
         t.b_row0 += grp * p.b_rows_per_group;
         t.b_load_row0 += grp * p.b_rows_per_group;
         t.b_k0 = grp * p.b_k_per_group;
     } else if (p.mode == MODE_GROUPED_K) {
-        const int64_t k0 = __ldg(p.row_offsets + g), k1 = __ldg(p.row_offsets + g + 1);
+        const int64_t k0 = goffs ? (int64_t)goffs[g] : __ldg(p.row_offsets + g), k1 = goffs ? (int64_t)goffs[g + 1] : __ldg(p.row_offsets + g + 1);
         t.a_k0 = t.b_k0 = (int32_t)k0;
         t.k_len = (int32_t)(k1 - k0);
         t.c_row0 = g * p.M + t.a_row0;
@@ -450,20 +459,21 @@ __device__ __forceinline__ void load_scale(const ScaleView &v, int row, int kb, 
 // The stream of ring stages one CTA works through: its tiles in order, each with its contraction stages.
 struct StageIter {
     int tile, step, rank, it, n_it;
+    const int32_t *goffs;
     Tile t;
     __device__ __forceinline__ void seek(const GemmParams &p, int stage_elems)
     {
         while (tile < p.n_tile_total) {
-            decode_tile(p, tile, rank, t);
+            decode_tile(p, tile, rank, t, goffs);
             n_it = (t.k_len + stage_elems - 1) / stage_elems;
             if (n_it > 0) { it = 0; return; }
             tile += step;
         }
         n_it = 0;
     }
-    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, int stage_elems)
+    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, int stage_elems, const int32_t *goffs_)
     {
-        tile = first; step = step_; rank = rank_; it = 0;
+        tile = first; step = step_; rank = rank_; it = 0; goffs = goffs_;
         seek(p, stage_elems);
     }
     __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
@@ -790,17 +800,22 @@ struct BufRing {
 // The stream of scale units (kUnitStages stages of one tile) a CTA works through.
 struct UnitIter {
     int tile, step, rank, k0;
+    const int32_t *goffs;
     Tile t;
     __device__ __forceinline__ void seek(const GemmParams &p)
     {
         while (tile < p.n_tile_total) {
-            decode_tile(p, tile, rank, t);
+            decode_tile(p, tile, rank, t, goffs);
             if (k0 < t.k_len) return;
             tile += step;
             k0 = 0;
         }
     }
-    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_) { tile = first; step = step_; rank = rank_; k0 = 0; seek(p); }
+    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, const int32_t *goffs_)
+    {
+        tile = first; step = step_; rank = rank_; k0 = 0; goffs = goffs_;
+        seek(p);
+    }
     __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
     __device__ __forceinline__ void next(const GemmParams &p, int unit_elems) { k0 += unit_elems; seek(p); }
 };
@@ -950,6 +965,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     // bars[32..35] (leader of a pair) the second CTA's scale images full - one of each per image buffer
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 21);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bars + 21) + 1;
+    int32_t *goffs_smem = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(bars) + kSmemTail);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
@@ -996,6 +1012,11 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
         }
     }
+    // grouped products: a 32-bit copy of the group boundaries for the per-tile lookups of every role
+    const bool goffs_ok = CTAS == 1 && p.mode != MODE_DENSE && p.n_groups <= kMaxGroupsShared;
+    if (goffs_ok)
+        for (int g = threadIdx.x; g <= p.n_groups; g += kThreads) goffs_smem[g] = (int32_t)__ldg(p.row_offsets + g);
+    const int32_t *goffs = goffs_ok ? goffs_smem : nullptr;
     tcgen05_fence_before();
     __syncwarp();
     if (CTAS == 2) cluster_sync_all();   // the peer's barriers must exist before anything is signalled across CTAs
@@ -1011,7 +1032,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // more - and only then issues the loads of all slots found free, back to back.
         constexpr int kBatch = 3;
         StageIter pr;
-        pr.init(p, first_tile, tile_step, rank, kStageElems);
+        pr.init(p, first_tile, tile_step, rank, kStageElems, goffs);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         const bool issuer = elect_one();
@@ -1083,7 +1104,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_T0(tt);
         for (int tile = first_tile; leader && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, rank, t);
+            decode_tile(p, tile, rank, t, goffs);
             const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
             if (n_it == 0) continue;
             TRACE_ADD(c_acc, tt);
@@ -1168,8 +1189,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             // (a suspended try_wait is not reliably woken early by a remote arrival).
             constexpr int kRawBufs = Cfg<KIND, CTAS>::kRawBufs > 0 ? Cfg<KIND, CTAS>::kRawBufs : 1;
             UnitIter ahead, cur;
-            ahead.init(p, first_tile, tile_step, rank);
-            cur.init(p, first_tile, tile_step, rank);
+            ahead.init(p, first_tile, tile_step, rank, goffs);
+            cur.init(p, first_tile, tile_step, rank, goffs);
             uint32_t raw_fill = 0, raw_read = 0;
             for (int i = 0; i < kRawBufs; i++) {
                 if (ahead.valid(p)) {
@@ -1211,7 +1232,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         }
         for (int tile = first_tile; KIND == KIND_MXF4 && ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, rank, t);
+            decode_tile(p, tile, rank, t, goffs);
             for (int k0 = 0; ok && k0 < t.k_len; k0 += kUnitStages * kStageElems, ring.next(kImageBufs)) {
                 const int buf = ring.buf;
                 uint8_t *images = smem_images + buf * kCacheBufBytes;
@@ -1259,7 +1280,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // stage is released unseen, so that the MMA warp, which cannot time out on a named barrier, always runs
         // to its end.
         StageIter sg;
-        sg.init(p, first_tile, tile_step, rank, kStageElems);
+        sg.init(p, first_tile, tile_step, rank, kStageElems, goffs);
         uint32_t stage = 0, phase = 0, acc_phase = 0;
         BufRing ring;   // image buffer of the current unit
         bool ok = true;
@@ -1377,7 +1398,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             bool fwd_ok = true;
             BufRing fr;
             UnitIter un;
-            for (un.init(p, first_tile, tile_step, rank); fwd_ok && un.valid(p); un.next(p, kUnitStages * kStageElems), fr.next(kImageBufs)) {
+            for (un.init(p, first_tile, tile_step, rank, goffs); fwd_ok && un.valid(p); un.next(p, kUnitStages * kStageElems), fr.next(kImageBufs)) {
                 fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * fr.buf, fr.phase, abort_flag, p.status, 0x530u + fr.buf);
                 if (fwd_ok) mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * fr.buf, 0));
             }
@@ -1395,7 +1416,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_T0(tt);
         for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, rank, t);
+            decode_tile(p, tile, rank, t, goffs);
             const int row_in_tile = 32 * quarter + lane;
             const int64_t row = (int64_t)t.c_row0 + row_in_tile;
             const bool row_ok = row_in_tile < t.m_valid;
