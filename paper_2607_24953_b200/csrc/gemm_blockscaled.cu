@@ -1731,11 +1731,12 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     p.sfb = B.sf;
     p.status = reinterpret_cast<uint32_t *>(ws);
     // Dense products (FP4 and MXFP8) with more than one row tile run as cta_group::2 pairs: 256x256 tiles, each CTA
-    // loads half of the B rows.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the
-    // first GEMM call) selects the one-CTA kernel instead; grouped products (token groups are only 128-row aligned)
+    // loads half of the B rows; so does the grouped weight gradient, whose groups cut the contraction axis, not the
+    // output rows of a tile.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the first GEMM call) selects
+    // the one-CTA kernel instead; grouped forward / input-gradient products (token groups are only 128-row aligned)
     // always use one CTA per 128x256 tile.
     static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return !(e && e[0] == '0'); }();
-    if (use_pairs && p.mode == MODE_DENSE && p.M > BM) return launch_gemm_impl<KIND, 2>(A, B, p, stream);
+    if (use_pairs && (p.mode == MODE_DENSE || p.mode == MODE_GROUPED_K) && p.M > BM) return launch_gemm_impl<KIND, 2>(A, B, p, stream);
     return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
 

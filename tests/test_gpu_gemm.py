@@ -205,6 +205,30 @@ def test_grouped_small_with_empty_and_uneven_groups(ws):
     _moe_case(ws, E=5, H=256, F=192, counts=np.array([130, 0, 1, 300, 128]), seed=11)
 
 
+def test_grouped_expert_width_not_a_multiple_of_the_tile_and_accumulation(ws):
+    # expert width 320: in the weight gradient's second pair tile the first CTA holds 64 valid rows and the second none;
+    # the rows below belong to the next expert's block of the output and must stay untouched; then the same product
+    # accumulated into FP32
+    E, H, F = 3, 320, 320
+    counts = np.array([64, 200, 0])
+    _moe_case(ws, E=E, H=H, F=F, counts=counts, seed=13)
+    offs = workloads.padded_row_offsets(counts, 128)
+    T = int(offs[-1])
+    g = torch.Generator(device="cuda").manual_seed(14)
+    X = workloads.zero_padding_rows(torch.randn(T, H, generator=g, device="cuda").to(torch.bfloat16), counts, offs)
+    dY = workloads.zero_padding_rows((torch.randn(T, F, generator=g, device="cuda") * 0.01).to(torch.bfloat16), counts, offs)
+    qx, xd = quantized(X, 0, 1, 1)
+    qdy, dyd = quantized(dY, 1, 1, 2)
+    acc = torch.full((E * F, H), 0.5, dtype=torch.float32, device="cuda")
+    binding.fp4q_gemm_wgrad(qdy, qx, out=acc, dt=binding.OUT_F32, accumulate=True, row_offsets=torch.from_numpy(offs).cuda(), ws=ws)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    ref = oracle.grouped_wgrad(dyd, xd, offs) + 0.5
+    got = acc.double().cpu().numpy()
+    assert np.array_equal(got[2 * F:], np.full((F, H), 0.5))      # the empty expert adds nothing
+    check(acc[:2 * F], ref[:2 * F], "grouped wgrad, accumulate")
+
+
 def test_grouped_moe_shapes_reduced_expert_count(ws):
     # expert-layer shapes of the MoE configuration (hidden 2048, expert FFN 768), Zipf(1.2) top-8 loads,
     # on 16 experts and 2048 tokens so that the oracle finishes in seconds
