@@ -472,36 +472,38 @@ def run_extras(torch, binding, workloads, dev, ws):
         "all_2d_fwd_tflops": 2.0 * T * H * H / (ms_p * 1e-3) / 1e12, "all_2d_wgrad_tflops": 2.0 * T * H * H / (ms_w2 * 1e-3) / 1e12}
     del X, Wq, Wk, qx4, qw4, y, qy, dY4, x1q, x1s, x1tq, x1ts, dw
 
-    # --- grouped MoE expert layer: 128 experts, hidden 2048, expert FFN 768, top-8 of 16384 tokens
+    # --- grouped MoE expert layer: 128 experts, hidden 2048, expert FFN 768, top-8 of 16384 tokens; token groups padded
+    # to 128 rows (the configuration's figure) and to 256 rows, which lets forward and input gradient run on CTA pairs
     moe = workloads.CONFIG_MOE
     counts = workloads.moe_routing(moe)
-    offs = workloads.padded_row_offsets(counts, moe.pad)
-    Tp = int(offs[-1])
-    d_offs = torch.from_numpy(offs).to(dev)
-    E, H, F = moe.experts, moe.hidden, moe.expert_ffn
-    res = {"workload": "%d experts, hidden %d, expert FFN %d, %d routed rows padded to %d; loads max %d / median %d / min %d" %
-                       (E, H, F, int(counts.sum()), Tp, int(counts.max()), int(np.median(counts)), int(counts.min()))}
-    tot_ms, tot_flops = 0.0, 0.0
-    for name, n, k in moe.layers():
-        Xm = workloads.zero_padding_rows(workloads.activations_student_t(Tp, k, moe.data_seed + 1, dev), counts, offs)
-        dYm = workloads.zero_padding_rows(workloads.gradients_rowscaled(Tp, n, moe.data_seed + 2, dev), counts, offs)
-        Wm = workloads.weights(E * n, k, moe.data_seed, dev)
-        qx, qw, qdy = (binding.fp4q_quantize2d(t, mode=1, seed=moe.philox_seed, tensor_id=i) for i, t in enumerate((Xm, Wm, dYm)))
-        y = torch.empty((Tp, n), dtype=torch.bfloat16, device=dev)
-        dx = torch.empty((Tp, k), dtype=torch.bfloat16, device=dev)
-        dw = torch.empty((E * n, k), dtype=torch.float32, device=dev)
-        flops = 2.0 * float(counts.sum()) * n * k
-        ms = [timed(lambda: binding.fp4q_gemm_fwd(qx, qw, out=y, row_offsets=d_offs, ws=ws)),
-              timed(lambda: binding.fp4q_gemm_dgrad(qdy, qw, out=dx, row_offsets=d_offs, ws=ws)),
-              timed(lambda: binding.fp4q_gemm_wgrad(qdy, qx, out=dw, row_offsets=d_offs, ws=ws))]
-        res[name] = {"fwd_tflops": flops / (ms[0] * 1e-3) / 1e12, "dgrad_tflops": flops / (ms[1] * 1e-3) / 1e12,
-                     "wgrad_tflops": flops / (ms[2] * 1e-3) / 1e12, "ms": ms,
-                     "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9}
-        tot_ms += sum(ms)
-        tot_flops += 3 * flops
-        del Xm, dYm, Wm, qx, qw, qdy, y, dx, dw
-    res["all_tflops"] = tot_flops / (tot_ms * 1e-3) / 1e12
-    out["moe_grouped"] = res
+    for pad, key in ((moe.pad, "moe_grouped"), (256, "moe_grouped_groups_padded_to_256")):
+        offs = workloads.padded_row_offsets(counts, pad)
+        Tp = int(offs[-1])
+        d_offs = torch.from_numpy(offs).to(dev)
+        E, H, F = moe.experts, moe.hidden, moe.expert_ffn
+        res = {"workload": "%d experts, hidden %d, expert FFN %d, %d routed rows padded to %d; loads max %d / median %d / min %d" %
+                           (E, H, F, int(counts.sum()), Tp, int(counts.max()), int(np.median(counts)), int(counts.min()))}
+        tot_ms, tot_flops = 0.0, 0.0
+        for name, n, k in moe.layers():
+            Xm = workloads.zero_padding_rows(workloads.activations_student_t(Tp, k, moe.data_seed + 1, dev), counts, offs)
+            dYm = workloads.zero_padding_rows(workloads.gradients_rowscaled(Tp, n, moe.data_seed + 2, dev), counts, offs)
+            Wm = workloads.weights(E * n, k, moe.data_seed, dev)
+            qx, qw, qdy = (binding.fp4q_quantize2d(t, mode=1, seed=moe.philox_seed, tensor_id=i) for i, t in enumerate((Xm, Wm, dYm)))
+            y = torch.empty((Tp, n), dtype=torch.bfloat16, device=dev)
+            dx = torch.empty((Tp, k), dtype=torch.bfloat16, device=dev)
+            dw = torch.empty((E * n, k), dtype=torch.float32, device=dev)
+            flops = 2.0 * float(counts.sum()) * n * k      # routed rows only: padding rows are not counted as work
+            ms = [timed(lambda: binding.fp4q_gemm_fwd(qx, qw, out=y, row_offsets=d_offs, ws=ws, row_alignment=pad)),
+                  timed(lambda: binding.fp4q_gemm_dgrad(qdy, qw, out=dx, row_offsets=d_offs, ws=ws, row_alignment=pad)),
+                  timed(lambda: binding.fp4q_gemm_wgrad(qdy, qx, out=dw, row_offsets=d_offs, ws=ws))]
+            res[name] = {"fwd_tflops": flops / (ms[0] * 1e-3) / 1e12, "dgrad_tflops": flops / (ms[1] * 1e-3) / 1e12,
+                         "wgrad_tflops": flops / (ms[2] * 1e-3) / 1e12, "ms": ms,
+                         "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9}
+            tot_ms += sum(ms)
+            tot_flops += 3 * flops
+            del Xm, dYm, Wm, qx, qw, qdy, y, dx, dw
+        res["all_tflops"] = tot_flops / (tot_ms * 1e-3) / 1e12
+        out[key] = res
     if binding.fp4q_workspace_status(ws) != 0:
         out["status"] = "device-side timeout reported"
     return out

@@ -91,10 +91,14 @@ typedef struct {
  * of n_groups+1 non-decreasing int64 values, each a multiple of 128, with row_offsets[0] = 0
  * and row_offsets[n_groups] = the token matrices' row count; padding rows inside a group must
  * hold zeros (the boundary-block rule of the appendix then makes them inert).  Groups may be
- * empty.
+ * empty.  row_alignment is the caller's statement about the offsets: 0 or 128 = multiples of 128 (the general
+ * case); 256 = every offset is a multiple of 256, which lets the grouped forward and input-gradient products
+ * run on the 256-row CTA-pair tiles of the dense products (a wrong statement gives wrong results for the rows
+ * of a tile that straddles two groups, nothing worse).  Other values: FP4Q_ERR_UNSUPPORTED.
  */
 typedef struct {
     int32_t n_groups;
+    int32_t row_alignment;
     const int64_t *row_offsets;
 } fp4q_groups;
 

@@ -44,7 +44,7 @@ class _CTensor(ctypes.Structure):
 
 
 class _CGroups(ctypes.Structure):
-    _fields_ = [("n_groups", ctypes.c_int32), ("row_offsets", ctypes.c_void_p)]
+    _fields_ = [("n_groups", ctypes.c_int32), ("row_alignment", ctypes.c_int32), ("row_offsets", ctypes.c_void_p)]
 
 
 _lib = None
@@ -316,13 +316,13 @@ def fp4q_workspace_status(ws: torch.Tensor, stream=None) -> int:
     return int(lib().fp4q_workspace_status(ws.data_ptr(), _stream(stream)))
 
 
-def _groups(row_offsets: Optional[torch.Tensor]):
+def _groups(row_offsets: Optional[torch.Tensor], row_alignment: int = 128):
     if row_offsets is None:
         return None, None
     _dev(row_offsets, "row_offsets")
     if row_offsets.dtype != torch.int64 or not row_offsets.is_contiguous():
         raise ValueError("row_offsets must be a contiguous int64 device tensor")
-    g = _CGroups(row_offsets.numel() - 1, row_offsets.data_ptr())
+    g = _CGroups(row_offsets.numel() - 1, row_alignment, row_offsets.data_ptr())
     return g, ctypes.byref(g)
 
 
@@ -330,7 +330,8 @@ def _out_dtype(dt: int):
     return torch.bfloat16 if dt == OUT_BF16 else torch.float32
 
 
-def _gemm(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, row_offsets, ws, stream, accumulate=None):
+def _gemm(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, row_offsets, ws, stream, accumulate=None,
+          row_alignment: int = 128):
     dev = a.q_rm.device
     if out is None:
         # the ABI wants the leading dimension to be a multiple of 16 bytes: pad it and return a view
@@ -340,7 +341,7 @@ def _gemm(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, row_offs
     if ws is None:
         ws = alloc_workspace(dev)
     ca, cb = a.c_struct(), b.c_struct()
-    g, gref = _groups(row_offsets)
+    g, gref = _groups(row_offsets, row_alignment)
     fn = getattr(lib(), fn_name)
     args = [ctypes.byref(ca), ctypes.byref(cb), out.data_ptr(), out.stride(0) if out.numel() else out_cols, dt]
     if accumulate is not None:
@@ -350,10 +351,11 @@ def _gemm(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, row_offs
     return out
 
 
-def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None):
+def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None,
+                  row_alignment: int = 128):
     """Y[T,N] = X^ W^^T. Grouped when row_offsets is given (W is then the expert stack [E*N, K])."""
     n = W.rows if row_offsets is None else W.rows // (row_offsets.numel() - 1)
-    return _gemm("fp4q_gemm_fwd", X, W, X.rows, n, out, dt, row_offsets, ws, stream)
+    return _gemm("fp4q_gemm_fwd", X, W, X.rows, n, out, dt, row_offsets, ws, stream, row_alignment=row_alignment)
 
 
 def fp4q_gemm_fwd_quantized(X: QTensor, W: QTensor, out: Optional[QTensor] = None, mode: int = ROUND_NEAREST,
@@ -399,9 +401,10 @@ def fp4q_gemm_fwd_static_workspace(X: QTensor, W: QTensor, out: torch.Tensor, dt
     return out
 
 
-def fp4q_gemm_dgrad(dY: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None):
+def fp4q_gemm_dgrad(dY: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offsets=None, ws=None, stream=None,
+                    row_alignment: int = 128):
     """dX[T,K] = dY^ W^."""
-    return _gemm("fp4q_gemm_dgrad", dY, W, dY.rows, W.cols, out, dt, row_offsets, ws, stream)
+    return _gemm("fp4q_gemm_dgrad", dY, W, dY.rows, W.cols, out, dt, row_offsets, ws, stream, row_alignment=row_alignment)
 
 
 def fp4q_gemm_wgrad(dY: QTensor, X: QTensor, out=None, dt: int = OUT_F32, accumulate: bool = False,

@@ -37,7 +37,8 @@ namespace fp4q {
 constexpr int BM = 128, BN = 256;            // per-CTA accumulator: 128 rows x 256 columns (a CTA pair covers 256 x 256)
 constexpr int kMaxStages = 6;
 constexpr int kAStageBytes = BM * 128;
-constexpr int kMaxGroupsShared = 1023;       // grouped products: group boundaries kept in shared memory up to this many groups
+constexpr int kMaxGroupsShared = 1023;       // grouped contraction: boundaries kept in shared memory up to this many groups
+constexpr int kMaxRowTilesShared = 2048;     // grouped rows: group of each 128-row tile kept in shared memory up to this many tiles
 constexpr int kSmemTail = 512;               // barriers, TMEM base, abort flag, scale scratch (one per loader warp)
 // 2D-block scales: the scale images of a whole unit (up to 16 stages = 4096 contraction elements of one tile) are
 // built once, ahead of time, and tcgen05.cp reads them in place.  Per 128-element chunk the compact form is one
@@ -91,7 +92,8 @@ struct Cfg {
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
     static constexpr int kSmemStaging = CTAS == 2 ? 8 * kStagingWarpBytes : 0;
-    static constexpr int kSmemGroups = CTAS == 1 ? (kMaxGroupsShared + 1) * 4 : 0;   // grouped products: group boundaries
+    static constexpr int kSmemGroups = (CTAS == 1 || KIND == KIND_MXF4) ? (kMaxGroupsShared + 1) * 4 : 0;   // grouped products: group table
+    static_assert(kSmemGroups == 0 || kSmemGroups >= kMaxRowTilesShared * 2, "group table");
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail + kSmemGroups;
     static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
@@ -147,6 +149,7 @@ struct GemmParams {
     int32_t out_f32, accumulate;
     int32_t wide_stores;             // output base and row pitch are 32-byte aligned: 256-bit stores (whole sectors)
     int32_t mode, n_groups;
+    int32_t rows_pair_aligned;       // grouped rows: every group starts on a multiple of 256 rows (caller's statement)
     const int64_t *row_offsets;
     int32_t b_rows_per_group;        // grouped rows: B row offset per group (forward)
     int32_t b_k_per_group;           // grouped rows: B contraction offset per group (dgrad)
@@ -391,10 +394,12 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_i
 
 // ---------------------------------------------------------------------------------------- tile decoding
 
-// Grouped products look up their group boundaries once per tile and role.  From global memory that is a chain of
-// dependent loads (seven for 128 groups) of a few hundred cycles each - more than a tile with a short contraction
-// runs - so the one-CTA kernel keeps a 32-bit copy of the boundaries in shared memory (`goffs`, null when there are
-// more than kMaxGroupsShared groups or the kernel has no room for it).
+// Grouped products need their group once per tile.  Searching the boundaries is a chain of dependent loads (seven
+// for 128 groups), and in the TMA producer every load queues behind the copies it has just issued (about 500 cycles
+// each): 4000 cycles per tile, more than a tile with a short contraction runs.  So the CTA fills a table in shared
+// memory before its roles start (`goffs`, 4 KB, null when the problem is too large for it or the kernel's
+// configuration has no room): with grouped rows the group of every 128-row tile as 16 bits (one load per tile),
+// with a grouped contraction a 32-bit copy of the boundaries.
 
 __device__ __forceinline__ int find_group(const int64_t *offs, const int32_t *goffs, int n_groups, int64_t row)
 {
@@ -407,7 +412,11 @@ __device__ __forceinline__ int find_group(const int64_t *offs, const int32_t *go
     return lo;
 }
 
-__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int rank, Tile &t, const int32_t *goffs)
+// need_b = false leaves out the B operand's position: with grouped rows that is the group lookup, which only the
+// producer and the scale builder need - the MMA issuer, the watcher and the epilogue use the contraction length and
+// the output position alone, and a lookup in the MMA warp (shared-memory reads behind its pending MMAs) costs
+// about 1900 cycles per tile.
+__device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int rank, Tile &t, const int32_t *goffs, bool need_b = true)
 {
     const int per_problem = p.m_tiles * p.n_tiles;
     const int g = p.mode == MODE_GROUPED_K ? tile / per_problem : 0;
@@ -429,7 +438,9 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int r
     t.m_valid = min(BM, p.M - t.a_row0);
     t.n_valid = min(BN, p.N - t.b_row0);
     if (p.mode == MODE_GROUPED_ROWS) {
-        const int grp = find_group(p.row_offsets, goffs, p.n_groups, (int64_t)t.a_row0);
+        if (!need_b) return;
+        const int grp = goffs ? (int)reinterpret_cast<const uint16_t *>(goffs)[t.a_row0 / BM]
+                              : find_group(p.row_offsets, nullptr, p.n_groups, (int64_t)t.a_row0);
         t.b_row0 += grp * p.b_rows_per_group;
         t.b_load_row0 += grp * p.b_rows_per_group;
         t.b_k0 = grp * p.b_k_per_group;
@@ -460,20 +471,22 @@ __device__ __forceinline__ void load_scale(const ScaleView &v, int row, int kb, 
 struct StageIter {
     int tile, step, rank, it, n_it;
     const int32_t *goffs;
+    bool need_b;
     Tile t;
     __device__ __forceinline__ void seek(const GemmParams &p, int stage_elems)
     {
         while (tile < p.n_tile_total) {
-            decode_tile(p, tile, rank, t, goffs);
+            decode_tile(p, tile, rank, t, goffs, need_b);
             n_it = (t.k_len + stage_elems - 1) / stage_elems;
             if (n_it > 0) { it = 0; return; }
             tile += step;
         }
         n_it = 0;
     }
-    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, int stage_elems, const int32_t *goffs_)
+    __device__ __forceinline__ void init(const GemmParams &p, int first, int step_, int rank_, int stage_elems, const int32_t *goffs_,
+                                         bool need_b_)
     {
-        tile = first; step = step_; rank = rank_; it = 0; goffs = goffs_;
+        tile = first; step = step_; rank = rank_; it = 0; goffs = goffs_; need_b = need_b_;
         seek(p, stage_elems);
     }
     __device__ __forceinline__ bool valid(const GemmParams &p) const { return tile < p.n_tile_total; }
@@ -1013,9 +1026,15 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         }
     }
     // grouped products: a 32-bit copy of the group boundaries for the per-tile lookups of every role
-    const bool goffs_ok = CTAS == 1 && p.mode != MODE_DENSE && p.n_groups <= kMaxGroupsShared;
-    if (goffs_ok)
+    const int n_row_tiles = (p.M + BM - 1) / BM;
+    const bool goffs_ok = Cfg<KIND, CTAS>::kSmemGroups > 0 &&
+                          ((p.mode == MODE_GROUPED_K && p.n_groups <= kMaxGroupsShared) ||
+                           (p.mode == MODE_GROUPED_ROWS && n_row_tiles <= kMaxRowTilesShared && p.n_groups <= 65535));
+    if (goffs_ok && p.mode == MODE_GROUPED_K)
         for (int g = threadIdx.x; g <= p.n_groups; g += kThreads) goffs_smem[g] = (int32_t)__ldg(p.row_offsets + g);
+    if (goffs_ok && p.mode == MODE_GROUPED_ROWS)
+        for (int i = threadIdx.x; i < n_row_tiles; i += kThreads)
+            reinterpret_cast<uint16_t *>(goffs_smem)[i] = (uint16_t)find_group(p.row_offsets, nullptr, p.n_groups, (int64_t)i * BM);
     const int32_t *goffs = goffs_ok ? goffs_smem : nullptr;
     tcgen05_fence_before();
     __syncwarp();
@@ -1032,7 +1051,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // more - and only then issues the loads of all slots found free, back to back.
         constexpr int kBatch = 3;
         StageIter pr;
-        pr.init(p, first_tile, tile_step, rank, kStageElems, goffs);
+        pr.init(p, first_tile, tile_step, rank, kStageElems, goffs, true);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         const bool issuer = elect_one();
@@ -1104,7 +1123,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_T0(tt);
         for (int tile = first_tile; leader && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, rank, t, goffs);
+            decode_tile(p, tile, rank, t, goffs, false);
             const int n_it = (t.k_len + kStageElems - 1) / kStageElems;
             if (n_it == 0) continue;
             TRACE_ADD(c_acc, tt);
@@ -1280,7 +1299,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // stage is released unseen, so that the MMA warp, which cannot time out on a named barrier, always runs
         // to its end.
         StageIter sg;
-        sg.init(p, first_tile, tile_step, rank, kStageElems, goffs);
+        sg.init(p, first_tile, tile_step, rank, kStageElems, goffs, false);
         uint32_t stage = 0, phase = 0, acc_phase = 0;
         BufRing ring;   // image buffer of the current unit
         bool ok = true;
@@ -1416,7 +1435,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_T0(tt);
         for (int tile = first_tile; ok && tile < p.n_tile_total; tile += tile_step) {
             Tile t;
-            decode_tile(p, tile, rank, t, goffs);
+            decode_tile(p, tile, rank, t, goffs, false);
             const int row_in_tile = 32 * quarter + lane;
             const int64_t row = (int64_t)t.c_row0 + row_in_tile;
             const bool row_ok = row_in_tile < t.m_valid;
@@ -1733,10 +1752,11 @@ static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p
     // Dense products (FP4 and MXFP8) with more than one row tile run as cta_group::2 pairs: 256x256 tiles, each CTA
     // loads half of the B rows; so does the grouped weight gradient, whose groups cut the contraction axis, not the
     // output rows of a tile.  FP4Q_CTA_PAIRS=0 in the environment (read once, before the first GEMM call) selects
-    // the one-CTA kernel instead; grouped forward / input-gradient products (token groups are only 128-row aligned)
-    // always use one CTA per 128x256 tile.
+    // the one-CTA kernel instead; grouped forward / input-gradient products use one CTA per 128x256 tile unless the
+    // caller states that every token group starts on a multiple of 256 rows.
     static const bool use_pairs = [] { const char *e = getenv("FP4Q_CTA_PAIRS"); return !(e && e[0] == '0'); }();
-    if (use_pairs && (p.mode == MODE_DENSE || p.mode == MODE_GROUPED_K) && p.M > BM) return launch_gemm_impl<KIND, 2>(A, B, p, stream);
+    const bool pair_mode = p.mode == MODE_DENSE || p.mode == MODE_GROUPED_K || (p.mode == MODE_GROUPED_ROWS && p.rows_pair_aligned);
+    if (use_pairs && pair_mode && p.M > BM) return launch_gemm_impl<KIND, 2>(A, B, p, stream);
     return launch_gemm_impl<KIND, 1>(A, B, p, stream);
 }
 
@@ -1746,6 +1766,7 @@ static fp4q_status check_groups(const fp4q_groups *g)
 {
     if (!g) return FP4Q_OK;
     if (g->n_groups <= 0) return FP4Q_ERR_SHAPE;
+    if (g->row_alignment != 0 && g->row_alignment != 128 && g->row_alignment != 256) return FP4Q_ERR_UNSUPPORTED;
     if (!g->row_offsets) return FP4Q_ERR_NULL;
     return FP4Q_OK;
 }
@@ -1806,6 +1827,7 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
     dense_tiles(p);
     if (g) {
         p.mode = MODE_GROUPED_ROWS; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.rows_pair_aligned = g->row_alignment == 256;
         p.b_rows_per_group = (int32_t)N; p.b_k_per_group = 0;
     }
     return launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, ws_bytes, stream);
@@ -1876,6 +1898,7 @@ extern "C" fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor 
     dense_tiles(p);
     if (g) {
         p.mode = MODE_GROUPED_ROWS; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.rows_pair_aligned = g->row_alignment == 256;
         p.b_rows_per_group = 0; p.b_k_per_group = (int32_t)N;
     }
     return launch_gemm<KIND_MXF4>(operand_rm(dY), operand_t(W), p, ws, ws_bytes, stream);

@@ -173,8 +173,8 @@ def _deq_col(qt, c):
 
 # ----------------------------------------------------------------------------------------- grouped (MoE)
 
-def _moe_case(ws, E, H, F, counts, seed):
-    offs = workloads.padded_row_offsets(counts, 128)
+def _moe_case(ws, E, H, F, counts, seed, pad=128):
+    offs = workloads.padded_row_offsets(counts, pad)
     T = int(offs[-1])
     g = torch.Generator(device="cuda").manual_seed(seed)
     X = workloads.zero_padding_rows(torch.randn(T, H, generator=g, device="cuda").to(torch.bfloat16), counts, offs)
@@ -184,8 +184,8 @@ def _moe_case(ws, E, H, F, counts, seed):
     qw, wd = quantized(W, 1, seed, 0)
     qdy, dyd = quantized(dY, 1, seed, 2)
     d_offs = torch.from_numpy(offs).cuda()
-    y = binding.fp4q_gemm_fwd(qx, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws)
-    dx = binding.fp4q_gemm_dgrad(qdy, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws)
+    y = binding.fp4q_gemm_fwd(qx, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws, row_alignment=pad)
+    dx = binding.fp4q_gemm_dgrad(qdy, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws, row_alignment=pad)
     dw = binding.fp4q_gemm_wgrad(qdy, qx, dt=binding.OUT_F32, row_offsets=d_offs, ws=ws)
     torch.cuda.synchronize()
     assert binding.fp4q_workspace_status(ws) == 0
@@ -227,6 +227,15 @@ def test_grouped_expert_width_not_a_multiple_of_the_tile_and_accumulation(ws):
     got = acc.double().cpu().numpy()
     assert np.array_equal(got[2 * F:], np.full((F, H), 0.5))      # the empty expert adds nothing
     check(acc[:2 * F], ref[:2 * F], "grouped wgrad, accumulate")
+
+
+def test_grouped_with_groups_aligned_to_256_rows_runs_on_pairs(ws):
+    # the caller states that every group starts on a multiple of 256 rows: forward and input gradient then use the
+    # 256-row pair tiles; empty, tiny and uneven groups as above
+    _moe_case(ws, E=5, H=256, F=192, counts=np.array([130, 0, 1, 300, 128]), seed=15, pad=256)
+    cfg = workloads.CONFIG_MOE
+    counts = workloads.moe_routing(cfg, tokens=1024, experts=8)
+    _moe_case(ws, E=8, H=cfg.hidden, F=cfg.expert_ffn, counts=counts, seed=16, pad=256)
 
 
 def test_grouped_moe_shapes_reduced_expert_count(ws):
