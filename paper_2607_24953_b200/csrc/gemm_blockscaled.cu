@@ -85,13 +85,18 @@ struct Cfg {
     static constexpr bool kRowImages = KIND != KIND_MXF4;
     static constexpr int kImageBufs = (CTAS == 2 && kRowImages) ? 3 : 2;
     static constexpr int kRawBufs = kRowImages ? 2 : 0;
-    static constexpr int kStages = (CTAS == 2 ? 5 : 4) - (kRowImages ? 1 : 0);
+    // The output leaves through staging rows and TMA stores wherever shared memory allows (everything but the
+    // one-CTA kernel of the per-row kinds).  In the one-CTA kernel of the 2D kind - grouped products with short
+    // contractions - plain stores of the 64 KB tile filled the SM's path to L2 and the TMA loads issued meanwhile
+    // took 6500-8000 cycles instead of 3000; the staging costs that kernel its fourth ring stage.
+    static constexpr bool kTmaStores = CTAS == 2 || !kRowImages;
+    static constexpr int kStages = (CTAS == 2 ? 5 : (kTmaStores ? 3 : 4)) - (kRowImages ? 1 : 0);
     static constexpr int kSmemCache = kCompactBytes + (kImageBufs + kRawBufs) * kCacheBufBytes;
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
-    static constexpr int kSmemStaging = CTAS == 2 ? 8 * kStagingWarpBytes : 0;
+    static constexpr int kSmemStaging = kTmaStores ? 8 * kStagingWarpBytes : 0;
     static constexpr int kSmemGroups = (CTAS == 1 || KIND == KIND_MXF4) ? (kMaxGroupsShared + 1) * 4 : 0;   // grouped products: group table
     static_assert(kSmemGroups == 0 || kSmemGroups >= kMaxRowTilesShared * 2, "group table");
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail + kSmemGroups;
@@ -1011,7 +1016,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-        if (CTAS == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
+        if (Cfg<KIND, CTAS>::kTmaStores) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
         if (EPI == EPI_QUANT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
     }
     if (warp == 1) {
@@ -1547,8 +1552,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         bulk_commit();
                     }
                 }
-            } else if (CTAS == 2) {
-                // Pair kernel (dense products only): 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
+            } else if (Cfg<KIND, CTAS>::kTmaStores) {
+                // 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
                 // through this warp's staging rows and leave by a TMA store, which clips rows and columns past the
                 // output's edge.  With accumulation the store is the TMA's FP32 add-reduction.
                 if (t.m_valid > 32 * quarter) {
@@ -1587,7 +1592,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
-        if ((CTAS == 2 || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
+        if ((Cfg<KIND, CTAS>::kTmaStores || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
         if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
