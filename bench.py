@@ -321,9 +321,49 @@ def run_gpu(args):
                        "PCIe-bound"}
         del host_in, host_out
 
+    # ---- per-operand quantize and GEMM rates (each launch timed on its own; a weight that fits in L2 is evicted first
+    # by a write of a buffer larger than L2)
+    per_operand = None
+    if not args.no_extras and rank == 0:
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+        def timed_cold(fn, iters=5):
+            tot = 0.0
+            for _ in range(iters + 1):
+                flush.fill_(1)
+                a, b = ev(), ev()
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                tot += a.elapsed_time(b)
+                if _ == 0:
+                    tot = 0.0      # first call: warm-up
+            return tot / iters
+
+        q_rates = {}
+        names = ["W_" + o["name"] for o in ops] + ["X_" + k for k in xs] + ["dY_" + o["name"] for o in ops]
+        for (x, q, tid), nm in zip(quant_jobs, names):
+            ms = timed_cold(lambda: binding.fp4q_quantize2d(x, q, mode=SR, seed=seed, tensor_id=tid))
+            q_rates[nm] = {"shape": list(x.shape), "gbs": x.numel() * BYTES_PER_ELEMENT / (ms * 1e-3) / 1e9}
+        g_rates = {}
+        for i, o in enumerate(ops):
+            fl = 2.0 * T * o["N"] * o["K"]
+            y, dx, dw = outputs(o)
+            g_rates[o["name"]] = {
+                "T_N_K": [T, o["N"], o["K"]],
+                "fwd_tflops": fl / (timed_cold(lambda: binding.fp4q_gemm_fwd(q_x[o["x_key"]], q_w[i], out=y, ws=ws)) * 1e-3) / 1e12,
+                "dgrad_tflops": fl / (timed_cold(lambda: binding.fp4q_gemm_dgrad(q_dy[i], q_w[i], out=dx, ws=ws)) * 1e-3) / 1e12,
+                "wgrad_tflops": fl / (timed_cold(lambda: binding.fp4q_gemm_wgrad(q_dy[i], q_x[o["x_key"]], out=dw, dt=binding.OUT_F32, ws=ws)) * 1e-3) / 1e12}
+        per_operand = {"quantize": q_rates, "gemm": g_rates,
+                       "note": "one launch at a time, L2 flushed before each (256 MB written), mean of 5"}
+        del flush
+
     extras = {}
     if not args.no_extras:
         extras = run_extras(torch, binding, workloads, dev, ws)
+        if per_operand is not None:
+            extras["per_operand"] = per_operand
 
     if rank != 0:
         if dist is not None:
