@@ -303,3 +303,16 @@ def test_one_cta_kernel_for_dense_products():
                         "-k", "tiny_linear or ragged or exact_case or scale_layout or multi_tile"],
                        env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_group_descriptor_is_validated(ws):
+    x = workloads.weights(256, 64, 1, "cuda")
+    w = workloads.weights(64, 64, 2, "cuda")
+    qx, qw = binding.fp4q_quantize2d(x), binding.fp4q_quantize2d(w)
+    offs = torch.tensor([0, 256], dtype=torch.int64, device="cuda")
+    with pytest.raises(binding.Fp4qError):
+        binding.fp4q_gemm_fwd(qx, qw, row_offsets=offs, ws=ws, row_alignment=64)     # only 0, 128 and 256 are statements the library knows
+    y = binding.fp4q_gemm_fwd(qx, qw, row_offsets=offs, ws=ws, row_alignment=256)
+    y0 = binding.fp4q_gemm_fwd(qx, qw, ws=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y0)                                                       # one group = the dense product
