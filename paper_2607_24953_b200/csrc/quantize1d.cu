@@ -184,6 +184,173 @@ __global__ void __launch_bounds__(128) quantize1d_t_kernel(const __grid_constant
     }
 }
 
+// In-register transpose of an 8x8 matrix of nibbles: a[r] holds row r (nibble c = column c); on return a[c] holds
+// column c (nibble r = row r).
+__device__ __forceinline__ void transpose8x8_nibbles_1d(uint32_t a[8])
+{
+#pragma unroll
+    for (int r = 0; r < 4; r++) {   // swap 4x4 quadrants (16-bit halves between rows r and r+4)
+        const uint32_t lo = __byte_perm(a[r], a[r + 4], 0x5410), hi = __byte_perm(a[r], a[r + 4], 0x7632);
+        a[r] = lo; a[r + 4] = hi;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; q++) {   // swap 2x2 blocks (bytes between rows r and r+2)
+        const int r = (q & 1) + 4 * (q >> 1);
+        const uint32_t lo = __byte_perm(a[r], a[r + 2], 0x6240), hi = __byte_perm(a[r], a[r + 2], 0x7351);
+        a[r] = lo; a[r + 2] = hi;
+    }
+#pragma unroll
+    for (int r = 0; r < 8; r += 2) {  // swap single nibbles between rows r and r+1
+        const uint32_t lo = (a[r] & 0x0F0F0F0Fu) | ((a[r + 1] & 0x0F0F0F0Fu) << 4);
+        const uint32_t hi = ((a[r] >> 4) & 0x0F0F0F0Fu) | (a[r + 1] & 0xF0F0F0F0u);
+        a[r] = lo; a[r + 1] = hi;
+    }
+}
+
+// One row of 16 elements, each with its own column factor 2^(-e-14), through the scalar path (non-finite values).
+// (arguments by value, so that nothing of the caller's has to live in local memory)
+__device__ __noinline__ uint32_t round_half_row_scalar(uint4 raw, float4 inv_a, float4 inv_b)
+{
+    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+    const float inv[8] = {inv_a.x, inv_a.y, inv_a.z, inv_a.w, inv_b.x, inv_b.y, inv_b.z, inv_b.w};
+    uint32_t w = 0u;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const uint32_t lo = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] & 0xFFFFu, inv[2 * k], 0u);
+        const uint32_t hi = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] >> 16, inv[2 * k + 1], 0u);
+        w |= (lo | (hi << 4)) << (8 * k);
+    }
+    return w;
+}
+
+// The same encoding for tensors whose shape and alignment allow full 128x128 tiles (rows and cols multiples of 128,
+// 32-byte aligned rows): the access pattern of the 2D quantizer.  A CTA of 4 warps owns 128x128 elements, a warp 32
+// rows x 128 columns, a lane 8 rows x 16 columns (one 256-bit load per row).  A block is now one column of the warp's
+// 32 rows: the four lanes that share 16 columns reduce 16 column maxima with two shuffles of packed BF16 pairs, every
+// element is scaled by its own column's factor, and the payload leaves through the 8x8 nibble transpose and the
+// swizzled staging rows as 64 contiguous bytes per column; the four scale bytes of a column (one per warp) leave as
+// one 32-bit store.
+__global__ void __launch_bounds__(128, 4) quantize1d_t_tile_kernel(const __grid_constant__ Quant1dParams p)
+{
+    __shared__ uint4 qt_stage[128 * 4];      // 128 output rows (columns of x) x 64 B, 16-byte chunks XOR-swizzled
+    __shared__ uint32_t sc_stage[128];       // per column of x: the scale codes of the CTA's four row blocks
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = lane >> 3, rg = (lane >> 1) & 3, ch = lane & 1;
+    const int64_t grid_x = p.cols >> 7;
+    const int64_t bx = (int64_t)blockIdx.x % grid_x, by = (int64_t)blockIdx.x / grid_x;
+    const int64_t row0 = by * 128 + warp * 32 + rg * 8, col0 = bx * 128 + t * 32 + ch * 16;
+
+    uint32_t raw[8][8];
+    {
+        const uint16_t *src = p.x + row0 * p.ld_x + col0;
+#pragma unroll
+        for (int r = 0; r < 8; r++)
+            asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(raw[r][0]), "=r"(raw[r][1]), "=r"(raw[r][2]), "=r"(raw[r][3]), "=r"(raw[r][4]),
+                           "=r"(raw[r][5]), "=r"(raw[r][6]), "=r"(raw[r][7])
+                         : "l"(src + r * p.ld_x));
+    }
+    // column maxima over the lane's 8 rows, then over the four lanes (rg) that hold the other rows of the block
+    uint32_t m2[8];
+    bool nonfinite = false;
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        __nv_bfloat162 m = __float2bfloat162_rn(0.0f);
+#pragma unroll
+        for (int r = 0; r < 8; r++) m = __hmax2_nan(m, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r][k])));
+#pragma unroll
+        for (int sft = 2; sft <= 4; sft <<= 1) {
+            uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m), sft);
+            m = __hmax2_nan(m, *reinterpret_cast<__nv_bfloat162 *>(&other));
+        }
+        m2[k] = *reinterpret_cast<uint32_t *>(&m) & 0x7FFF7FFFu;
+        nonfinite |= (m2[k] & 0xFFFFu) >= 0x7F80u || (m2[k] >> 16) >= 0x7F80u;
+    }
+    const bool careful = __any_sync(0xFFFFFFFFu, nonfinite);   // warp-uniform: the shuffles below need every lane
+    if (careful) {   // maxima over the finite entries only
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            uint32_t lo = 0, hi = 0;
+#pragma unroll
+            for (int r = 0; r < 8; r++) {
+                const uint32_t a = raw[r][k] & 0x7FFFu, b = (raw[r][k] >> 16) & 0x7FFFu;
+                if (a < 0x7F80u && a > lo) lo = a;
+                if (b < 0x7F80u && b > hi) hi = b;
+            }
+#pragma unroll
+            for (int sft = 2; sft <= 4; sft <<= 1) {
+                const uint32_t ol = __shfl_xor_sync(0xFFFFFFFFu, lo, sft), oh = __shfl_xor_sync(0xFFFFFFFFu, hi, sft);
+                lo = ol > lo ? ol : lo;
+                hi = oh > hi ? oh : hi;
+            }
+            m2[k] = lo | (hi << 16);
+        }
+    }
+    uint32_t codes[4] = {0u, 0u, 0u, 0u};   // 16 scale codes, one byte each
+    float inv[16];
+#pragma unroll
+    for (int c = 0; c < 16; c++) {
+        const int code = scale_code_from_max((m2[c >> 1] >> (16 * (c & 1))) & 0x7FFFu);
+        codes[c >> 2] |= (uint32_t)code << (8 * (c & 3));
+        inv[c] = careful ? inv_scale_f16_aligned(code) : inv_scale(code);
+    }
+    if (rg == 0) {
+        uint8_t *sc = reinterpret_cast<uint8_t *>(sc_stage);
+#pragma unroll
+        for (int c = 0; c < 16; c++) sc[(32 * t + 16 * ch + c) * 4 + warp] = (uint8_t)(codes[c >> 2] >> (8 * (c & 3)));
+    }
+    // codes of the lane's 8 x 16 elements, nearest rounding: W[r][g] = nibbles of columns 8g .. 8g+7 of row r
+    uint32_t W[8][2];
+    if (!careful) {
+#pragma unroll
+        for (int r = 0; r < 8; r++) {
+#pragma unroll
+            for (int g = 0; g < 2; g++) {
+                uint32_t w = 0;
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const uint32_t word = raw[r][4 * g + e];
+                    const int c = 8 * g + 2 * e;
+                    w |= cvt_rn_e2m1x2(__uint_as_float(word & 0xFFFF0000u) * inv[c + 1], __uint_as_float(word << 16) * inv[c]) << (8 * e);
+                }
+                W[r][g] = w;
+            }
+        }
+    } else {   // rare: kept small and out of the hot loop's instruction footprint
+#pragma unroll
+        for (int r = 0; r < 8; r++) {
+#pragma unroll
+            for (int g = 0; g < 2; g++)
+                W[r][g] = round_half_row_scalar(make_uint4(raw[r][4 * g], raw[r][4 * g + 1], raw[r][4 * g + 2], raw[r][4 * g + 3]),
+                                                make_float4(inv[8 * g], inv[8 * g + 1], inv[8 * g + 2], inv[8 * g + 3]),
+                                                make_float4(inv[8 * g + 4], inv[8 * g + 5], inv[8 * g + 6], inv[8 * g + 7]));
+        }
+    }
+    // transposed payload: per lane two 8x8 nibble blocks -> 16 words (one per column, 8 rows each)
+    uint32_t *stage = reinterpret_cast<uint32_t *>(qt_stage);
+#pragma unroll
+    for (int g = 0; g < 2; g++) {
+        uint32_t a[8];
+#pragma unroll
+        for (int r = 0; r < 8; r++) a[r] = W[r][g];
+        transpose8x8_nibbles_1d(a);
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+            const int col_local = 32 * t + 16 * ch + 8 * g + c;
+            stage[col_local * 16 + (((warp ^ t) << 2) | rg)] = a[c];
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const int row_local = (threadIdx.x >> 2) + 32 * k;   // output row = column of x; its 32-column group is k
+        const int chunk = threadIdx.x & 3;                    // 32 rows of x = one source warp
+        const uint4 v = qt_stage[row_local * 4 + (chunk ^ k)];
+        *reinterpret_cast<uint4 *>(p.q + (bx * 128 + row_local) * p.ld_q + by * 64 + chunk * 16) = v;
+    }
+    *reinterpret_cast<uint32_t *>(p.scale + (bx * 128 + threadIdx.x) * p.ld_s + by * 4) = sc_stage[threadIdx.x];
+}
+
 }  // namespace fp4q
 
 using namespace fp4q;
@@ -228,6 +395,12 @@ extern "C" fp4q_status fp4q_quantize1d_t(const void *x_bf16, int64_t rows, int64
     p.rows = rows; p.cols = cols; p.ld_x = ld_x;
     p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
     p.x_vec_ok = aligned(x_bf16, 4) && ld_x % 2 == 0;
+    // full 128x128 tiles and aligned rows: the tile kernel (coalesced 64-byte column stores)
+    if (rows % 128 == 0 && cols % 128 == 0 && aligned(x_bf16, 32) && ld_x % 16 == 0 && ld_s % 4 == 0 && aligned(scale, 4) &&
+        (rows / 128) * (cols / 128) <= 0x7FFFFFFF) {
+        quantize1d_t_tile_kernel<<<(unsigned)((rows / 128) * (cols / 128)), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
+        return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    }
     const int64_t gx = ceil_div(cols, 64), gy = ceil_div(ceil_div(rows, 32), 4);
     if (gx > 0x7FFFFFFF || gy > 65535) return FP4Q_ERR_UNSUPPORTED;
     quantize1d_t_kernel<<<dim3((unsigned)gx, (unsigned)gy), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);

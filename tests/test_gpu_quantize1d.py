@@ -102,6 +102,22 @@ def test_ragged_and_nonfinite_transposed():
     check_transposed(bits_tensor(b))
 
 
+def test_transposed_tile_path_with_nonfinite_values_and_all_scale_codes():
+    # shapes made of full 128 x 128 tiles take the tile kernel: random bit patterns (every exponent), zero column
+    # blocks, +-Inf, NaN, a column block without a finite entry
+    rng = np.random.default_rng(6)
+    b = _random_finite_bits(rng, 256, 384)
+    check_transposed(bits_tensor(b))
+    b[3, 5] = 0x7F80
+    b[40, 70] = 0xFF80
+    b[100, 200] = 0x7FC1
+    b[128:160, 17] = 0
+    b[160:192, 18] = 0x8000
+    b[192:224, 19] = 0x7F80
+    check_transposed(bits_tensor(b))
+    check_transposed(workloads.activations_gauss_outliers(512, 256, seed=9, device="cuda"))
+
+
 def test_empty_and_rejected_arguments():
     e = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
     q, s = binding.fp4q_quantize1d(e)
