@@ -181,6 +181,117 @@ __global__ void __launch_bounds__(128) mxfp8_quantize1d_t_kernel(const __grid_co
     }
 }
 
+// The same encoding for tensors made of full 128x128 tiles with 32-byte aligned rows: the access pattern of the 2D
+// FP4 quantizer.  A CTA of 4 warps owns 128x128 elements, a warp 32 rows x 128 columns, a lane 8 rows x 16 columns (one
+// 256-bit load per row).  The four lanes that share 16 columns reduce the 16 column maxima of the warp's 32 rows with
+// two shuffles of packed BF16 pairs; one convert takes the same column of two consecutive rows, so a lane holds 8
+// payload bytes per column as they are stored; they cross 16 KB of shared memory (16-byte chunks XOR-swizzled by the
+// column's group) and leave as 128 contiguous bytes per column; the four scale bytes of a column as one word.
+__global__ void __launch_bounds__(128, 4) mxfp8_quantize1d_t_tile_kernel(const __grid_constant__ Mxfp8QuantParams p)
+{
+    __shared__ uint4 stage[128 * 8];         // 128 output rows (columns of x) x 128 B
+    __shared__ uint32_t sc_stage[128];       // per column of x: the scale codes of the CTA's four row blocks
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = lane >> 3, rg = (lane >> 1) & 3, ch = lane & 1;
+    const int64_t grid_x = p.cols >> 7;
+    const int64_t bx = (int64_t)blockIdx.x % grid_x, by = (int64_t)blockIdx.x / grid_x;
+    const int64_t row0 = by * 128 + warp * 32 + rg * 8, col0 = bx * 128 + t * 32 + ch * 16;
+
+    uint32_t raw[8][8];
+    {
+        const uint16_t *src = p.x + row0 * p.ld_x + col0;
+#pragma unroll
+        for (int r = 0; r < 8; r++)
+            asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(raw[r][0]), "=r"(raw[r][1]), "=r"(raw[r][2]), "=r"(raw[r][3]), "=r"(raw[r][4]),
+                           "=r"(raw[r][5]), "=r"(raw[r][6]), "=r"(raw[r][7])
+                         : "l"(src + r * p.ld_x));
+    }
+    uint32_t m2[8];
+    bool nonfinite = false;
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        __nv_bfloat162 m = __float2bfloat162_rn(0.0f);
+#pragma unroll
+        for (int r = 0; r < 8; r++) m = __hmax2_nan(m, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[r][k])));
+#pragma unroll
+        for (int sft = 2; sft <= 4; sft <<= 1) {
+            uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m), sft);
+            m = __hmax2_nan(m, *reinterpret_cast<__nv_bfloat162 *>(&other));
+        }
+        m2[k] = *reinterpret_cast<uint32_t *>(&m) & 0x7FFF7FFFu;
+        nonfinite |= (m2[k] & 0xFFFFu) >= 0x7F80u || (m2[k] >> 16) >= 0x7F80u;
+    }
+    const bool careful = __any_sync(0xFFFFFFFFu, nonfinite);   // warp-uniform: the shuffles below need every lane
+    if (careful) {   // maxima over the finite entries only; NaN -> +0 (+-Inf saturates in the conversion)
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            uint32_t lo = 0, hi = 0;
+#pragma unroll
+            for (int r = 0; r < 8; r++) {
+                const uint32_t a = raw[r][k] & 0x7FFFu, b = (raw[r][k] >> 16) & 0x7FFFu;
+                if (a < 0x7F80u && a > lo) lo = a;
+                if (b < 0x7F80u && b > hi) hi = b;
+                if (a > 0x7F80u) raw[r][k] &= 0xFFFF0000u;
+                if (b > 0x7F80u) raw[r][k] &= 0x0000FFFFu;
+            }
+#pragma unroll
+            for (int sft = 2; sft <= 4; sft <<= 1) {
+                const uint32_t ol = __shfl_xor_sync(0xFFFFFFFFu, lo, sft), oh = __shfl_xor_sync(0xFFFFFFFFu, hi, sft);
+                lo = ol > lo ? ol : lo;
+                hi = oh > hi ? oh : hi;
+            }
+            m2[k] = lo | (hi << 16);
+        }
+    }
+    uint32_t codes[4] = {0u, 0u, 0u, 0u};
+    float inv[16];
+#pragma unroll
+    for (int c = 0; c < 16; c++) {
+        const uint32_t fm = (m2[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;
+        const int be = (int)(fm >> 7), m7 = (int)(fm & 0x7F);
+        int code = be == 0 ? 0 : be - 8 + (m7 > 0x60 ? 1 : 0);   // smallest e with 448*2^e >= M
+        code = code < 0 ? 0 : code;
+        codes[c >> 2] |= (uint32_t)code << (8 * (c & 3));
+        inv[c] = __uint_as_float((uint32_t)(254 - code) << 23);
+    }
+    if (rg == 0) {
+        uint8_t *sc = reinterpret_cast<uint8_t *>(sc_stage);
+#pragma unroll
+        for (int c = 0; c < 16; c++) sc[(32 * t + 16 * ch + c) * 4 + warp] = (uint8_t)(codes[c >> 2] >> (8 * (c & 3)));
+    }
+    // per column the lane's 8 payload bytes (rows row0 .. row0 + 7), into the column's staging row
+#pragma unroll
+    for (int c = 0; c < 16; c++) {
+        uint32_t w[2];
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int e = 0; e < 2; e++) {
+                const int r = 4 * h + 2 * e;
+                const uint32_t w0 = raw[r][c >> 1], w1 = raw[r + 1][c >> 1];
+                const float v0 = __uint_as_float((c & 1) ? (w0 & 0xFFFF0000u) : (w0 << 16)) * inv[c];
+                const float v1 = __uint_as_float((c & 1) ? (w1 & 0xFFFF0000u) : (w1 << 16)) * inv[c];
+                acc |= cvt_rn_e4m3x2(v1, v0) << (16 * e);
+            }
+            w[h] = acc;
+        }
+        const int col_local = 32 * t + 16 * ch + c;
+        const int chunk = (warp * 2 + (rg >> 1)) ^ ((col_local >> 4) & 7);
+        reinterpret_cast<uint2 *>(stage)[(col_local * 8 + chunk) * 2 + (rg & 1)] = make_uint2(w[0], w[1]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+        const int row_local = (threadIdx.x >> 3) + 16 * k;   // output row = column of x
+        const int chunk = threadIdx.x & 7;                    // 16 source rows
+        const uint4 v = stage[row_local * 8 + (chunk ^ ((row_local >> 4) & 7))];
+        *reinterpret_cast<uint4 *>(p.q + (bx * 128 + row_local) * p.ld_q + by * 128 + chunk * 16) = v;
+    }
+    *reinterpret_cast<uint32_t *>(p.scale + (bx * 128 + threadIdx.x) * p.ld_s + by * 4) = sc_stage[threadIdx.x];
+}
+
 }  // namespace fp4q
 
 using namespace fp4q;
@@ -224,6 +335,12 @@ extern "C" fp4q_status fp4q_mxfp8_quantize1d_t(const void *x_bf16, int64_t rows,
     p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
     p.segs_per_row = 0;
     p.x_vec_ok = aligned(x_bf16, 4) && ld_x % 2 == 0;
+    // full 128x128 tiles and aligned rows: the tile kernel (coalesced 128-byte column stores)
+    if (rows % 128 == 0 && cols % 128 == 0 && aligned(x_bf16, 32) && ld_x % 16 == 0 && ld_s % 4 == 0 && aligned(scale, 4) &&
+        (rows / 128) * (cols / 128) <= 0x7FFFFFFF) {
+        mxfp8_quantize1d_t_tile_kernel<<<(unsigned)((rows / 128) * (cols / 128)), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);
+        return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+    }
     const int64_t gx = ceil_div(cols, 64), gy = ceil_div(ceil_div(rows, 32), 4);
     if (gx > 0x7FFFFFFF || gy > 65535) return FP4Q_ERR_UNSUPPORTED;
     mxfp8_quantize1d_t_kernel<<<dim3((unsigned)gx, (unsigned)gy), 128, 0, static_cast<cudaStream_t>(stream)>>>(p);

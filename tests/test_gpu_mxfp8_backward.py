@@ -76,3 +76,20 @@ def test_backward_products_of_an_mxfp8_projection(T, N, K):
     assert binding.fp4q_workspace_status(ws) == 0
     check(dx, dyd @ wtd.T, "dgrad")                 # dX[t,k] = sum_n dY^[t,n] W^T^[k,n]
     check(dw, dytd @ xtd.T, "wgrad")                # dW[n,k] = sum_t dY^T^[n,t] X^T^[k,t]
+
+
+def test_transposing_quantizer_tile_path_with_nonfinite_values():
+    # shapes made of full 128 x 128 tiles take the tile kernel: random bit patterns (every exponent), zero column
+    # blocks, +-Inf, NaN, a column block without a finite entry
+    rng = np.random.default_rng(16)
+    b = rng.integers(0, 1 << 16, size=(256, 384), dtype=np.uint32).astype(np.uint16)
+    b[(b & 0x7F80) == 0x7F80] &= 0xBFFF
+    quantize_t_checked(workloads.bits_to_bf16(b, "cuda"))
+    b[3, 5] = 0x7F80
+    b[40, 70] = 0xFF80
+    b[100, 200] = 0x7FC1
+    b[128:160, 17] = 0
+    b[160:192, 18] = 0x8000
+    b[192:224, 19] = 0x7F80
+    quantize_t_checked(workloads.bits_to_bf16(b, "cuda"))
+    quantize_t_checked(workloads.activations_gauss_outliers(512, 256, seed=9, device="cuda"))
