@@ -184,40 +184,17 @@ __global__ void __launch_bounds__(128) quantize1d_t_kernel(const __grid_constant
     }
 }
 
-// In-register transpose of an 8x8 matrix of nibbles: a[r] holds row r (nibble c = column c); on return a[c] holds
-// column c (nibble r = row r).
-__device__ __forceinline__ void transpose8x8_nibbles_1d(uint32_t a[8])
+// Eight consecutive rows of one column (two BF16 per word, low half = even row) through the scalar path, for blocks
+// that hold a non-finite value; inv = 2^(-e-14).  Arguments by value, so that nothing of the caller's has to live in
+// local memory.
+__device__ __noinline__ uint32_t round_column_scalar(uint4 rows, float inv)
 {
-#pragma unroll
-    for (int r = 0; r < 4; r++) {   // swap 4x4 quadrants (16-bit halves between rows r and r+4)
-        const uint32_t lo = __byte_perm(a[r], a[r + 4], 0x5410), hi = __byte_perm(a[r], a[r + 4], 0x7632);
-        a[r] = lo; a[r + 4] = hi;
-    }
-#pragma unroll
-    for (int q = 0; q < 4; q++) {   // swap 2x2 blocks (bytes between rows r and r+2)
-        const int r = (q & 1) + 4 * (q >> 1);
-        const uint32_t lo = __byte_perm(a[r], a[r + 2], 0x6240), hi = __byte_perm(a[r], a[r + 2], 0x7351);
-        a[r] = lo; a[r + 2] = hi;
-    }
-#pragma unroll
-    for (int r = 0; r < 8; r += 2) {  // swap single nibbles between rows r and r+1
-        const uint32_t lo = (a[r] & 0x0F0F0F0Fu) | ((a[r + 1] & 0x0F0F0F0Fu) << 4);
-        const uint32_t hi = ((a[r] >> 4) & 0x0F0F0F0Fu) | (a[r + 1] & 0xF0F0F0F0u);
-        a[r] = lo; a[r + 1] = hi;
-    }
-}
-
-// One row of 16 elements, each with its own column factor 2^(-e-14), through the scalar path (non-finite values).
-// (arguments by value, so that nothing of the caller's has to live in local memory)
-__device__ __noinline__ uint32_t round_half_row_scalar(uint4 raw, float4 inv_a, float4 inv_b)
-{
-    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-    const float inv[8] = {inv_a.x, inv_a.y, inv_a.z, inv_a.w, inv_b.x, inv_b.y, inv_b.z, inv_b.w};
+    const uint32_t r[4] = {rows.x, rows.y, rows.z, rows.w};
     uint32_t w = 0u;
 #pragma unroll
     for (int k = 0; k < 4; k++) {
-        const uint32_t lo = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] & 0xFFFFu, inv[2 * k], 0u);
-        const uint32_t hi = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] >> 16, inv[2 * k + 1], 0u);
+        const uint32_t lo = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] & 0xFFFFu, inv, 0u);
+        const uint32_t hi = quantize_scalar<FP4Q_ROUND_NEAREST>(r[k] >> 16, inv, 0u);
         w |= (lo | (hi << 4)) << (8 * k);
     }
     return w;
@@ -227,8 +204,9 @@ __device__ __noinline__ uint32_t round_half_row_scalar(uint4 raw, float4 inv_a, 
 // 32-byte aligned rows): the access pattern of the 2D quantizer.  A CTA of 4 warps owns 128x128 elements, a warp 32
 // rows x 128 columns, a lane 8 rows x 16 columns (one 256-bit load per row).  A block is now one column of the warp's
 // 32 rows: the four lanes that share 16 columns reduce 16 column maxima with two shuffles of packed BF16 pairs, every
-// element is scaled by its own column's factor, and the payload leaves through the 8x8 nibble transpose and the
-// swizzled staging rows as 64 contiguous bytes per column; the four scale bytes of a column (one per warp) leave as
+// element is scaled by its own column's factor, one convert takes the same column of two consecutive rows (its result
+// byte is a payload byte as it stands), and the payload leaves through swizzled staging rows as 64 contiguous bytes
+// per column; the four scale bytes of a column (one per warp) leave as
 // one 32-bit store.
 __global__ void __launch_bounds__(128, 4) quantize1d_t_tile_kernel(const __grid_constant__ Quant1dParams p)
 {
@@ -299,46 +277,33 @@ __global__ void __launch_bounds__(128, 4) quantize1d_t_tile_kernel(const __grid_
 #pragma unroll
         for (int c = 0; c < 16; c++) sc[(32 * t + 16 * ch + c) * 4 + warp] = (uint8_t)(codes[c >> 2] >> (8 * (c & 3)));
     }
-    // codes of the lane's 8 x 16 elements, nearest rounding: W[r][g] = nibbles of columns 8g .. 8g+7 of row r
-    uint32_t W[8][2];
-    if (!careful) {
-#pragma unroll
-        for (int r = 0; r < 8; r++) {
-#pragma unroll
-            for (int g = 0; g < 2; g++) {
-                uint32_t w = 0;
-#pragma unroll
-                for (int e = 0; e < 4; e++) {
-                    const uint32_t word = raw[r][4 * g + e];
-                    const int c = 8 * g + 2 * e;
-                    w |= cvt_rn_e2m1x2(__uint_as_float(word & 0xFFFF0000u) * inv[c + 1], __uint_as_float(word << 16) * inv[c]) << (8 * e);
-                }
-                W[r][g] = w;
-            }
-        }
-    } else {   // rare: kept small and out of the hot loop's instruction footprint
-#pragma unroll
-        for (int r = 0; r < 8; r++) {
-#pragma unroll
-            for (int g = 0; g < 2; g++)
-                W[r][g] = round_half_row_scalar(make_uint4(raw[r][4 * g], raw[r][4 * g + 1], raw[r][4 * g + 2], raw[r][4 * g + 3]),
-                                                make_float4(inv[8 * g], inv[8 * g + 1], inv[8 * g + 2], inv[8 * g + 3]),
-                                                make_float4(inv[8 * g + 4], inv[8 * g + 5], inv[8 * g + 6], inv[8 * g + 7]));
-        }
-    }
-    // transposed payload: per lane two 8x8 nibble blocks -> 16 words (one per column, 8 rows each)
+    // Per column the lane's 8 codes (rows row0 .. row0 + 7) as one word: one convert takes the same column of two
+    // consecutive rows, so its result byte is a payload byte of that column as it stands.
     uint32_t *stage = reinterpret_cast<uint32_t *>(qt_stage);
 #pragma unroll
-    for (int g = 0; g < 2; g++) {
-        uint32_t a[8];
+    for (int c = 0; c < 16; c++) {
+        uint32_t word = 0;
+        if (!careful) {
 #pragma unroll
-        for (int r = 0; r < 8; r++) a[r] = W[r][g];
-        transpose8x8_nibbles_1d(a);
+            for (int e = 0; e < 4; e++) {
+                const uint32_t w0 = raw[2 * e][c >> 1], w1 = raw[2 * e + 1][c >> 1];
+                const float v0 = __uint_as_float((c & 1) ? (w0 & 0xFFFF0000u) : (w0 << 16)) * inv[c];
+                const float v1 = __uint_as_float((c & 1) ? (w1 & 0xFFFF0000u) : (w1 << 16)) * inv[c];
+                word |= cvt_rn_e2m1x2(v1, v0) << (8 * e);
+            }
+        } else {   // rare: kept small and out of the hot loop's instruction footprint
+            uint32_t h[4];
 #pragma unroll
-        for (int c = 0; c < 8; c++) {
-            const int col_local = 32 * t + 16 * ch + 8 * g + c;
-            stage[col_local * 16 + (((warp ^ t) << 2) | rg)] = a[c];
+            for (int e = 0; e < 4; e++) {
+                const uint32_t w0 = raw[2 * e][c >> 1], w1 = raw[2 * e + 1][c >> 1];
+                h[e] = (c & 1) ? ((w0 >> 16) | (w1 & 0xFFFF0000u)) : ((w0 & 0xFFFFu) | (w1 << 16));
+            }
+            word = round_column_scalar(make_uint4(h[0], h[1], h[2], h[3]), inv[c]);
         }
+        const int col_local = 32 * t + 16 * ch + c;
+        // word index inside the 64-byte row: 4*(source warp) + rg, with the 16-byte chunk index XORed by the
+        // column's block index so that a warp's stores spread over the banks
+        stage[col_local * 16 + (((warp ^ t) << 2) | rg)] = word;
     }
     __syncthreads();
 #pragma unroll
