@@ -33,8 +33,16 @@ __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_cons
     const int64_t total = p.rows * p.segs_per_row;
     // whole warps stay in the shuffle below: total is a multiple of 2 and lanes pair as (even, odd)
     const bool active = gid < total;
-    const int64_t i = active ? gid / p.segs_per_row : 0;
-    const int64_t seg = active ? gid % p.segs_per_row : 0;
+    int64_t i = 0, seg = 0;
+    if (active) {
+        if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
+            i = (uint32_t)gid / (uint32_t)p.segs_per_row;
+            seg = (uint32_t)gid - (uint32_t)i * (uint32_t)p.segs_per_row;
+        } else {
+            i = gid / p.segs_per_row;
+            seg = gid - i * p.segs_per_row;
+        }
+    }
     const int64_t j0 = seg * 16;
 
     uint32_t raw[8];
@@ -57,16 +65,32 @@ __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_cons
         }
     }
 
-    // block maximum over finite magnitudes (BF16 magnitudes order like unsigned integers)
-    uint32_t fm = 0;
+    // block maximum: packed BF16 |.| max with NaN propagation; a non-finite entry sends the warp through the
+    // careful pass (maximum over the finite magnitudes, NaN -> +0; +-Inf saturates in the conversion)
+    __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int k = 0; k < 8; k++) {
-        const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
-        if (lo < 0x7F80u && lo > fm) fm = lo;
-        if (hi < 0x7F80u && hi > fm) fm = hi;
+    for (int k = 0; k < 8; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
+    {
+        uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), 1);
+        m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
     }
-    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, fm, 1);
-    fm = other > fm ? other : fm;
+    const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
+    uint32_t fm = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
+    const bool nonfinite = fm >= 0x7F80u;
+    if (__any_sync(0xFFFFFFFFu, nonfinite)) {
+        uint32_t f = 0;
+#pragma unroll
+        for (int k = 0; k < 8; k++) {
+            const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
+            if (lo < 0x7F80u && lo > f) f = lo;
+            if (hi < 0x7F80u && hi > f) f = hi;
+            if (lo > 0x7F80u) raw[k] &= 0xFFFF0000u;
+            if (hi > 0x7F80u) raw[k] &= 0x0000FFFFu;
+        }
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, f, 1);
+        f = other > f ? other : f;
+        if (nonfinite) fm = f;
+    }
 
     // smallest e with 448*2^e >= M: code = be - 8 + (m7 > 0x60), clamped at 0
     const int be = (int)(fm >> 7), m7 = (int)(fm & 0x7F);
@@ -85,9 +109,8 @@ __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_cons
         for (int h = 0; h < 2; h++) {
             const uint32_t word = raw[2 * w + h];
             const uint32_t lo = word << 16, hi = word & 0xFFFF0000u;
-            // NaN -> +0; +-Inf saturates to +-448 in the conversion
-            v[2 * h] = ((lo & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(lo) * inv;
-            v[2 * h + 1] = ((hi & 0x7FFFFFFFu) > 0x7F800000u) ? 0.0f : __uint_as_float(hi) * inv;
+            v[2 * h] = __uint_as_float(lo) * inv;          // NaN entries were zeroed above
+            v[2 * h + 1] = __uint_as_float(hi) * inv;
         }
         out[w] = cvt_rn_e4m3x2(v[1], v[0]) | (cvt_rn_e4m3x2(v[3], v[2]) << 16);
     }
