@@ -411,22 +411,27 @@ def run_gpu(args):
                          "bytes_per_launch": quant_bytes / len(quant_jobs), "ms_per_launch": q_ms / len(quant_jobs),
                          "time_share_of_step": q_ms / ms_per_step}
     if not args.no_graphs and not args.serial_quantize:
-        # the same sweep with its launches in one stream, one after the other, for comparison
+        # the sweep on its own (no GEMMs between repetitions, so at cooler clocks than inside the step), as captured
+        # for the step and with its launches in one stream, one after the other
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             phase_quantize()
-        g.replay()
-        torch.cuda.synchronize()
-        a, b = ev(), ev()
-        a.record()
-        for _ in range(10):
-            g.replay()
-        b.record()
-        torch.cuda.synchronize()
-        roofline_quantize["achieved_one_stream"] = quant_bytes / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
+
+        def sweep_rate(replay):
+            replay()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record()
+            for _ in range(10):
+                replay()
+            b.record()
+            torch.cuda.synchronize()
+            return quant_bytes / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
+
+        roofline_quantize["sweep_alone_gbs"] = {"two_streams": sweep_rate(phases[0]), "one_stream": sweep_rate(g.replay)}
         roofline_quantize["note"] = ("launches of independent operands overlap (two streams in the graph), so ms_per_launch is "
-                                     "the phase time divided by the launch count; achieved_one_stream is the same sweep with "
-                                     "its launches one after the other")
+                                     "the phase time divided by the launch count; sweep_alone_gbs compares the two captures "
+                                     "of the sweep run on their own")
     fill_traffic(roofline, roofline_quantize)
 
     cpu = cpu_baseline_quantize(workloads, cfg, seconds=args.cpu_seconds)
