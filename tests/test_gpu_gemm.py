@@ -316,3 +316,17 @@ def test_group_descriptor_is_validated(ws):
     y0 = binding.fp4q_gemm_fwd(qx, qw, ws=ws)
     torch.cuda.synchronize()
     assert torch.equal(y, y0)                                                       # one group = the dense product
+
+
+def test_seeded_random_shapes_all_three_products(ws):
+    # two dozen seeded shapes around the tile edges (one CTA / pairs, ragged rows, columns and contraction tails)
+    rng = np.random.default_rng(2024)
+    for n in range(24):
+        T = int(rng.choice([1, 31, 64, 127, 128, 129, 255, 256, 257, 300, 513, 640]))
+        N = int(rng.choice([8, 32, 96, 200, 256, 264, 512, 520, 768]))
+        K = int(rng.choice([32, 64, 96, 256, 288, 1000, 1024, 2080]))
+        g = torch.Generator(device="cuda").manual_seed(1000 + n)
+        W = (torch.randn(N, K, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+        X = torch.randn(T, K, generator=g, device="cuda").to(torch.bfloat16)
+        dY = (torch.randn(T, N, generator=g, device="cuda") * 1e-3).to(torch.bfloat16)
+        linear_layer_case(W, X, dY, seed=n, ws=ws, dt_fwd=binding.OUT_BF16 if n & 1 else binding.OUT_F32)
