@@ -330,3 +330,15 @@ def test_seeded_random_shapes_all_three_products(ws):
         X = torch.randn(T, K, generator=g, device="cuda").to(torch.bfloat16)
         dY = (torch.randn(T, N, generator=g, device="cuda") * 1e-3).to(torch.bfloat16)
         linear_layer_case(W, X, dY, seed=n, ws=ws, dt_fwd=binding.OUT_BF16 if n & 1 else binding.OUT_F32)
+
+
+def test_seeded_random_grouped_cases(ws):
+    # random expert counts (empty experts included), widths and paddings; both paddings run (pairs with 256)
+    rng = np.random.default_rng(77)
+    for n in range(8):
+        E = int(rng.integers(1, 7))
+        counts = rng.integers(0, 400, size=E)
+        counts[rng.integers(0, E)] = 0 if E > 1 else counts[0]
+        H = int(rng.choice([64, 256, 320, 1024]))
+        F = int(rng.choice([64, 128, 192, 448]))
+        _moe_case(ws, E=E, H=H, F=F, counts=counts, seed=200 + n, pad=128 if n & 1 else 256)

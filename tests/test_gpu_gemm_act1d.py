@@ -127,3 +127,25 @@ def test_full_size_attention_projection_sampled_rows():
     oq_t, os_t = oracle.quantize1d(np.ascontiguousarray(workloads.bf16_bits(x[:, torch.from_numpy(sample_cols).cuda()]).T))
     assert np.array_equal(xtq.cpu().numpy()[sample_cols, :T // 2], oq_t) and np.array_equal(xts.cpu().numpy()[sample_cols], os_t)
     check(dw[torch.from_numpy(ncols).cuda()], dyd.T @ xt_hat.T, "wgrad sample, 1D activations")
+
+
+def test_seeded_random_shapes_with_1d_activations():
+    rng = np.random.default_rng(31)
+    ws = binding.alloc_workspace("cuda")
+    for n in range(10):
+        T = int(rng.choice([1, 96, 128, 129, 256, 300, 513]))
+        N = int(rng.choice([32, 200, 256, 264, 512]))
+        K = int(rng.choice([32, 96, 256, 288, 1000, 1024, 2080]))
+        x = workloads.activations_gauss_outliers(T, K, seed=40 + n, device="cuda")
+        w = workloads.weights(N, K, seed=60 + n, device="cuda")
+        dy = workloads.gradients_rowscaled(T, N, seed=80 + n, device="cuda")
+        xq, xs, x_hat = act1d(x)
+        xtq, xts, x_hat_t = act1d_t(x)
+        W = assert_matches_oracle(w, binding.ROUND_NEAREST, seed=0, tensor_id=0)
+        dY = assert_matches_oracle(dy, binding.ROUND_STOCHASTIC, seed=n, tensor_id=2)
+        y = binding.fp4q_gemm_fwd_act1d(xq, xs, T, W, dt=binding.OUT_BF16 if n & 1 else binding.OUT_F32, ws=ws)
+        dw = binding.fp4q_gemm_wgrad_act1d(dY, xtq, xts, K, dt=binding.OUT_F32, ws=ws)
+        torch.cuda.synchronize()
+        assert binding.fp4q_workspace_status(ws) == 0
+        check(y, oracle.gemm_fwd(x_hat, dequant_from_gpu(W)), "forward, 1D activations, shape %d" % n)
+        check(dw, oracle.gemm_wgrad(dequant_from_gpu(dY), x_hat_t), "wgrad, 1D activations, shape %d" % n)
