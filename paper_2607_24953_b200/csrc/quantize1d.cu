@@ -27,88 +27,79 @@ struct Quant1dParams {
     PhiloxRoundKeys keys;
 };
 
-// Each thread owns 16 consecutive elements of a row (two 128-bit loads, one 64-bit store); two neighbouring lanes
-// own one 32-element block and exchange their maxima with one shuffle.
+// Each thread owns one whole block of 32 consecutive elements of a row (four 128-bit loads, one 128-bit store): no
+// exchange between lanes, and the index arithmetic, the scale code and the scale store are paid once per block.
 template <int MODE>
 __global__ void __launch_bounds__(256) quantize1d_kernel(const __grid_constant__ Quant1dParams p)
 {
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t total = p.rows * p.segs_per_row;
-    const bool active = gid < total;   // whole warps stay in the shuffle below (total is even, lanes pair up)
-    int64_t i = 0, seg = 0;
-    if (active) {
-        if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
-            i = (uint32_t)gid / (uint32_t)p.segs_per_row;
-            seg = (uint32_t)gid - (uint32_t)i * (uint32_t)p.segs_per_row;
-        } else {
-            i = gid / p.segs_per_row;
-            seg = gid - i * p.segs_per_row;
-        }
+    const int64_t blocks_per_row = p.segs_per_row >> 1, total = p.rows * blocks_per_row;
+    if (gid >= total) return;
+    int64_t i, blk;
+    if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
+        i = (uint32_t)gid / (uint32_t)blocks_per_row;
+        blk = (uint32_t)gid - (uint32_t)i * (uint32_t)blocks_per_row;
+    } else {
+        i = gid / blocks_per_row;
+        blk = gid - i * blocks_per_row;
     }
-    const int64_t j0 = seg * 16;
+    const int64_t j0 = blk * 32;
 
-    uint32_t raw[8];
+    uint32_t raw[16];
+    const uint16_t *src = p.x + i * p.ld_x + j0;
+    if (p.x_vec_ok && j0 + 32 <= p.cols) {
 #pragma unroll
-    for (int k = 0; k < 8; k++) raw[k] = 0u;
-    if (active && j0 < p.cols) {
-        const uint16_t *src = p.x + i * p.ld_x + j0;
-        if (p.x_vec_ok && j0 + 16 <= p.cols) {
-            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
-            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
-            raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
-            raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
-        } else {
+        for (int q = 0; q < 4; q++) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src) + q);
+            raw[4 * q] = a.x; raw[4 * q + 1] = a.y; raw[4 * q + 2] = a.z; raw[4 * q + 3] = a.w;
+        }
+    } else {
 #pragma unroll
-            for (int k = 0; k < 8; k++) {
-                const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
-                const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
-                raw[k] = lo | (hi << 16);
-            }
+        for (int k = 0; k < 16; k++) {
+            const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
+            const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
+            raw[k] = lo | (hi << 16);
         }
     }
     // block maximum: packed BF16 |.| max with NaN propagation, so that any non-finite entry shows up in the
     // result and routes the block to the scalar path
     __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int k = 0; k < 8; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
-    {
-        uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), 1);
-        m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
-    }
+    for (int k = 0; k < 16; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
     const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
     uint32_t fm = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
     const bool nonfinite = fm >= 0x7F80u;
-    if (__any_sync(0xFFFFFFFFu, nonfinite)) {   // maximum over the finite entries only
-        uint32_t f = 0;
+    if (nonfinite) {   // maximum over the finite entries only
+        fm = 0;
 #pragma unroll
-        for (int k = 0; k < 8; k++) {
+        for (int k = 0; k < 16; k++) {
             const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
-            if (lo < 0x7F80u && lo > f) f = lo;
-            if (hi < 0x7F80u && hi > f) f = hi;
+            if (lo < 0x7F80u && lo > fm) fm = lo;
+            if (hi < 0x7F80u && hi > fm) fm = hi;
         }
-        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, f, 1);
-        f = other > f ? other : f;
-        if (nonfinite) fm = f;
     }
     const int code = scale_code_from_max(fm);
-    if (!active) return;
-    if ((seg & 1) == 0) p.scale[i * p.ld_s + (seg >> 1)] = (uint8_t)code;
+    p.scale[i * p.ld_s + blk] = (uint8_t)code;
 
-    uint32_t R[4] = {0u, 0u, 0u, 0u};
-    if (MODE == FP4Q_ROUND_STOCHASTIC) {   // cols % 16 == 0: the segment is one Philox block
-        const uint64_t blk = (uint64_t)(i * p.cols + j0) >> 4;
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), p.tensor_id, 0u, p.keys, R);
+    uint32_t W[4];
+#pragma unroll
+    for (int h = 0; h < 2; h++) {   // the block's two 16-element segments (one Philox block each: cols % 16 == 0)
+        uint32_t R[4] = {0u, 0u, 0u, 0u};
+        if (MODE == FP4Q_ROUND_STOCHASTIC) {
+            const uint64_t pb = (uint64_t)(i * p.cols + j0 + 16 * h) >> 4;
+            philox4x32_10((uint32_t)pb, (uint32_t)(pb >> 32), p.tensor_id, 0u, p.keys, R);
+        }
+        if (!nonfinite) {
+            round_segment<MODE>(raw + 8 * h, inv_scale(code), R, W + 2 * h);
+        } else {
+            const uint2 w = round_segment_scalar<MODE>(make_uint4(raw[8 * h], raw[8 * h + 1], raw[8 * h + 2], raw[8 * h + 3]),
+                                                       make_uint4(raw[8 * h + 4], raw[8 * h + 5], raw[8 * h + 6], raw[8 * h + 7]),
+                                                       make_uint4(R[0], R[1], R[2], R[3]), inv_scale_f16_aligned(code));
+            W[2 * h] = w.x;
+            W[2 * h + 1] = w.y;
+        }
     }
-    uint32_t W[2];
-    if (!nonfinite) {
-        round_segment<MODE>(raw, inv_scale(code), R, W);
-    } else {
-        const uint2 w = round_segment_scalar<MODE>(make_uint4(raw[0], raw[1], raw[2], raw[3]), make_uint4(raw[4], raw[5], raw[6], raw[7]),
-                                                   make_uint4(R[0], R[1], R[2], R[3]), inv_scale_f16_aligned(code));
-        W[0] = w.x;
-        W[1] = w.y;
-    }
-    *reinterpret_cast<uint2 *>(p.q + i * p.ld_q + (j0 >> 1)) = make_uint2(W[0], W[1]);
+    *reinterpret_cast<uint4 *>(p.q + i * p.ld_q + (j0 >> 1)) = make_uint4(W[0], W[1], W[2], W[3]);
 }
 
 // The encoding of x^T, nearest rounding.  A warp owns 32 rows x 64 columns: each row is one coalesced 128-byte load,
@@ -339,7 +330,7 @@ extern "C" fp4q_status fp4q_quantize1d(const void *x_bf16, int64_t rows, int64_t
     p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
     p.tensor_id = tensor_id;
     philox_round_keys(seed, p.keys);
-    const int64_t n_cta = ceil_div(rows * p.segs_per_row, 256);
+    const int64_t n_cta = ceil_div(rows * (p.segs_per_row / 2), 256);
     if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (mode == FP4Q_ROUND_STOCHASTIC) quantize1d_kernel<FP4Q_ROUND_STOCHASTIC><<<(unsigned)n_cta, 256, 0, s>>>(p);
