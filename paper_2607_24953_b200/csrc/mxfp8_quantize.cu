@@ -1,7 +1,6 @@
 // fp4q_mxfp8_quantize1d: BF16 -> MXFP8 operand (E4M3 payload, one UE8M0 scale per 32 consecutive
 // elements of a row), the operand format of the query/key projections.  Streaming kernel: each
-// thread owns 16 consecutive elements (two 128-bit loads, one 128-bit store); two neighbouring
-// lanes own one 32-element block and exchange their maxima with one shuffle.
+// thread owns one block of 32 consecutive elements (four 128-bit loads, two 128-bit stores).
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -29,67 +28,54 @@ __device__ __forceinline__ uint32_t cvt_rn_e4m3x2(float hi, float lo)
 
 __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_constant__ Mxfp8QuantParams p)
 {
+    // one whole block of 32 elements per thread: four 128-bit loads, two 128-bit stores, no exchange between lanes
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t total = p.rows * p.segs_per_row;
-    // whole warps stay in the shuffle below: total is a multiple of 2 and lanes pair as (even, odd)
-    const bool active = gid < total;
-    int64_t i = 0, seg = 0;
-    if (active) {
-        if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
-            i = (uint32_t)gid / (uint32_t)p.segs_per_row;
-            seg = (uint32_t)gid - (uint32_t)i * (uint32_t)p.segs_per_row;
-        } else {
-            i = gid / p.segs_per_row;
-            seg = gid - i * p.segs_per_row;
-        }
+    const int64_t blocks_per_row = p.segs_per_row >> 1, total = p.rows * blocks_per_row;
+    if (gid >= total) return;
+    int64_t i, blk;
+    if (total <= 0x7FFFFFFF) {   // 32-bit division is several times cheaper than the 64-bit one
+        i = (uint32_t)gid / (uint32_t)blocks_per_row;
+        blk = (uint32_t)gid - (uint32_t)i * (uint32_t)blocks_per_row;
+    } else {
+        i = gid / blocks_per_row;
+        blk = gid - i * blocks_per_row;
     }
-    const int64_t j0 = seg * 16;
+    const int64_t j0 = blk * 32;
 
-    uint32_t raw[8];
+    uint32_t raw[16];
+    const uint16_t *src = p.x + i * p.ld_x + j0;
+    if (p.x_vec_ok && j0 + 32 <= p.cols) {
 #pragma unroll
-    for (int k = 0; k < 8; k++) raw[k] = 0u;
-    if (active && j0 < p.cols) {
-        const uint16_t *src = p.x + i * p.ld_x + j0;
-        if (p.x_vec_ok && j0 + 16 <= p.cols) {
-            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src));
-            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(src) + 1);
-            raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
-            raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
-        } else {
+        for (int q = 0; q < 4; q++) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4 *>(src) + q);
+            raw[4 * q] = a.x; raw[4 * q + 1] = a.y; raw[4 * q + 2] = a.z; raw[4 * q + 3] = a.w;
+        }
+    } else {
 #pragma unroll
-            for (int k = 0; k < 8; k++) {
-                const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
-                const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
-                raw[k] = lo | (hi << 16);
-            }
+        for (int k = 0; k < 16; k++) {
+            const uint32_t lo = (j0 + 2 * k < p.cols) ? (uint32_t)__ldg(src + 2 * k) : 0u;
+            const uint32_t hi = (j0 + 2 * k + 1 < p.cols) ? (uint32_t)__ldg(src + 2 * k + 1) : 0u;
+            raw[k] = lo | (hi << 16);
         }
     }
 
-    // block maximum: packed BF16 |.| max with NaN propagation; a non-finite entry sends the warp through the
+    // block maximum: packed BF16 |.| max with NaN propagation; a non-finite entry sends the thread through the
     // careful pass (maximum over the finite magnitudes, NaN -> +0; +-Inf saturates in the conversion)
     __nv_bfloat162 m2 = __float2bfloat162_rn(0.0f);
 #pragma unroll
-    for (int k = 0; k < 8; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
-    {
-        uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, *reinterpret_cast<uint32_t *>(&m2), 1);
-        m2 = __hmax2_nan(m2, *reinterpret_cast<__nv_bfloat162 *>(&other));
-    }
+    for (int k = 0; k < 16; k++) m2 = __hmax2_nan(m2, __habs2(*reinterpret_cast<const __nv_bfloat162 *>(&raw[k])));
     const __nv_bfloat16 m1 = __hmax_nan(m2.x, m2.y);
     uint32_t fm = (uint32_t)(*reinterpret_cast<const uint16_t *>(&m1)) & 0x7FFFu;
-    const bool nonfinite = fm >= 0x7F80u;
-    if (__any_sync(0xFFFFFFFFu, nonfinite)) {
-        uint32_t f = 0;
+    if (fm >= 0x7F80u) {
+        fm = 0;
 #pragma unroll
-        for (int k = 0; k < 8; k++) {
+        for (int k = 0; k < 16; k++) {
             const uint32_t lo = raw[k] & 0x7FFFu, hi = (raw[k] >> 16) & 0x7FFFu;
-            if (lo < 0x7F80u && lo > f) f = lo;
-            if (hi < 0x7F80u && hi > f) f = hi;
+            if (lo < 0x7F80u && lo > fm) fm = lo;
+            if (hi < 0x7F80u && hi > fm) fm = hi;
             if (lo > 0x7F80u) raw[k] &= 0xFFFF0000u;
             if (hi > 0x7F80u) raw[k] &= 0x0000FFFFu;
         }
-        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, f, 1);
-        f = other > f ? other : f;
-        if (nonfinite) fm = f;
     }
 
     // smallest e with 448*2^e >= M: code = be - 8 + (m7 > 0x60), clamped at 0
@@ -97,24 +83,18 @@ __global__ void __launch_bounds__(256) mxfp8_quantize1d_kernel(const __grid_cons
     int code = be == 0 ? 0 : be - 8 + (m7 > 0x60 ? 1 : 0);
     code = code < 0 ? 0 : code;
     const float inv = __uint_as_float((uint32_t)(254 - code) << 23);   // 2^(127-code) = 2^-e
+    p.scale[i * p.ld_s + blk] = (uint8_t)code;
 
-    if (!active) return;
-    if ((seg & 1) == 0) p.scale[i * p.ld_s + (seg >> 1)] = (uint8_t)code;
-
-    uint32_t out[4];
+    uint32_t out[8];
 #pragma unroll
-    for (int w = 0; w < 4; w++) {
-        float v[4];
-#pragma unroll
-        for (int h = 0; h < 2; h++) {
-            const uint32_t word = raw[2 * w + h];
-            const uint32_t lo = word << 16, hi = word & 0xFFFF0000u;
-            v[2 * h] = __uint_as_float(lo) * inv;          // NaN entries were zeroed above
-            v[2 * h + 1] = __uint_as_float(hi) * inv;
-        }
-        out[w] = cvt_rn_e4m3x2(v[1], v[0]) | (cvt_rn_e4m3x2(v[3], v[2]) << 16);
+    for (int w = 0; w < 8; w++) {
+        const uint32_t w0 = raw[2 * w], w1 = raw[2 * w + 1];
+        out[w] = cvt_rn_e4m3x2(__uint_as_float(w0 & 0xFFFF0000u) * inv, __uint_as_float(w0 << 16) * inv) |
+                 (cvt_rn_e4m3x2(__uint_as_float(w1 & 0xFFFF0000u) * inv, __uint_as_float(w1 << 16) * inv) << 16);
     }
-    *reinterpret_cast<uint4 *>(p.q + i * p.ld_q + j0) = make_uint4(out[0], out[1], out[2], out[3]);
+    uint4 *dst = reinterpret_cast<uint4 *>(p.q + i * p.ld_q + j0);
+    dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+    dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
 }
 
 // The transpose of the same operand: q_t[j, i] = E4M3 of x[i, j] with one scale per column j and 32 consecutive rows i
@@ -335,7 +315,7 @@ extern "C" fp4q_status fp4q_mxfp8_quantize1d(const void *x_bf16, int64_t rows, i
     p.q = q; p.ld_q = ld_q; p.scale = scale; p.ld_s = ld_s;
     p.segs_per_row = round_up(cols, 32) / 16;
     p.x_vec_ok = aligned(x_bf16, 16) && ld_x % 8 == 0;
-    const int64_t total = rows * p.segs_per_row;
+    const int64_t total = rows * (p.segs_per_row / 2);
     const int64_t n_cta = ceil_div(total, 256);
     if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
     mxfp8_quantize1d_kernel<<<(unsigned)n_cta, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
