@@ -146,8 +146,8 @@ class QTensor:
     scale: torch.Tensor              # uint8 [ceil(rows/32), ld_s] ([ceil(rows/16), ld_s] after BLOCK_16)
     scale_granularity: int = 32      # 16 only for tensors quantized with BLOCK_16, which the GEMMs cannot take
 
-    def c_struct(self) -> _CTensor:
-        if self.scale_granularity != 32 and not getattr(self, "_quantizing", False):
+    def c_struct(self, as_quantizer_output: bool = False) -> _CTensor:
+        if self.scale_granularity != 32 and not as_quantizer_output:
             raise ValueError("a tensor quantized in 16 x 16 blocks is not a GEMM operand (the hardware's scale vectors are 32 wide)")
         return _CTensor(self.rows, self.cols,
                         self.q_rm.data_ptr(), self.q_rm.stride(0),
@@ -180,11 +180,7 @@ def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = 
     rows, cols = x.shape
     if out is None:
         out = alloc_qtensor(rows, cols, x.device, want_t, 16 if flags & BLOCK_16 else 32)
-    out._quantizing = True
-    try:
-        cs = out.c_struct()
-    finally:
-        out._quantizing = False
+    cs = out.c_struct(as_quantizer_output=True)
     st = lib().fp4q_quantize2d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, ctypes.byref(cs),
                                mode, seed, tensor_id, flags, _stream(stream))
     _check(st, "fp4q_quantize2d")
