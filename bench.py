@@ -604,6 +604,13 @@ def run_extras(torch, binding, workloads, dev, ws):
             res[name] = {"fwd_tflops": flops / (ms[0] * 1e-3) / 1e12, "dgrad_tflops": flops / (ms[1] * 1e-3) / 1e12,
                          "wgrad_tflops": flops / (ms[2] * 1e-3) / 1e12, "ms": ms,
                          "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9}
+            if pad == 256:   # forward product with the output quantization in the epilogue, against product + quantize
+                qy = binding.alloc_qtensor(Tp, n, dev)
+                ms_fq = timed(lambda: binding.fp4q_gemm_fwd_quantized(qx, qw, out=qy, mode=1, seed=1, tensor_id=9, ws=ws, row_offsets=d_offs))
+                ms_q = timed(lambda: binding.fp4q_quantize2d(y, out=qy, mode=1, seed=1, tensor_id=9))
+                res[name]["fwd_quantized_ms"] = ms_fq
+                res[name]["fwd_quantized_speedup_vs_unfused"] = (ms[0] + ms_q) / ms_fq
+                del qy
             tot_ms += sum(ms)
             tot_flops += 3 * flops
             del Xm, dYm, Wm, qx, qw, qdy, y, dx, dw

@@ -265,10 +265,12 @@ fp4q_status fp4q_mxfp8_gemm(const uint8_t *aq, int64_t ld_aq, const uint8_t *as,
  *   maxima, scales, codes, both payload layouts; Y itself is never written.
  * X [T,K], W [N,K] as for fp4q_gemm_fwd (dense form).  Yq: rows = T, cols = N, layouts and alignment as for
  * fp4q_quantize2d (q_t may be NULL).  N must be a multiple of 16 (FP4Q_ERR_UNSUPPORTED otherwise); T is free.
+ * Grouped form (g != NULL; NULL = dense): as fp4q_gemm_fwd, with g->row_alignment = 256 required (the epilogue lives
+ * in the CTA-pair kernel, whose tiles span 256 rows; FP4Q_ERR_UNSUPPORTED otherwise).
  * ws/ws_bytes/stream and the asynchronous FP4Q_ERR_TIMEOUT report are those of fp4q_gemm_fwd.
  */
 fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, const fp4q_tensor *Yq,
-                                    fp4q_round mode, uint64_t seed, uint32_t tensor_id,
+                                    fp4q_round mode, uint64_t seed, uint32_t tensor_id, const fp4q_groups *g,
                                     void *ws, size_t ws_bytes, void *stream);
 
 /*
@@ -277,10 +279,11 @@ fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, 
  * i*K + j): the layer's dX is the previous layer's dY, which the backward pass quantizes with stochastic rounding
  * (Section 3.1), so that quantization can happen here and dX never reaches memory in BF16.
  * dY [T,N] (row-major payload used), W [N,K] (transposed payload used) as for fp4q_gemm_dgrad (dense form).
- * dXq: rows = T, cols = K (multiple of 16), otherwise as Yq of fp4q_gemm_fwd_quantized; errors as there.
+ * dXq: rows = T, cols = K (multiple of 16), otherwise as Yq of fp4q_gemm_fwd_quantized; errors and grouped form as
+ * there (W then is the stack [n_groups*N, K], N a multiple of 64).
  */
 fp4q_status fp4q_gemm_dgrad_quantized(const fp4q_tensor *dY, const fp4q_tensor *W, const fp4q_tensor *dXq,
-                                      fp4q_round mode, uint64_t seed, uint32_t tensor_id,
+                                      fp4q_round mode, uint64_t seed, uint32_t tensor_id, const fp4q_groups *g,
                                       void *ws, size_t ws_bytes, void *stream);
 
 /*

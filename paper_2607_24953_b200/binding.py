@@ -106,11 +106,11 @@ def lib() -> ctypes.CDLL:
                                           ctypes.c_size_t, vp]
         if hasattr(L, "fp4q_gemm_dgrad_quantized"):
             L.fp4q_gemm_dgrad_quantized.restype = ci
-            L.fp4q_gemm_dgrad_quantized.argtypes = [vp, vp, vp, ci, u64, u32, vp, ctypes.c_size_t, vp]
+            L.fp4q_gemm_dgrad_quantized.argtypes = [vp, vp, vp, ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
         if hasattr(L, "fp4q_gemm_fwd_quantized"):
             L.fp4q_gemm_fwd_quantized.restype = ci
             L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
-                                                  ctypes.POINTER(_CTensor), ci, u64, u32, vp, ctypes.c_size_t, vp]
+                                                  ctypes.POINTER(_CTensor), ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -355,30 +355,36 @@ def fp4q_gemm_fwd(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, row_offs
 
 
 def fp4q_gemm_fwd_quantized(X: QTensor, W: QTensor, out: Optional[QTensor] = None, mode: int = ROUND_NEAREST,
-                            seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None) -> QTensor:
-    """Yq = 2D-block FP4 of the BF16-rounded product X^ W^^T, quantized in the GEMM's epilogue."""
+                            seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None,
+                            row_offsets=None) -> QTensor:
+    """Yq = 2D-block FP4 of the BF16-rounded product X^ W^^T, quantized in the GEMM's epilogue.  Grouped when
+    row_offsets is given (every group then starts on a multiple of 256 rows)."""
     dev = X.q_rm.device
+    g, gref = _groups(row_offsets, 256)
     if out is None:
-        out = alloc_qtensor(X.rows, W.rows, dev, want_t)
+        out = alloc_qtensor(X.rows, W.rows if row_offsets is None else W.rows // (row_offsets.numel() - 1), dev, want_t)
     if ws is None:
         ws = alloc_workspace(dev)
     cx, cw, cy = X.c_struct(), W.c_struct(), out.c_struct()
-    st = lib().fp4q_gemm_fwd_quantized(ctypes.byref(cx), ctypes.byref(cw), ctypes.byref(cy), mode, seed, tensor_id,
+    st = lib().fp4q_gemm_fwd_quantized(ctypes.byref(cx), ctypes.byref(cw), ctypes.byref(cy), mode, seed, tensor_id, gref,
                                        ws.data_ptr(), ws.numel(), _stream(stream))
     _check(st, "fp4q_gemm_fwd_quantized")
     return out
 
 
 def fp4q_gemm_dgrad_quantized(dY: QTensor, W: QTensor, out: Optional[QTensor] = None, mode: int = ROUND_STOCHASTIC,
-                              seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None) -> QTensor:
-    """dXq = 2D-block FP4 of the BF16-rounded product dY^ W^, quantized in the GEMM's epilogue."""
+                              seed: int = 0, tensor_id: int = 0, want_t: bool = True, ws=None, stream=None,
+                              row_offsets=None) -> QTensor:
+    """dXq = 2D-block FP4 of the BF16-rounded product dY^ W^, quantized in the GEMM's epilogue.  Grouped when
+    row_offsets is given (every group then starts on a multiple of 256 rows)."""
     dev = dY.q_rm.device
+    g, gref = _groups(row_offsets, 256)
     if out is None:
         out = alloc_qtensor(dY.rows, W.cols, dev, want_t)
     if ws is None:
         ws = alloc_workspace(dev)
     cd, cw, cx = dY.c_struct(), W.c_struct(), out.c_struct()
-    st = lib().fp4q_gemm_dgrad_quantized(ctypes.byref(cd), ctypes.byref(cw), ctypes.byref(cx), mode, seed, tensor_id,
+    st = lib().fp4q_gemm_dgrad_quantized(ctypes.byref(cd), ctypes.byref(cw), ctypes.byref(cx), mode, seed, tensor_id, gref,
                                          ws.data_ptr(), ws.numel(), _stream(stream))
     _check(st, "fp4q_gemm_dgrad_quantized")
     return out

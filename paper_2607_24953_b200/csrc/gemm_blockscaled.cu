@@ -1839,10 +1839,15 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
 }
 
 // C[M, N] = A B^T with the output leaving as the 2D-block FP4 tensor Cq (dense, pair kernel).
+// Grouped form (g != NULL): b_rows_per_group / b_k_per_group as in the plain grouped products; the pair tiles need
+// every group to start on a multiple of 256 rows.
 static fp4q_status launch_gemm_quantized(const Operand &A, const Operand &B, int64_t M, int64_t N, int64_t K, const fp4q_tensor *Cq,
-                                         fp4q_round mode, uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+                                         fp4q_round mode, uint64_t seed, uint32_t tensor_id, const fp4q_groups *g,
+                                         int32_t b_rows_per_group, int32_t b_k_per_group, void *ws, size_t ws_bytes, void *stream)
 {
     if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
+    if (fp4q_status s = check_groups(g)) return s;
+    if (g && g->row_alignment != 256) return FP4Q_ERR_UNSUPPORTED;
     if (Cq->rows != M || Cq->cols != N) return FP4Q_ERR_SHAPE;
     if (M > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
     if (N % 16 != 0) return FP4Q_ERR_UNSUPPORTED;   // one Philox block per 16-element row segment of the output
@@ -1865,23 +1870,35 @@ static fp4q_status launch_gemm_quantized(const Operand &A, const Operand &B, int
     p.q_scale = Cq->scale; p.q_ld_s = Cq->ld_s;
     p.q_mode = (int32_t)mode; p.q_tensor_id = tensor_id;
     philox_round_keys(seed, p.q_keys);
+    if (g) {
+        p.mode = MODE_GROUPED_ROWS; p.n_groups = g->n_groups; p.row_offsets = g->row_offsets;
+        p.rows_pair_aligned = 1;
+        p.b_rows_per_group = b_rows_per_group; p.b_k_per_group = b_k_per_group;
+    }
     return launch_gemm_impl<KIND_MXF4, 2, EPI_QUANT>(A, B, p, stream);
 }
 
 extern "C" fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, const fp4q_tensor *Yq, fp4q_round mode,
-                                               uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+                                               uint64_t seed, uint32_t tensor_id, const fp4q_groups *g, void *ws, size_t ws_bytes,
+                                               void *stream)
 {
     if (!tensor_ok(X) || !tensor_ok(W) || !tensor_ok(Yq)) return X && W && Yq ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
     if (X->cols != W->cols) return FP4Q_ERR_SHAPE;
-    return launch_gemm_quantized(operand_rm(X), operand_rm(W), X->rows, W->rows, X->cols, Yq, mode, seed, tensor_id, ws, ws_bytes, stream);
+    if (g && g->n_groups > 0 && (W->rows % g->n_groups || (W->rows / g->n_groups) % 32)) return FP4Q_ERR_SHAPE;
+    const int64_t N = g && g->n_groups > 0 ? W->rows / g->n_groups : W->rows;
+    return launch_gemm_quantized(operand_rm(X), operand_rm(W), X->rows, N, X->cols, Yq, mode, seed, tensor_id, g, (int32_t)N, 0, ws,
+                                 ws_bytes, stream);
 }
 
 extern "C" fp4q_status fp4q_gemm_dgrad_quantized(const fp4q_tensor *dY, const fp4q_tensor *W, const fp4q_tensor *dXq, fp4q_round mode,
-                                                 uint64_t seed, uint32_t tensor_id, void *ws, size_t ws_bytes, void *stream)
+                                                 uint64_t seed, uint32_t tensor_id, const fp4q_groups *g, void *ws, size_t ws_bytes,
+                                                 void *stream)
 {
     if (!tensor_ok(dY) || !tensor_ok(W) || !tensor_ok(dXq)) return dY && W && dXq ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
-    if (dY->cols != W->rows) return FP4Q_ERR_SHAPE;
-    return launch_gemm_quantized(operand_rm(dY), operand_t(W), dY->rows, W->cols, dY->cols, dXq, mode, seed, tensor_id, ws, ws_bytes, stream);
+    const int64_t N = dY->cols;
+    if (g && g->n_groups > 0 ? (W->rows != N * g->n_groups || N % 64) : (W->rows != N)) return FP4Q_ERR_SHAPE;
+    return launch_gemm_quantized(operand_rm(dY), operand_t(W), dY->rows, W->cols, N, dXq, mode, seed, tensor_id, g, 0, (int32_t)N, ws,
+                                 ws_bytes, stream);
 }
 
 extern "C" fp4q_status fp4q_gemm_dgrad(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt,

@@ -118,3 +118,38 @@ def test_fused_dgrad_exact_operands_match_the_oracle_bit_for_bit():
     dx_bits = workloads.bf16_bits(torch.from_numpy(dx).to(torch.bfloat16))
     o_rm, o_t, o_s = oracle.quantize2d(dx_bits, oracle.MODE_STOCHASTIC, 9, 4)
     compare_logical(dxq, o_rm, o_t, o_s, T, K)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_grouped_fused_products_equal_product_then_quantize(mode):
+    """The quantizing epilogue on grouped (mixture-of-experts) products, groups padded to 256 rows: forward and input
+    gradient against the plain grouped product followed by fp4q_quantize2d, bit for bit."""
+    E, H, F = 5, 256, 192
+    counts = np.array([130, 0, 1, 300, 128])
+    offs = workloads.padded_row_offsets(counts, 256)
+    T = int(offs[-1])
+    g = torch.Generator(device="cuda").manual_seed(21)
+    X = workloads.zero_padding_rows(torch.randn(T, H, generator=g, device="cuda").to(torch.bfloat16), counts, offs)
+    dY = workloads.zero_padding_rows((torch.randn(T, F, generator=g, device="cuda") * 0.01).to(torch.bfloat16), counts, offs)
+    W = (torch.randn(E * F, H, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    qx, qw = binding.fp4q_quantize2d(X), binding.fp4q_quantize2d(W)
+    qdy = binding.fp4q_quantize2d(dY, mode=1, seed=4, tensor_id=2)
+    d_offs = torch.from_numpy(offs).cuda()
+    ws = binding.alloc_workspace("cuda")
+    fused_y = binding.fp4q_gemm_fwd_quantized(qx, qw, mode=mode, seed=3, tensor_id=8, ws=ws, row_offsets=d_offs)
+    y = binding.fp4q_gemm_fwd(qx, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws, row_alignment=256)
+    chain_y = binding.fp4q_quantize2d(y.contiguous(), mode=mode, seed=3, tensor_id=8)
+    fused_dx = binding.fp4q_gemm_dgrad_quantized(qdy, qw, mode=mode, seed=5, tensor_id=9, ws=ws, row_offsets=d_offs)
+    dx = binding.fp4q_gemm_dgrad(qdy, qw, dt=binding.OUT_BF16, row_offsets=d_offs, ws=ws, row_alignment=256)
+    chain_dx = binding.fp4q_quantize2d(dx.contiguous(), mode=mode, seed=5, tensor_id=9)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    compare_logical(fused_y, *logical(chain_y), T, F)
+    compare_logical(fused_dx, *logical(chain_dx), T, H)
+    offs128 = torch.from_numpy(workloads.padded_row_offsets(counts, 128)).cuda()
+    with pytest.raises(binding.Fp4qError):      # the binding states 256-row alignment; the library refuses anything else
+        g128 = binding._CGroups(E, 128, offs128.data_ptr())
+        cx, cw, cy = qx.c_struct(), qw.c_struct(), fused_y.c_struct()
+        import ctypes
+        binding._check(binding.lib().fp4q_gemm_fwd_quantized(ctypes.byref(cx), ctypes.byref(cw), ctypes.byref(cy), 0, 0, 0,
+                                                             ctypes.byref(g128), ws.data_ptr(), ws.numel(), None), "fwd_quantized")
