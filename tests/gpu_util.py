@@ -49,3 +49,79 @@ def dequant_from_gpu(qt: binding.QTensor) -> np.ndarray:
     g_rm, _, g_s = logical(qt)
     return oracle.dequantize2d(np.ascontiguousarray(g_rm[:, :(qt.cols + 1) // 2]), np.ascontiguousarray(g_s),
                                qt.rows, qt.cols)
+
+
+def check_gemm(got: torch.Tensor, ref: np.ndarray, what=""):
+    """The GEMM tolerance of the build target: relative Frobenius error <= 1e-3 and, per output row,
+    max |G - O| <= 1e-2 * ||O_row||_inf.  BF16 outputs are compared with the oracle rounded to BF16."""
+    g = got.double().cpu().numpy()
+    if got.dtype == torch.bfloat16:
+        ref = oracle.bf16_round(ref)
+    assert g.shape == ref.shape, (g.shape, ref.shape)
+    denom = np.linalg.norm(ref)
+    rel = np.linalg.norm(g - ref) / denom if denom > 0 else np.abs(g).max()
+    assert rel <= 1e-3, "%s: relative Frobenius error %.3e" % (what, rel)
+    row_inf = np.abs(ref).max(axis=1, keepdims=True)
+    assert (np.abs(g - ref) <= 1e-2 * row_inf + 1e-300).all(), "%s: per-row max-abs bound violated" % what
+    return rel
+
+
+class HostQ:
+    """Host copy of a 2D-block-quantized tensor; rows and columns are decoded with the oracle's decoder and
+    value table (row-major payload for rows, transposed payload for columns, so both layouts are exercised)."""
+
+    def __init__(self, qt: binding.QTensor):
+        self.rows, self.cols = qt.rows, qt.cols
+        self.q_rm = qt.q_rm.cpu().numpy()
+        self.q_t = qt.q_t.cpu().numpy() if qt.q_t is not None else None
+        self.scale = qt.scale.cpu().numpy()
+        self._values = np.array([oracle.e2m1_value(k) for k in range(16)])
+
+    def row_range(self, r0: int, r1: int) -> np.ndarray:
+        """Dequantized rows r0..r1 (r0 a multiple of 32)."""
+        assert r0 % 32 == 0
+        n = r1 - r0
+        if n <= 0:
+            return np.zeros((0, self.cols))
+        q = np.ascontiguousarray(self.q_rm[r0:r1, :(self.cols + 1) // 2])
+        s = np.ascontiguousarray(self.scale[r0 // 32:(r1 + 31) // 32, :max((self.cols + 31) // 32, 1)])
+        return oracle.dequantize2d(q, s, n, self.cols)
+
+    def take_rows(self, rows) -> np.ndarray:
+        out = np.empty((len(rows), self.cols))
+        for i, r in enumerate(rows):
+            b = int(r) // 32 * 32
+            out[i] = self.row_range(b, min(b + 32, self.rows))[int(r) - b]
+        return out
+
+    def take_cols(self, cols, r0: int = 0, r1: int = None) -> np.ndarray:
+        """Dequantized columns (as an array [r1 - r0, len(cols)]) decoded from the transposed payload."""
+        r1 = self.rows if r1 is None else r1
+        assert r0 % 32 == 0
+        out = np.empty((r1 - r0, len(cols)))
+        for i, c in enumerate(cols):
+            q = self.q_t[int(c), r0 // 2:(r1 + 1) // 2]
+            codes = np.empty(2 * q.size, dtype=np.uint8)
+            codes[0::2] = q & 0xF
+            codes[1::2] = q >> 4
+            e = np.repeat(self.scale[r0 // 32:(r1 + 31) // 32, int(c) // 32].astype(np.int64), 32)[:r1 - r0]
+            out[:, i] = self._values[codes[:r1 - r0]] * np.ldexp(1.0, e - 127)
+        return out
+
+
+def assert_windows_match_oracle(x: torch.Tensor, qt: binding.QTensor, block_rows, mode, seed, tensor_id):
+    """Bit-exact comparison of whole block rows (32 rows, every column) of a large quantized tensor with the
+    oracle, which is run on a window of the full tensor (the rounding stream stays keyed on the global index)."""
+    bits = workloads.bf16_bits(x)
+    rows, cols = bits.shape
+    ct = (cols + 31) // 32
+    for I in block_rows:
+        I = int(I)
+        o_rm, o_t, o_s = oracle.quantize2d(bits, mode, seed, tensor_id, window=(I, I + 1, 0, ct))
+        n = o_rm.shape[0]
+        g_rm = qt.q_rm[32 * I:32 * I + n, :(cols + 1) // 2].cpu().numpy()
+        g_t = qt.q_t[:cols, 16 * I:16 * I + (n + 1) // 2].cpu().numpy()
+        g_s = qt.scale[I, :ct].cpu().numpy()
+        assert np.array_equal(g_s, o_s[0]), ("scale", I)
+        assert np.array_equal(g_rm, o_rm), ("q_rm", I)
+        assert np.array_equal(g_t, o_t), ("q_t", I)

@@ -34,6 +34,8 @@ def test_forward_and_backward_match_the_oracle_products():
         want = oracle.bf16_round(want)   # all three leave the layer in BF16
         rel = np.linalg.norm(got - want) / np.linalg.norm(want)
         assert rel <= 1e-3, (name, rel)
+        # and, per output row, max |G - O| <= 1e-2 * ||O_row||_inf
+        assert (np.abs(got - want) <= 1e-2 * np.abs(want).max(axis=1, keepdims=True)).all(), name
 
 
 def test_student_fits_a_random_teacher():

@@ -4,15 +4,16 @@ own BF16-rounded output.
 Oracle: quantize2d(BF16(gemm_fwd(X^, W^))).  FP32 accumulation order is not the oracle's, so a bit-exact comparison
 with the oracle needs operands for which every partial sum is exact (E2M1-grid values times a power of two): then
 the GPU's BF16 output is the oracle's and payloads and scales must agree bit for bit.  On general operands the fused
-call is compared, bit for bit, with the unfused chain (fp4q_gemm_fwd to BF16, then fp4q_quantize2d), whose two
-halves are each tied to the oracle by their own tests."""
+call is compared, bit for bit, with the unfused chain (fp4q_gemm_fwd to BF16, then fp4q_quantize2d) and with the
+oracle in two steps: the BF16 product against the oracle's product within the GEMM tolerance, and the fused payloads
+and scales against the oracle's quantizer applied to that very BF16 product, bit for bit."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2607_24953_b200 import binding, workloads
-from tests.gpu_util import assert_matches_oracle, dequant_from_gpu, logical
+from tests.gpu_util import assert_matches_oracle, check_gemm, dequant_from_gpu, logical
 
 pytestmark = pytest.mark.gpu
 
@@ -69,6 +70,31 @@ def test_fused_equals_product_then_quantize(T, N, K, mode):
     assert binding.fp4q_workspace_status(ws) == 0
     c_rm, c_t, c_s = logical(chain)
     compare_logical(fused, c_rm, c_t, c_s, T, N)
+
+
+@pytest.mark.parametrize("T,N,K", [(300, 272, 1000), (1000, 1040, 320)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_general_operands_against_the_oracle_in_two_steps(T, N, K, mode):
+    """General operands (FP32 accumulation order differs from the oracle's): the BF16 product is within the GEMM
+    tolerance of the oracle's, and the fused encoding is exactly the oracle's quantizer applied to that BF16 product."""
+    X = workloads.activations_student_t(T, K, 720, "cuda")
+    W = workloads.weights(N, K, 721, "cuda")
+    dY = workloads.gradients_rowscaled(T, N, 722, "cuda")
+    qx = assert_matches_oracle(X, 0)
+    qw = assert_matches_oracle(W, 0)
+    qdy = assert_matches_oracle(dY, 1, seed=2, tensor_id=5)
+    xd, wd, dyd = dequant_from_gpu(qx), dequant_from_gpu(qw), dequant_from_gpu(qdy)
+    ws = binding.alloc_workspace("cuda")
+    y = binding.fp4q_gemm_fwd(qx, qw, dt=binding.OUT_BF16, ws=ws).contiguous()
+    dx = binding.fp4q_gemm_dgrad(qdy, qw, dt=binding.OUT_BF16, ws=ws).contiguous()
+    fused_y = binding.fp4q_gemm_fwd_quantized(qx, qw, mode=mode, seed=3, tensor_id=8, ws=ws)
+    fused_dx = binding.fp4q_gemm_dgrad_quantized(qdy, qw, mode=mode, seed=4, tensor_id=9, ws=ws)
+    torch.cuda.synchronize()
+    assert binding.fp4q_workspace_status(ws) == 0
+    check_gemm(y, oracle.gemm_fwd(xd, wd), "forward product")
+    check_gemm(dx, oracle.gemm_dgrad(dyd, wd), "input-gradient product")
+    compare_logical(fused_y, *oracle.quantize2d(workloads.bf16_bits(y), mode, 3, 8), T, N)
+    compare_logical(fused_dx, *oracle.quantize2d(workloads.bf16_bits(dx), mode, 4, 9), T, K)
 
 
 def test_output_width_must_be_a_multiple_of_16():
