@@ -12,10 +12,12 @@
  * Conventions common to every entry point
  *   - Every data pointer is a DEVICE pointer owned by the caller; the descriptor structs
  *     themselves (fp4q_tensor, fp4q_groups) are read on the HOST during the call.
- *   - The library allocates no device memory, never synchronises the device, and only
- *     enqueues work on `stream` (a cudaStream_t passed as void*; NULL = default stream).
- *     The first call in a process creates per-process state (module load, driver entry
- *     point lookup) and should be made outside stream capture.
+ *   - The library allocates no device memory and the compute entry points (quantizers, GEMMs)
+ *     never synchronise: they only enqueue work on `stream` (a cudaStream_t passed as void*;
+ *     NULL = default stream).  The three small workspace calls (fp4q_workspace_status,
+ *     fp4q_workspace_set_wait_limit, fp4q_debug_withhold_load) copy a few bytes and DO
+ *     synchronise `stream`.  The first call on a device creates per-device state (module load,
+ *     driver entry point lookup, kernel attributes) and should be made outside stream capture.
  *   - Every function returns an fp4q_status; nothing throws, traps or aborts.  Argument
  *     errors are reported before any work is enqueued.  Device-side anomalies (a bounded
  *     wait that ran out) are recorded in the workspace status word and read back with
@@ -126,8 +128,23 @@ fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int6
 size_t fp4q_workspace_bytes(void);
 
 /* Reads the status word of a workspace (synchronous 4-byte device-to-host copy on `stream`
- * followed by a stream synchronise) and clears it.  FP4Q_OK, FP4Q_ERR_TIMEOUT or FP4Q_ERR_CUDA. */
+ * followed by a stream synchronise) and clears it.  FP4Q_OK, FP4Q_ERR_TIMEOUT or FP4Q_ERR_CUDA.
+ * After FP4Q_ERR_TIMEOUT the outputs of the calls that used the workspace since the last read
+ * are unspecified; the context stays usable and later calls are unaffected. */
 fp4q_status fp4q_workspace_status(void *ws, void *stream);
+
+/* Every wait inside the GEMM kernels is bounded by a number of polls (default 2^22, far beyond
+ * anything a healthy run needs; the one wait that spans a whole tile scales it with the tile's
+ * contraction length).  This call stores another limit in the workspace (0 restores the default);
+ * it applies to every later call that uses the workspace.  Synchronises `stream`. */
+fp4q_status fp4q_workspace_set_wait_limit(void *ws, uint32_t polls, void *stream);
+
+/* Development aid for exercising the timeout path without faulting or hanging anything: with
+ * nth_load = n > 0 stored in the workspace, the first CTA of every later GEMM call that uses the
+ * workspace leaves out its n-th operand load, so the wait for it runs out, the kernel records
+ * FP4Q_ERR_TIMEOUT and leaves through its normal exit.  0 switches the hook off (the state of a
+ * zeroed workspace).  Combine with a small wait limit.  Synchronises `stream`. */
+fp4q_status fp4q_debug_withhold_load(void *ws, uint32_t nth_load, void *stream);
 
 /*
  * fp4q_gemm_fwd -- Y[T,N] = X^[T,K] W^[N,K]^T  (Section 3, first product), FP32 accumulation.

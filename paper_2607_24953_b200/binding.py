@@ -27,7 +27,9 @@ BLOCK_64 = 4
 
 EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgrad",
            "fp4q_mxfp8_quantize1d", "fp4q_mxfp8_qk", "fp4q_workspace_bytes", "fp4q_workspace_status",
-           "fp4q_status_string", "fp4q_version", "fp4q_gemm_fwd_static_workspace"]
+           "fp4q_status_string", "fp4q_version", "fp4q_gemm_fwd_static_workspace", "fp4q_workspace_set_wait_limit",
+           "fp4q_debug_withhold_load", "fp4q_quantize1d", "fp4q_quantize1d_t", "fp4q_gemm_fwd_act1d", "fp4q_gemm_wgrad_act1d",
+           "fp4q_mxfp8_quantize1d_t", "fp4q_mxfp8_gemm", "fp4q_gemm_fwd_quantized", "fp4q_gemm_dgrad_quantized"]
 
 
 class Fp4qError(RuntimeError):
@@ -67,50 +69,46 @@ def lib() -> ctypes.CDLL:
         L.fp4q_workspace_bytes.argtypes = []
         L.fp4q_workspace_status.restype = ci
         L.fp4q_workspace_status.argtypes = [vp, vp]
+        L.fp4q_workspace_set_wait_limit.restype = ci
+        L.fp4q_workspace_set_wait_limit.argtypes = [vp, u32, vp]
+        L.fp4q_debug_withhold_load.restype = ci
+        L.fp4q_debug_withhold_load.argtypes = [vp, u32, vp]
         L.fp4q_status_string.restype = ctypes.c_char_p
         L.fp4q_status_string.argtypes = [ci]
         L.fp4q_version.restype = ci
         L.fp4q_version.argtypes = []
         gemm_args = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64, ci, ctypes.POINTER(_CGroups),
                      vp, ctypes.c_size_t, vp]
-        if hasattr(L, "fp4q_gemm_fwd"):
-            L.fp4q_gemm_fwd.restype = ci
-            L.fp4q_gemm_fwd.argtypes = gemm_args
-            L.fp4q_gemm_dgrad.restype = ci
-            L.fp4q_gemm_dgrad.argtypes = gemm_args
-            L.fp4q_gemm_wgrad.restype = ci
-            L.fp4q_gemm_wgrad.argtypes = gemm_args[:5] + [ci] + gemm_args[5:]
-        if hasattr(L, "fp4q_mxfp8_qk"):
-            L.fp4q_mxfp8_qk.restype = ci
-            L.fp4q_mxfp8_qk.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, i64, i64, i64, vp, vp, i64,
-                                        ci, vp, ctypes.c_size_t, vp]
-        if hasattr(L, "fp4q_gemm_fwd_static_workspace"):
-            L.fp4q_gemm_fwd_static_workspace.restype = ci
-            L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
-                                                         ci, vp, vp]
-        if hasattr(L, "fp4q_quantize1d"):
-            L.fp4q_quantize1d.restype = ci
-            L.fp4q_quantize1d.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, ci, u64, u32, vp]
-            L.fp4q_quantize1d_t.restype = ci
-            L.fp4q_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
-        if hasattr(L, "fp4q_gemm_fwd_act1d"):
-            L.fp4q_gemm_fwd_act1d.restype = ci
-            L.fp4q_gemm_fwd_act1d.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, ci, vp, ctypes.c_size_t, vp]
-            L.fp4q_gemm_wgrad_act1d.restype = ci
-            L.fp4q_gemm_wgrad_act1d.argtypes = [vp, vp, i64, vp, i64, i64, vp, i64, ci, ci, vp, ctypes.c_size_t, vp]
-        if hasattr(L, "fp4q_mxfp8_gemm"):
-            L.fp4q_mxfp8_quantize1d_t.restype = ci
-            L.fp4q_mxfp8_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
-            L.fp4q_mxfp8_gemm.restype = ci
-            L.fp4q_mxfp8_gemm.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp, i64, i64, i64, vp, i64, ci, vp,
-                                          ctypes.c_size_t, vp]
-        if hasattr(L, "fp4q_gemm_dgrad_quantized"):
-            L.fp4q_gemm_dgrad_quantized.restype = ci
-            L.fp4q_gemm_dgrad_quantized.argtypes = [vp, vp, vp, ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
-        if hasattr(L, "fp4q_gemm_fwd_quantized"):
-            L.fp4q_gemm_fwd_quantized.restype = ci
-            L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
-                                                  ctypes.POINTER(_CTensor), ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
+        L.fp4q_gemm_fwd.restype = ci
+        L.fp4q_gemm_fwd.argtypes = gemm_args
+        L.fp4q_gemm_dgrad.restype = ci
+        L.fp4q_gemm_dgrad.argtypes = gemm_args
+        L.fp4q_gemm_wgrad.restype = ci
+        L.fp4q_gemm_wgrad.argtypes = gemm_args[:5] + [ci] + gemm_args[5:]
+        L.fp4q_mxfp8_qk.restype = ci
+        L.fp4q_mxfp8_qk.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, i64, i64, i64, vp, vp, i64,
+                                    ci, vp, ctypes.c_size_t, vp]
+        L.fp4q_gemm_fwd_static_workspace.restype = ci
+        L.fp4q_gemm_fwd_static_workspace.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64,
+                                                     ci, vp, vp]
+        L.fp4q_quantize1d.restype = ci
+        L.fp4q_quantize1d.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, ci, u64, u32, vp]
+        L.fp4q_quantize1d_t.restype = ci
+        L.fp4q_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
+        L.fp4q_gemm_fwd_act1d.restype = ci
+        L.fp4q_gemm_fwd_act1d.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, ci, vp, ctypes.c_size_t, vp]
+        L.fp4q_gemm_wgrad_act1d.restype = ci
+        L.fp4q_gemm_wgrad_act1d.argtypes = [vp, vp, i64, vp, i64, i64, vp, i64, ci, ci, vp, ctypes.c_size_t, vp]
+        L.fp4q_mxfp8_quantize1d_t.restype = ci
+        L.fp4q_mxfp8_quantize1d_t.argtypes = [vp, i64, i64, i64, vp, i64, vp, i64, vp]
+        L.fp4q_mxfp8_gemm.restype = ci
+        L.fp4q_mxfp8_gemm.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp, i64, i64, i64, vp, i64, ci, vp,
+                                      ctypes.c_size_t, vp]
+        L.fp4q_gemm_dgrad_quantized.restype = ci
+        L.fp4q_gemm_dgrad_quantized.argtypes = [vp, vp, vp, ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
+        L.fp4q_gemm_fwd_quantized.restype = ci
+        L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
+                                              ctypes.POINTER(_CTensor), ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -310,6 +308,16 @@ def alloc_workspace(device) -> torch.Tensor:
 
 def fp4q_workspace_status(ws: torch.Tensor, stream=None) -> int:
     return int(lib().fp4q_workspace_status(ws.data_ptr(), _stream(stream)))
+
+
+def fp4q_workspace_set_wait_limit(ws: torch.Tensor, polls: int, stream=None):
+    """Poll limit of the kernels' bounded waits for every later call that uses ws (0 = default)."""
+    _check(lib().fp4q_workspace_set_wait_limit(ws.data_ptr(), int(polls), _stream(stream)), "fp4q_workspace_set_wait_limit")
+
+
+def fp4q_debug_withhold_load(ws: torch.Tensor, nth_load: int, stream=None):
+    """Development aid: the first CTA of later GEMM calls on ws leaves out its n-th operand load (0 = off)."""
+    _check(lib().fp4q_debug_withhold_load(ws.data_ptr(), int(nth_load), _stream(stream)), "fp4q_debug_withhold_load")
 
 
 def _groups(row_offsets: Optional[torch.Tensor], row_alignment: int = 128):

@@ -1,4 +1,6 @@
 // Small host-side entry points of libfp4q: status strings, version, workspace handling.
+#include <cstddef>
+
 #include "common.cuh"
 
 using namespace fp4q;
@@ -33,4 +35,24 @@ extern "C" fp4q_status fp4q_workspace_status(void *ws, void *stream)
     if (cudaMemsetAsync(ws, 0, sizeof host, s) != cudaSuccess) return FP4Q_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return FP4Q_ERR_CUDA;
     return host[0] == (uint32_t)FP4Q_ERR_TIMEOUT ? FP4Q_ERR_TIMEOUT : FP4Q_ERR_CUDA;
+}
+
+// The two configuration words of a workspace (they persist until rewritten; fp4q_workspace_status clears only the status).
+static fp4q_status set_workspace_word(void *ws, size_t offset, uint32_t value, void *stream)
+{
+    if (!ws) return FP4Q_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(static_cast<uint8_t *>(ws) + offset, &value, sizeof value, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return FP4Q_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;   // `value` lives on this stack frame
+}
+
+extern "C" fp4q_status fp4q_workspace_set_wait_limit(void *ws, uint32_t polls, void *stream)
+{
+    return set_workspace_word(ws, offsetof(Workspace, wait_limit), polls, stream);
+}
+
+extern "C" fp4q_status fp4q_debug_withhold_load(void *ws, uint32_t nth_load, void *stream)
+{
+    return set_workspace_word(ws, offsetof(Workspace, withhold_load), nth_load, stream);
 }

@@ -16,9 +16,11 @@ static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<u
 
 // Layout of the GEMM workspace (device memory, caller-owned).
 struct Workspace {
-    uint32_t status;      // 0 = ok, otherwise an fp4q_status written by a kernel
-    uint32_t detail;      // where the kernel gave up (role/stage), for diagnostics
-    uint32_t pad[62];
+    uint32_t status;         // 0 = ok, otherwise an fp4q_status written by a kernel
+    uint32_t detail;         // where the kernel gave up (role/stage), for diagnostics
+    uint32_t wait_limit;     // polls after which a bounded wait gives up; 0 = the kernels' default
+    uint32_t withhold_load;  // development hook, 0 in production: n > 0 = CTA 0 leaves out its n-th stage load
+    uint32_t pad[60];
 };
 
 }  // namespace fp4q

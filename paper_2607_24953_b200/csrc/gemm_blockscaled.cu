@@ -80,8 +80,13 @@ __host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8
 // and pay for the buffers with one ring stage; the pair kernel also keeps a third image buffer, because the way
 // from "the MMAs have finished with a buffer" to "the leader may copy the next unit out of it" (commit to both
 // CTAs, build, report to the leader) is longer than one unit as well.
-template <int KIND, int CTAS>
+// NT is the tile's width in output columns.  256: one accumulator of 256 tensor-memory columns (the other 256 hold the
+// ring of scale columns).  Narrower pair tiles (224, 192) leave room for TWO accumulators beside two or four scale
+// slots, so that the epilogue drains one tile while the MMAs of the next one already run.
+template <int KIND, int CTAS, int NT = 256>
 struct Cfg {
+    static_assert(NT == 256 || (CTAS == 2 && KIND == KIND_MXF4 && NT % 32 == 0 && 2 * NT + 64 <= 512), "two-accumulator tiles: FP4 pair kernel only");
+    static constexpr int kAccs = NT == 256 ? 1 : 2;
     static constexpr bool kRowImages = KIND != KIND_MXF4;
     static constexpr int kImageBufs = (CTAS == 2 && kRowImages) ? 3 : 2;
     static constexpr int kRawBufs = kRowImages ? 2 : 0;
@@ -92,7 +97,7 @@ struct Cfg {
     static constexpr bool kTmaStores = CTAS == 2 || !kRowImages;
     static constexpr int kStages = (CTAS == 2 ? 5 : (kTmaStores ? 3 : 4)) - (kRowImages ? 1 : 0);
     static constexpr int kSmemCache = kCompactBytes + (kImageBufs + kRawBufs) * kCacheBufBytes;
-    static constexpr int kBRows = CTAS == 2 ? 128 : 256;
+    static constexpr int kBRows = CTAS == 2 ? NT / 2 : NT;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
@@ -101,12 +106,16 @@ struct Cfg {
     static_assert(kSmemGroups == 0 || kSmemGroups >= kMaxRowTilesShared * 2, "group table");
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail + kSmemGroups;
     static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+    // tensor memory: accumulators first, then the scale slots (32 columns each: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk))
+    static constexpr int kTmemSfBase = kAccs * NT;
+    static constexpr int kSfSlots = kAccs == 1 ? kStages : (512 - kAccs * NT) / 32;
+    static_assert(kTmemSfBase % 32 == 0 && kTmemSfBase + kSfSlots * 32 <= 512 && kSfSlots >= 2, "tensor memory budget");
 };
 constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
-constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
-constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr int kTmemSfStride = 32;            // per scale slot: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
+constexpr uint32_t kWaitLimit = 1u << 22;       // default number of polls after which a wait gives up (workspace word 2 overrides it)
 constexpr int kRelaxedNs = 64, kLazyNs = 256;   // back-off between polls of roles with slack
 // Developer diagnostic (off by default): -DFP4Q_TRACE makes CTA 0 add up clock64() intervals of its roles in
 // registers and leave them in the workspace's padding words (status[16 + 2*slot], 64-bit each).
@@ -150,6 +159,7 @@ struct GemmParams {
     int32_t M, N, K;                 // per-problem output rows, output columns, contraction length (elements)
     int32_t m_tiles, n_tiles, n_tile_total;   // m_tiles counts rows of 128 * ctas
     int32_t ctas;                    // CTAs per tile (1, or 2 for cta_group::2 pairs)
+    int32_t bn;                      // tile width in output columns (256; 224 or 192 for the two-accumulator pair kernel)
     int32_t raster_m;                // tile order: groups of raster_m row tiles, within a group row tile fastest
     int32_t out_f32, accumulate;
     int32_t wide_stores;             // output base and row pitch are 32-byte aligned: 256-bit stores (whole sectors)
@@ -223,41 +233,43 @@ __device__ __forceinline__ void named_sync(uint32_t id) { asm volatile("bar.sync
 // slack (everything but the MMA issuer) sleep between polls.
 template <int BACKOFF_NS, bool PROBE = false>
 __device__ __forceinline__ bool mbar_wait_impl(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                               uint32_t where)
+                                               uint64_t limit, uint32_t where)
 {
-    for (uint32_t it = 0; it < kWaitLimit; it++) {
+    for (uint64_t it = 0; it < limit; it++) {
         if (PROBE ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);
-        if ((it & 255u) == 255u && *abort_flag) return false;
+        if (((uint32_t)it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1u;
     if (atomicCAS(status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) status[1] = where;
     return false;
 }
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint32_t where)
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint64_t limit,
+                                       uint32_t where)
 {
-    return mbar_wait_impl<0>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<0>(bar, parity, abort_flag, status, limit, where);
 }
 __device__ __noinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                               uint32_t where)
+                                               uint64_t limit, uint32_t where)
 {
-    return mbar_wait_impl<kRelaxedNs>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kRelaxedNs>(bar, parity, abort_flag, status, limit, where);
 }
 __device__ __noinline__ bool mbar_wait_lazy(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                            uint32_t where)
+                                            uint64_t limit, uint32_t where)
 {
-    return mbar_wait_impl<kLazyNs>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kLazyNs>(bar, parity, abort_flag, status, limit, where);
 }
 // For barriers that another CTA of the cluster completes (a multicast tcgen05.commit): probe instead of try_wait,
 // whose suspended thread is not reliably woken early by a remote arrival.
-__device__ __noinline__ bool mbar_poll(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint32_t where)
+__device__ __noinline__ bool mbar_poll(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint64_t limit,
+                                       uint32_t where)
 {
-    return mbar_wait_impl<0, true>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<0, true>(bar, parity, abort_flag, status, limit, where);
 }
 __device__ __noinline__ bool mbar_poll_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                               uint32_t where)
+                                               uint64_t limit, uint32_t where)
 {
-    return mbar_wait_impl<kRelaxedNs, true>(bar, parity, abort_flag, status, where);
+    return mbar_wait_impl<kRelaxedNs, true>(bar, parity, abort_flag, status, limit, where);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
@@ -378,11 +390,11 @@ __device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
 }
 
 // Instruction descriptor of the block-scaled MMA: formats, K-major operands, N, UE8M0 scales, M, scale byte ids.
-template <int KIND, int CTAS>
+template <int KIND, int CTAS, int NT>
 __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_id)
 {
     const uint32_t fmt = kind_fp4(KIND) ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
-    return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) |
+    return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(NT >> 3) << 17) | (1u << 23) |
            ((uint32_t)((BM * CTAS) >> 4) << 24) | (a_sf_id << 29);
 }
 
@@ -434,14 +446,14 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int r
     const int m0 = grp_m * p.raster_m, gsz = min(p.raster_m, p.m_tiles - m0);
     const int n_blk = in_grp / gsz, m_blk = m0 + (in_grp - n_blk * gsz);
     t.a_row0 = (m_blk * p.ctas + rank) * BM;
-    t.b_row0 = n_blk * BN;
-    t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * 128 : 0);
+    t.b_row0 = n_blk * p.bn;
+    t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * (p.bn >> 1) : 0);
     t.a_k0 = t.b_k0 = 0;
     t.k_len = p.K;
     t.c_row0 = t.a_row0;
     t.c_col0 = t.b_row0;
     t.m_valid = min(BM, p.M - t.a_row0);
-    t.n_valid = min(BN, p.N - t.b_row0);
+    t.n_valid = min(p.bn, p.N - t.b_row0);
     if (p.mode == MODE_GROUPED_ROWS) {
         if (!need_b) return;
         const int grp = goffs ? (int)reinterpret_cast<const uint16_t *>(goffs)[t.a_row0 / BM]
@@ -956,7 +968,7 @@ __device__ __forceinline__ void read_raw_scales(const GemmParams &p, const uint8
 
 // ---------------------------------------------------------------------------------------- kernel
 
-template <int KIND, int CTAS, int EPI>
+template <int KIND, int CTAS, int EPI, int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
@@ -965,20 +977,20 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kStageElems = kind_fp4(KIND) ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = kind_fp4(KIND) ? 64 : 32;           // contraction elements per MMA (32 B per row)
     constexpr int kElemsPerByte = kind_fp4(KIND) ? 2 : 1;
-    constexpr int kStages = Cfg<KIND, CTAS>::kStages;
-    constexpr int kBStageBytes = Cfg<KIND, CTAS>::kBStageBytes;
+    constexpr int kStages = Cfg<KIND, CTAS, NT>::kStages;
+    constexpr int kBStageBytes = Cfg<KIND, CTAS, NT>::kBStageBytes;
     constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8 : kUnitStagesMxf4R;   // stages whose scale images are built together
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_compact = smem + Cfg<KIND, CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
+    uint8_t *smem_compact = smem + Cfg<KIND, CTAS, NT>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
     uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and the buffers of ready scale images (any kind)
-    uint8_t *smem_raw_scales = smem_images + Cfg<KIND, CTAS>::kImageBufs * kCacheBufBytes;   // per-row scales: bytes in flight
-    uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS>::kSmemStaging);
-    // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
+    uint8_t *smem_raw_scales = smem_images + Cfg<KIND, CTAS, NT>::kImageBufs * kCacheBufBytes;   // per-row scales: bytes in flight
+    uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS, NT>::kSmemScales;   // 1024-byte aligned (pair kernel only)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS, NT>::kSmemStaging);
+    // bars[0..5] full, bars[6..11] empty, bars[12] / bars[14] accumulator 0 / 1 full, bars[13] / bars[15] accumulator 0 / 1 empty,
     // bars[18] tensor pipe drained (abort path), bars[24..27] scale images full, bars[28..31] scale images empty,
     // bars[32..35] (leader of a pair) the second CTA's scale images full - one of each per image buffer
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 21);
@@ -986,11 +998,18 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     int32_t *goffs_smem = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(bars) + kSmemTail);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Poll limit of every bounded wait (workspace word 2; 0 = the default) and the development hook of word 3 (n > 0:
+    // the producer of CTA 0 leaves out its n-th stage load, so that a test can watch a wait run out and the kernel
+    // leave through its timeout path without anything faulting or spinning for long).
+    const uint32_t wait_limit_word = __ldg(p.status + 2), withhold_load = blockIdx.x == 0 ? __ldg(p.status + 3) : 0u;
+    const uint64_t wait_limit = wait_limit_word != 0u ? wait_limit_word : kWaitLimit;
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + kMaxStages);
     const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
     const uint32_t bar_cache_full = smem_u32(bars + 24), bar_cache_empty = smem_u32(bars + 28);
     const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 32);
-    constexpr int kImageBufs = Cfg<KIND, CTAS>::kImageBufs;
+    constexpr int kImageBufs = Cfg<KIND, CTAS, NT>::kImageBufs;
+    constexpr int kAccs = Cfg<KIND, CTAS, NT>::kAccs;                 // accumulators in tensor memory (tiles alternate)
+    constexpr int kTmemSfBase = Cfg<KIND, CTAS, NT>::kTmemSfBase, kSfSlots = Cfg<KIND, CTAS, NT>::kSfSlots;
 
     // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
     const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
@@ -1004,10 +1023,12 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
         }
-        mbar_init(bar_acc_full, 1);
+        for (int a = 0; a < kAccs; a++) {
+            mbar_init(bar_acc_full + 16 * a, 1);
+            mbar_init(bar_acc_empty + 16 * a, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
+        }
         mbar_init(bar_drain, 1);
-        mbar_init(bar_acc_empty, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
-        for (int b = 0; b < Cfg<KIND, CTAS>::kImageBufs; b++) {
+        for (int b = 0; b < Cfg<KIND, CTAS, NT>::kImageBufs; b++) {
             mbar_init(bar_cache_full + 8 * b, 1);
             mbar_init(bar_cache_empty + 8 * b, 1);
             mbar_init(bar_peer_cache_full + 8 * b, 1);
@@ -1016,7 +1037,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-        if (Cfg<KIND, CTAS>::kTmaStores) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
+        if (Cfg<KIND, CTAS, NT>::kTmaStores) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
         if (EPI == EPI_QUANT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
     }
     if (warp == 1) {
@@ -1032,7 +1053,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     }
     // grouped products: a 32-bit copy of the group boundaries for the per-tile lookups of every role
     const int n_row_tiles = (p.M + BM - 1) / BM;
-    const bool goffs_ok = Cfg<KIND, CTAS>::kSmemGroups > 0 &&
+    const bool goffs_ok = Cfg<KIND, CTAS, NT>::kSmemGroups > 0 &&
                           ((p.mode == MODE_GROUPED_K && p.n_groups <= kMaxGroupsShared) ||
                            (p.mode == MODE_GROUPED_ROWS && n_row_tiles <= kMaxRowTilesShared && p.n_groups <= 65535));
     if (goffs_ok && p.mode == MODE_GROUPED_K)
@@ -1069,7 +1090,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             c_rounds++;
 #endif
             if (lane == 0) {
-                ok = mbar_wait_impl<0, true>(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, 0x100u + stage);
+                ok = mbar_wait_impl<0, true>(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, wait_limit, 0x100u + stage);
                 if (ok) {
                     n_free = 1;
                     uint32_t s2 = stage, ph2 = phase;
@@ -1085,7 +1106,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             TRACE_ADD(c_empty, tt);
             for (int b = 0; b < n_free && pr.valid(p); b++) {
                 if (lane == 0) TRACE_EV(0, ev_j);
-                if (issuer) {
+                if (issuer && !(withhold_load != 0u && (uint32_t)ev_j + 1u == withhold_load)) {
                     const Tile &t = pr.t;
                     const int xa = (t.a_k0 + pr.it * kStageElems) / kElemsPerByte, xb = (t.b_k0 + pr.it * kStageElems) / kElemsPerByte;
                     if (CTAS == 1) {
@@ -1120,7 +1141,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0;
+        uint32_t stage = 0, acc = 0, sf_slot = 0;
         BufRing ring;   // image buffer of the current unit
         const bool issuer = elect_one();
         int ev_j = 0;
@@ -1138,7 +1159,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
                 if (issuer) {
-                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
+                    // one accumulator: the scale slot follows the ring stage; two: a short ring of its own (copies
+                    // and MMAs execute in issue order, so a slot may be rewritten two stages later)
+                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + (kAccs == 1 ? stage : sf_slot) * kTmemSfStride;
+                    const uint32_t d_tmem = tmem_base + acc * NT;
                     if (KIND == KIND_MXF4) {
                         const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
@@ -1170,13 +1194,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         if (i < n_mma) {
                             const int chunk = kind_fp4(KIND) ? (i >> 1) : 0;
                             const uint32_t sf_id = kind_fp4(KIND) ? 2u * (i & 1) : (uint32_t)i;
-                            tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
-                                                                 instr_desc<KIND, CTAS>(sf_id, sf_id), sf_tmem + 4 * chunk,
+                            tcgen05_mma_block_scaled<KIND, CTAS>(d_tmem, adesc + 2 * i, bdesc + 2 * i,
+                                                                 instr_desc<KIND, CTAS, NT>(sf_id, sf_id), sf_tmem + 4 * chunk,
                                                                  sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
                         }
                     }
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
-                    if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
+                    if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full + 16 * acc);
                     if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
                         tcgen05_commit<CTAS>(bar_cache_empty + 8 * ring.buf);   // the unit's images have been copied
                 }
@@ -1185,15 +1209,20 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (lane == 0) TRACE_EV(3, ev_j);
                 ev_j++;
                 if (++stage == kStages) stage = 0;
+                if (++sf_slot == kSfSlots) sf_slot = 0;
             }
+            if (kAccs == 2) acc ^= 1u;
         }
         if (leader && *abort_flag) {
             // Some role gave up: the watchers then release every remaining stage unseen, and this warp has run
             // through them.  Wait (bounded) until the tensor pipe is idle before tensor memory is freed.
             if (issuer) tcgen05_commit<CTAS>(bar_drain);
             __syncwarp();
-            if (lane == 0) mbar_wait_lazy(bar_drain, 0u, abort_flag, p.status, 0x220u);   // gives up after 256 polls (abort is set)
+            if (lane == 0) mbar_wait_lazy(bar_drain, 0u, abort_flag, p.status, wait_limit, 0x220u);   // gives up after 256 polls (abort is set)
             __syncwarp();
+            // After an abort the stages were consumed without waiting for their operands, so loads of either CTA may
+            // still be on their way: hold the pair (the other roles wait at the final barrier) until they have landed.
+            for (int i = 0; i < 200; i++) __nanosleep(1000);
         }
         if (lane == 0) { TRACE_OUT(p, 2, c_acc); TRACE_OUT(p, 3, c_sync); TRACE_OUT(p, 4, c_issue); }
     } else if (warp == 3) {
@@ -1211,7 +1240,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             // per-row scales: the raw bytes of the next kRawBufs units are in flight (cp.async) while a unit is
             // turned into images.  In a pair an image buffer is released by the leader's multicast commit: probe
             // (a suspended try_wait is not reliably woken early by a remote arrival).
-            constexpr int kRawBufs = Cfg<KIND, CTAS>::kRawBufs > 0 ? Cfg<KIND, CTAS>::kRawBufs : 1;
+            constexpr int kRawBufs = Cfg<KIND, CTAS, NT>::kRawBufs > 0 ? Cfg<KIND, CTAS, NT>::kRawBufs : 1;
             UnitIter ahead, cur;
             ahead.init(p, first_tile, tile_step, rank, goffs);
             cur.init(p, first_tile, tile_step, rank, goffs);
@@ -1231,7 +1260,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 uint32_t w[12][8];
                 read_raw_scales(p, smem_raw_scales + raw_read * kCacheBufBytes, lane, w);
                 if (lane == 0)
-                    ok = mbar_wait_impl<kRelaxedNs, CTAS == 2>(bar_cache_empty + 8 * ring.buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + ring.buf);
+                    ok = mbar_wait_impl<kRelaxedNs, CTAS == 2>(bar_cache_empty + 8 * ring.buf, ring.phase ^ 1u, abort_flag, p.status, wait_limit, 0x500u + ring.buf);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 if (!ok) break;
                 store_row_scale_images<KIND>(w, min(kUnitStages, (cur.t.k_len - cur.k0 + kStageElems - 1) / kStageElems),
@@ -1267,8 +1296,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     build_scale_cache(p.sfb, t.b_row0 >> 5, ((t.b_k0 + k0) >> 5), n_chunks, 3, compact + kCacheChunks * 4, lane);
                     __syncwarp();
                     if (lane == 0)
-                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + buf)
-                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, 0x500u + buf);
+                        ok = CTAS == 2 ? mbar_poll_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, wait_limit, 0x500u + buf)
+                                       : mbar_wait_relaxed(bar_cache_empty + 8 * buf, ring.phase ^ 1u, abort_flag, p.status, wait_limit, 0x500u + buf);
                     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                     if (!ok) break;
                     const uint4 *rows = reinterpret_cast<const uint4 *>(smem_compact);
@@ -1305,7 +1334,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // to its end.
         StageIter sg;
         sg.init(p, first_tile, tile_step, rank, kStageElems, goffs, false);
-        uint32_t stage = 0, phase = 0, acc_phase = 0;
+        uint32_t stage = 0, phase = 0, acc_phase = 0, acc = 0;   // acc_phase: bit a = phase of accumulator a's "empty" barrier
         BufRing ring;   // image buffer of the current unit
         bool ok = true;
         TRACE_DECL(c_meet); TRACE_DECL(c_poll);
@@ -1330,7 +1359,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                                          " selp.b32 %0, 1, 0, p0;\n selp.b32 %1, 1, 0, p1;\n}"
                                          : "=r"(q0), "=r"(q1) : "r"(b0), "r"(b1), "r"(ring.phase) : "memory");
                             if (q0 && q1) break;
-                            if (spin >= kWaitLimit) {
+                            if (spin >= wait_limit) {
                                 ok = false;
                                 *abort_flag = 1u;
                                 if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = (q0 ? 0x520u : 0x510u) + ring.buf;
@@ -1349,7 +1378,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     const uint32_t nb0 = bar_cache_full + 8 * nu.buf, nb1 = (CTAS == 2 ? bar_peer_cache_full : bar_cache_full) + 8 * nu.buf;
                     if (KIND == KIND_MXF4 && ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen)
                         unit_seen = mbar_test_wait(nb0, nu.phase) && (CTAS == 1 || mbar_test_wait(nb1, nu.phase));
-                    if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, 0x200u);
+                    if (ok && sg.it == 0)
+                        ok = mbar_wait_impl<0, true>(bar_acc_empty + 16 * acc, ((acc_phase >> acc) & 1u) ^ 1u, abort_flag, p.status, wait_limit, 0x200u + acc);
                     if (ok) {
                         // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long
                         // complete, more than the MMA warp needs per stage.  So the slot's "full" barrier and those of
@@ -1391,7 +1421,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                                            "r"(bar_full + 8 * sl[2]), "r"(ph[2]), "r"(bar_full + 8 * sl[3]), "r"(ph[3]),
                                            "r"(nb0), "r"(nb1), "r"(nu.phase) : "memory");
                             if (r0) break;
-                            if (spin >= kWaitLimit) {
+                            if (spin >= wait_limit) {
                                 ok = false;
                                 *abort_flag = 1u;
                                 if (atomicCAS(p.status, 0u, (uint32_t)FP4Q_ERR_TIMEOUT) == 0u) p.status[1] = 0x300u + stage;
@@ -1411,7 +1441,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             ev_j++;
             named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
             TRACE_ADD(c_meet, tt);
-            if (sg.it == 0) acc_phase ^= 1u;
+            if (sg.it == 0) {
+                acc_phase ^= 1u << acc;
+                if (kAccs == 2) acc ^= 1u;
+            }
             if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) ring.next(kImageBufs);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
             sg.next(p, kStageElems);
@@ -1423,7 +1456,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             BufRing fr;
             UnitIter un;
             for (un.init(p, first_tile, tile_step, rank, goffs); fwd_ok && un.valid(p); un.next(p, kUnitStages * kStageElems), fr.next(kImageBufs)) {
-                fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * fr.buf, fr.phase, abort_flag, p.status, 0x530u + fr.buf);
+                fwd_ok = mbar_wait_impl<kRelaxedNs>(bar_cache_full + 8 * fr.buf, fr.phase, abort_flag, p.status, wait_limit, 0x530u + fr.buf);
                 if (fwd_ok) mbar_arrive_cluster_release(cluster_addr(bar_peer_cache_full + 8 * fr.buf, 0));
             }
         }
@@ -1446,9 +1479,12 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const bool row_ok = row_in_tile < t.m_valid;
             uint32_t v[4][32];
             if (t.k_len > 0) {
+                // this wait spans a whole tile (every other one spans a few stages at most): its limit grows with the
+                // tile's contraction length, so that a very long contraction cannot run into it on a healthy run
+                const uint64_t tile_limit = wait_limit * (uint64_t)(1 + (t.k_len >> 12));
                 if (lane == 0)
-                    ok = CTAS == 2 ? mbar_poll(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp)
-                                   : mbar_wait_relaxed(bar_acc_full, acc_phase, abort_flag, p.status, 0x400u + warp);
+                    ok = CTAS == 2 ? mbar_poll(bar_acc_full, acc_phase, abort_flag, p.status, tile_limit, 0x400u + warp)
+                                   : mbar_wait_relaxed(bar_acc_full, acc_phase, abort_flag, p.status, tile_limit, 0x400u + warp);
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 TRACE_ADD(c_wait, tt);
                 if (lane == 0) TRACE_EV(7, 16 * ev_t + 2 * (warp - 4));
@@ -1552,7 +1588,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         bulk_commit();
                     }
                 }
-            } else if (Cfg<KIND, CTAS>::kTmaStores) {
+            } else if (Cfg<KIND, CTAS, NT>::kTmaStores) {
                 // 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
                 // through this warp's staging rows and leave by a TMA store, which clips rows and columns past the
                 // output's edge.  With accumulation the store is the TMA's FP32 add-reduction.
@@ -1592,7 +1628,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
-        if ((Cfg<KIND, CTAS>::kTmaStores || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
+        if ((Cfg<KIND, CTAS, NT>::kTmaStores || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
         if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
@@ -1681,15 +1717,20 @@ struct Operand {
     ScaleView sf;
 };
 
-static int sm_count()
+constexpr int kMaxDevices = 64;   // per-device host state (attributes set, SM counts, static workspace address)
+
+static int current_device()
 {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+static int sm_count(int dev)
+{
+    static int n[kMaxDevices];
+    if (n[dev] == 0 && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)) n[dev] = 148;
+    return n[dev];
 }
 
 template <int KIND, int CTAS, int EPI = EPI_STORE>
@@ -1705,7 +1746,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
         if (!make_byte_map(&tmC, p.q_rm, p.M, round_up(p.N, 32) / 2, p.q_ld_rm, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return FP4Q_ERR_CUDA;
         if (p.q_t && !make_byte_map(&tmD, p.q_t, p.N, round_up(p.M, 32) / 2, p.q_ld_t, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) return FP4Q_ERR_CUDA;
     } else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
-    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<KIND, CTAS>::kBRows)) return FP4Q_ERR_CUDA;
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<KIND, CTAS, NT>::kBRows)) return FP4Q_ERR_CUDA;
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
@@ -1714,14 +1755,16 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     if (const char *g = getenv("FP4Q_DEBUG_RASTER")) { p.raster_m = atoi(g); if (p.raster_m > p.m_tiles) p.raster_m = p.m_tiles; }
 #endif
 
-    static bool attr_set = false;
-    if (!attr_set) {
+    const int dev = current_device();
+    if (dev < 0) return FP4Q_ERR_CUDA;
+    static bool attr_set[kMaxDevices];   // the attribute is a property of (kernel, device): one flag per device and instantiation
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<KIND, CTAS>::kSmemBytes) != cudaSuccess)
+                                 Cfg<KIND, CTAS, NT>::kSmemBytes) != cudaSuccess)
             return FP4Q_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev] = true;
     }
-    int slots = sm_count() / CTAS;
+    int slots = sm_count(dev) / CTAS;
 #ifdef FP4Q_TRACE
     if (const char *g = getenv("FP4Q_DEBUG_SLOTS")) slots = atoi(g);   // development only: use fewer SMs
 #endif
@@ -1729,7 +1772,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = Cfg<KIND, CTAS>::kSmemBytes;
+    cfg.dynamicSmemBytes = Cfg<KIND, CTAS, NT>::kSmemBytes;
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1741,14 +1784,22 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     return cudaLaunchKernelEx(&cfg, gemm_block_scaled_kernel<KIND, CTAS, EPI>, tmA, tmB, tmC, tmD, p) == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
 }
 
-template <int KIND>
-static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p, void *ws, size_t ws_bytes, void *stream)
+// Argument checks common to every product: everything that can be refused is refused here, before any work is enqueued.
+static fp4q_status check_gemm_args(const Operand &A, const Operand &B, const GemmParams &p, const void *ws, size_t ws_bytes)
 {
     if (!ws || ws_bytes < sizeof(Workspace)) return FP4Q_ERR_WORKSPACE;
     if (!aligned(ws, 256)) return FP4Q_ERR_ALIGN;
     if (!aligned(A.payload, 16) || !aligned(B.payload, 16) || A.ld_bytes % 16 || B.ld_bytes % 16) return FP4Q_ERR_ALIGN;
     const size_t esize = p.out_f32 ? 4 : 2;
     if (!aligned(p.C, 16) || (p.ldc * esize) % 16) return FP4Q_ERR_ALIGN;
+    return FP4Q_OK;
+}
+
+template <int KIND>
+static fp4q_status launch_gemm(const Operand &A, const Operand &B, GemmParams &p, void *ws, size_t ws_bytes, void *stream)
+{
+    if (fp4q_status s = check_gemm_args(A, B, p, ws, ws_bytes)) return s;
+    const size_t esize = p.out_f32 ? 4 : 2;
     if (p.n_tile_total <= 0) return FP4Q_OK;
     p.wide_stores = aligned(p.C, 32) && (p.ldc * esize) % 32 == 0;
     p.sfa = A.sf;
@@ -1812,9 +1863,11 @@ using namespace fp4q;
 
 static const int64_t kMaxDim = 0x7FFFFFFF - 4096;
 
-extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt,
-                                     const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream)
+// The forward product's arguments turned into kernel parameters.  *noop is set when there is nothing to compute.
+static fp4q_status prepare_fwd(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt, const fp4q_groups *g,
+                               GemmParams &p, bool *noop)
 {
+    *noop = false;
     if (!tensor_ok(X) || !tensor_ok(W)) return X && W ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
     if (fp4q_status s = check_groups(g)) return s;
     if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
@@ -1823,10 +1876,10 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
     const int64_t N = g ? W->rows / g->n_groups : W->rows;
     if (g && (W->rows % g->n_groups || N % 32)) return FP4Q_ERR_SHAPE;   // expert blocks must start on a 32-row tile
     if (T > kMaxDim || N > kMaxDim || K > kMaxDim || W->rows > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
-    if (T == 0 || N == 0) return FP4Q_OK;
+    if (T == 0 || N == 0) { *noop = true; return FP4Q_OK; }
     if (!Y || !X->q_rm || !W->q_rm || !X->scale || !W->scale) return FP4Q_ERR_NULL;
     if (ldy < N) return FP4Q_ERR_SHAPE;
-    GemmParams p = {};
+    p = GemmParams{};
     p.C = Y; p.ldc = ldy; p.M = (int32_t)T; p.N = (int32_t)N; p.K = (int32_t)K;
     p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = 0;
     dense_tiles(p);
@@ -1835,6 +1888,16 @@ extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W,
         p.rows_pair_aligned = g->row_alignment == 256;
         p.b_rows_per_group = (int32_t)N; p.b_k_per_group = 0;
     }
+    return FP4Q_OK;
+}
+
+extern "C" fp4q_status fp4q_gemm_fwd(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt,
+                                     const fp4q_groups *g, void *ws, size_t ws_bytes, void *stream)
+{
+    GemmParams p;
+    bool noop;
+    if (fp4q_status s = prepare_fwd(X, W, Y, ldy, dt, g, p, &noop)) return s;
+    if (noop) return FP4Q_OK;
     return launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, ws_bytes, stream);
 }
 
@@ -2068,16 +2131,14 @@ namespace fp4q {
 constexpr size_t kStaticWorkspaceBytes = 1024;   // stated maximum; the kernel's workspace must fit in it
 static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
 
-constexpr int kMaxDevices = 64;
 static void *g_static_workspace_addr[kMaxDevices];   // device address of the array, per device
 
 // In host code the array's name is only a handle: the device address has to be asked for, once per device,
 // with that device current.
 static fp4q_status static_workspace_address(void **out)
 {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return FP4Q_ERR_CUDA;
-    if (dev < 0 || dev >= kMaxDevices) return FP4Q_ERR_UNSUPPORTED;
+    const int dev = current_device();
+    if (dev < 0) return FP4Q_ERR_CUDA;
     if (g_static_workspace_addr[dev] == nullptr) {
         void *ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return FP4Q_ERR_CUDA;
@@ -2093,12 +2154,19 @@ extern "C" fp4q_status fp4q_gemm_fwd_static_workspace(const fp4q_tensor *X, cons
                                                       fp4q_out dt, uint32_t *status_out, void *stream)
 {
     if (fp4q_workspace_bytes() > kStaticWorkspaceBytes) return FP4Q_ERR_WORKSPACE;   // layout outgrew the array
+    // every argument error is reported before anything is put on the stream
+    GemmParams p;
+    bool noop;
+    if (fp4q_status s = prepare_fwd(X, W, Y, ldy, dt, nullptr, p, &noop)) return s;
     void *ws = nullptr;
     if (fp4q_status s = static_workspace_address(&ws)) return s;
+    if (!noop)
+        if (fp4q_status s = check_gemm_args(operand_rm(X), operand_rm(W), p, ws, kStaticWorkspaceBytes)) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: the status words must start at zero
     if (cudaMemsetAsync(ws, 0, sizeof(Workspace), st) != cudaSuccess) return FP4Q_ERR_CUDA;
-    if (fp4q_status s = fp4q_gemm_fwd(X, W, Y, ldy, dt, nullptr, ws, kStaticWorkspaceBytes, stream)) return s;
+    if (!noop)
+        if (fp4q_status s = launch_gemm<KIND_MXF4>(operand_rm(X), operand_rm(W), p, ws, kStaticWorkspaceBytes, stream)) return s;
     if (status_out &&
         cudaMemcpyAsync(status_out, ws, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return FP4Q_ERR_CUDA;
