@@ -80,13 +80,8 @@ __host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8
 // and pay for the buffers with one ring stage; the pair kernel also keeps a third image buffer, because the way
 // from "the MMAs have finished with a buffer" to "the leader may copy the next unit out of it" (commit to both
 // CTAs, build, report to the leader) is longer than one unit as well.
-// NT is the tile's width in output columns.  256: one accumulator of 256 tensor-memory columns (the other 256 hold the
-// ring of scale columns).  Narrower pair tiles (224, 192) leave room for TWO accumulators beside two or four scale
-// slots, so that the epilogue drains one tile while the MMAs of the next one already run.
-template <int KIND, int CTAS, int NT = 256>
+template <int KIND, int CTAS>
 struct Cfg {
-    static_assert(NT == 256 || (CTAS == 2 && KIND == KIND_MXF4 && NT % 32 == 0 && 2 * NT + 64 <= 512), "two-accumulator tiles: FP4 pair kernel only");
-    static constexpr int kAccs = NT == 256 ? 1 : 2;
     static constexpr bool kRowImages = KIND != KIND_MXF4;
     static constexpr int kImageBufs = (CTAS == 2 && kRowImages) ? 3 : 2;
     static constexpr int kRawBufs = kRowImages ? 2 : 0;
@@ -97,7 +92,7 @@ struct Cfg {
     static constexpr bool kTmaStores = CTAS == 2 || !kRowImages;
     static constexpr int kStages = (CTAS == 2 ? 5 : (kTmaStores ? 3 : 4)) - (kRowImages ? 1 : 0);
     static constexpr int kSmemCache = kCompactBytes + (kImageBufs + kRawBufs) * kCacheBufBytes;
-    static constexpr int kBRows = CTAS == 2 ? NT / 2 : NT;
+    static constexpr int kBRows = CTAS == 2 ? 128 : 256;
     static constexpr int kBStageBytes = kBRows * 128;
     static constexpr int kSmemOperands = kStages * (kAStageBytes + kBStageBytes);
     static constexpr int kSmemScales = (kSmemCache + 1023) / 1024 * 1024;
@@ -106,15 +101,11 @@ struct Cfg {
     static_assert(kSmemGroups == 0 || kSmemGroups >= kMaxRowTilesShared * 2, "group table");
     static constexpr int kSmemBytes = 1024 + kSmemOperands + kSmemScales + kSmemStaging + kSmemTail + kSmemGroups;
     static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
-    // tensor memory: accumulators first, then the scale slots (32 columns each: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk))
-    static constexpr int kTmemSfBase = kAccs * NT;
-    static constexpr int kSfSlots = kAccs == 1 ? kStages : (512 - kAccs * NT) / 32;
-    static_assert(kTmemSfBase % 32 == 0 && kTmemSfBase + kSfSlots * 32 <= 512 && kSfSlots >= 2, "tensor memory budget");
 };
 constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
-constexpr int kTmemSfStride = 32;            // per scale slot: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
+constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
 constexpr uint32_t kWaitLimit = 1u << 22;       // default number of polls after which a wait gives up (workspace word 2 overrides it)
 constexpr int kRelaxedNs = 64, kLazyNs = 256;   // back-off between polls of roles with slack
 // Developer diagnostic (off by default): -DFP4Q_TRACE makes CTA 0 add up clock64() intervals of its roles in
@@ -159,7 +150,6 @@ struct GemmParams {
     int32_t M, N, K;                 // per-problem output rows, output columns, contraction length (elements)
     int32_t m_tiles, n_tiles, n_tile_total;   // m_tiles counts rows of 128 * ctas
     int32_t ctas;                    // CTAs per tile (1, or 2 for cta_group::2 pairs)
-    int32_t bn;                      // tile width in output columns (256; 224 or 192 for the two-accumulator pair kernel)
     int32_t raster_m;                // tile order: groups of raster_m row tiles, within a group row tile fastest
     int32_t out_f32, accumulate;
     int32_t wide_stores;             // output base and row pitch are 32-byte aligned: 256-bit stores (whole sectors)
@@ -390,11 +380,11 @@ __device__ __forceinline__ uint64_t smem_desc_scale_image(uint32_t addr)
 }
 
 // Instruction descriptor of the block-scaled MMA: formats, K-major operands, N, UE8M0 scales, M, scale byte ids.
-template <int KIND, int CTAS, int NT>
+template <int KIND, int CTAS>
 __device__ __forceinline__ uint32_t instr_desc(uint32_t a_sf_id, uint32_t b_sf_id)
 {
     const uint32_t fmt = kind_fp4(KIND) ? 1u : 0u;   // mxf4: E2M1 = 1; mxf8f6f4: E4M3 = 0
-    return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(NT >> 3) << 17) | (1u << 23) |
+    return (b_sf_id << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) |
            ((uint32_t)((BM * CTAS) >> 4) << 24) | (a_sf_id << 29);
 }
 
@@ -446,14 +436,14 @@ __device__ __forceinline__ void decode_tile(const GemmParams &p, int tile, int r
     const int m0 = grp_m * p.raster_m, gsz = min(p.raster_m, p.m_tiles - m0);
     const int n_blk = in_grp / gsz, m_blk = m0 + (in_grp - n_blk * gsz);
     t.a_row0 = (m_blk * p.ctas + rank) * BM;
-    t.b_row0 = n_blk * p.bn;
-    t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * (p.bn >> 1) : 0);
+    t.b_row0 = n_blk * BN;
+    t.b_load_row0 = t.b_row0 + (p.ctas == 2 ? rank * 128 : 0);
     t.a_k0 = t.b_k0 = 0;
     t.k_len = p.K;
     t.c_row0 = t.a_row0;
     t.c_col0 = t.b_row0;
     t.m_valid = min(BM, p.M - t.a_row0);
-    t.n_valid = min(p.bn, p.N - t.b_row0);
+    t.n_valid = min(BN, p.N - t.b_row0);
     if (p.mode == MODE_GROUPED_ROWS) {
         if (!need_b) return;
         const int grp = goffs ? (int)reinterpret_cast<const uint16_t *>(goffs)[t.a_row0 / BM]
@@ -968,7 +958,7 @@ __device__ __forceinline__ void read_raw_scales(const GemmParams &p, const uint8
 
 // ---------------------------------------------------------------------------------------- kernel
 
-template <int KIND, int CTAS, int EPI, int NT>
+template <int KIND, int CTAS, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmD,
@@ -977,20 +967,20 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kStageElems = kind_fp4(KIND) ? 256 : 128;   // contraction elements per stage (128 B per row)
     constexpr int kMmaK = kind_fp4(KIND) ? 64 : 32;           // contraction elements per MMA (32 B per row)
     constexpr int kElemsPerByte = kind_fp4(KIND) ? 2 : 1;
-    constexpr int kStages = Cfg<KIND, CTAS, NT>::kStages;
-    constexpr int kBStageBytes = Cfg<KIND, CTAS, NT>::kBStageBytes;
+    constexpr int kStages = Cfg<KIND, CTAS>::kStages;
+    constexpr int kBStageBytes = Cfg<KIND, CTAS>::kBStageBytes;
     constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8 : kUnitStagesMxf4R;   // stages whose scale images are built together
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *smem_a = smem;
     uint8_t *smem_b = smem + kStages * kAStageBytes;
-    uint8_t *smem_compact = smem + Cfg<KIND, CTAS, NT>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
+    uint8_t *smem_compact = smem + Cfg<KIND, CTAS>::kSmemOperands;   // 2D blocks: compact scale rows of the unit being built ...
     uint8_t *smem_images = smem_compact + kCompactBytes;        // ... and the buffers of ready scale images (any kind)
-    uint8_t *smem_raw_scales = smem_images + Cfg<KIND, CTAS, NT>::kImageBufs * kCacheBufBytes;   // per-row scales: bytes in flight
-    uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS, NT>::kSmemScales;   // 1024-byte aligned (pair kernel only)
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS, NT>::kSmemStaging);
-    // bars[0..5] full, bars[6..11] empty, bars[12] / bars[14] accumulator 0 / 1 full, bars[13] / bars[15] accumulator 0 / 1 empty,
+    uint8_t *smem_raw_scales = smem_images + Cfg<KIND, CTAS>::kImageBufs * kCacheBufBytes;   // per-row scales: bytes in flight
+    uint8_t *smem_staging = smem_compact + Cfg<KIND, CTAS>::kSmemScales;   // 1024-byte aligned (pair kernel only)
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_staging + Cfg<KIND, CTAS>::kSmemStaging);
+    // bars[0..5] full, bars[6..11] empty, bars[12] accumulator full, bars[13] accumulator empty,
     // bars[18] tensor pipe drained (abort path), bars[24..27] scale images full, bars[28..31] scale images empty,
     // bars[32..35] (leader of a pair) the second CTA's scale images full - one of each per image buffer
     uint32_t *tmem_base_slot = reinterpret_cast<uint32_t *>(bars + 21);
@@ -1007,9 +997,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     const uint32_t bar_acc_full = smem_u32(bars + 12), bar_acc_empty = smem_u32(bars + 13);
     const uint32_t bar_cache_full = smem_u32(bars + 24), bar_cache_empty = smem_u32(bars + 28);
     const uint32_t bar_drain = smem_u32(bars + 18), bar_peer_cache_full = smem_u32(bars + 32);
-    constexpr int kImageBufs = Cfg<KIND, CTAS, NT>::kImageBufs;
-    constexpr int kAccs = Cfg<KIND, CTAS, NT>::kAccs;                 // accumulators in tensor memory (tiles alternate)
-    constexpr int kTmemSfBase = Cfg<KIND, CTAS, NT>::kTmemSfBase, kSfSlots = Cfg<KIND, CTAS, NT>::kSfSlots;
+    constexpr int kImageBufs = Cfg<KIND, CTAS>::kImageBufs;
 
     // In a pair, rank 0 leads: it owns the "full" and "accumulator empty" barriers and issues every tcgen05.mma.
     const int rank = CTAS == 2 ? (int)cluster_ctarank() : 0;
@@ -1023,12 +1011,10 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);    // tcgen05.commit
         }
-        for (int a = 0; a < kAccs; a++) {
-            mbar_init(bar_acc_full + 16 * a, 1);
-            mbar_init(bar_acc_empty + 16 * a, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
-        }
+        mbar_init(bar_acc_full, 1);
         mbar_init(bar_drain, 1);
-        for (int b = 0; b < Cfg<KIND, CTAS, NT>::kImageBufs; b++) {
+        mbar_init(bar_acc_empty, 8 * CTAS);     // one arrival per epilogue warp (of both CTAs of a pair)
+        for (int b = 0; b < Cfg<KIND, CTAS>::kImageBufs; b++) {
             mbar_init(bar_cache_full + 8 * b, 1);
             mbar_init(bar_cache_empty + 8 * b, 1);
             mbar_init(bar_peer_cache_full + 8 * b, 1);
@@ -1037,7 +1023,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
-        if (Cfg<KIND, CTAS, NT>::kTmaStores) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
+        if (Cfg<KIND, CTAS>::kTmaStores) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmC) : "memory");
         if (EPI == EPI_QUANT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmD) : "memory");
     }
     if (warp == 1) {
@@ -1053,7 +1039,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     }
     // grouped products: a 32-bit copy of the group boundaries for the per-tile lookups of every role
     const int n_row_tiles = (p.M + BM - 1) / BM;
-    const bool goffs_ok = Cfg<KIND, CTAS, NT>::kSmemGroups > 0 &&
+    const bool goffs_ok = Cfg<KIND, CTAS>::kSmemGroups > 0 &&
                           ((p.mode == MODE_GROUPED_K && p.n_groups <= kMaxGroupsShared) ||
                            (p.mode == MODE_GROUPED_ROWS && n_row_tiles <= kMaxRowTilesShared && p.n_groups <= 65535));
     if (goffs_ok && p.mode == MODE_GROUPED_K)
@@ -1141,7 +1127,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0, acc = 0, sf_slot = 0;
+        uint32_t stage = 0;
         BufRing ring;   // image buffer of the current unit
         const bool issuer = elect_one();
         int ev_j = 0;
@@ -1159,10 +1145,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
                 if (issuer) {
-                    // one accumulator: the scale slot follows the ring stage; two: a short ring of its own (copies
-                    // and MMAs execute in issue order, so a slot may be rewritten two stages later)
-                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + (kAccs == 1 ? stage : sf_slot) * kTmemSfStride;
-                    const uint32_t d_tmem = tmem_base + acc * NT;
+                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
                     if (KIND == KIND_MXF4) {
                         const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
@@ -1194,13 +1177,13 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         if (i < n_mma) {
                             const int chunk = kind_fp4(KIND) ? (i >> 1) : 0;
                             const uint32_t sf_id = kind_fp4(KIND) ? 2u * (i & 1) : (uint32_t)i;
-                            tcgen05_mma_block_scaled<KIND, CTAS>(d_tmem, adesc + 2 * i, bdesc + 2 * i,
-                                                                 instr_desc<KIND, CTAS, NT>(sf_id, sf_id), sf_tmem + 4 * chunk,
+                            tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
+                                                                 instr_desc<KIND, CTAS>(sf_id, sf_id), sf_tmem + 4 * chunk,
                                                                  sf_tmem + 8 + 8 * chunk, (it > 0 || i > 0) ? 1u : 0u);
                         }
                     }
                     tcgen05_commit<CTAS>(bar_empty + 8 * stage);
-                    if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full + 16 * acc);
+                    if (it == n_it - 1) tcgen05_commit<CTAS>(bar_acc_full);
                     if ((it & (kUnitStages - 1)) == kUnitStages - 1 || it == n_it - 1)
                         tcgen05_commit<CTAS>(bar_cache_empty + 8 * ring.buf);   // the unit's images have been copied
                 }
@@ -1209,9 +1192,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (lane == 0) TRACE_EV(3, ev_j);
                 ev_j++;
                 if (++stage == kStages) stage = 0;
-                if (++sf_slot == kSfSlots) sf_slot = 0;
             }
-            if (kAccs == 2) acc ^= 1u;
         }
         if (leader && *abort_flag) {
             // Some role gave up: the watchers then release every remaining stage unseen, and this warp has run
@@ -1240,7 +1221,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             // per-row scales: the raw bytes of the next kRawBufs units are in flight (cp.async) while a unit is
             // turned into images.  In a pair an image buffer is released by the leader's multicast commit: probe
             // (a suspended try_wait is not reliably woken early by a remote arrival).
-            constexpr int kRawBufs = Cfg<KIND, CTAS, NT>::kRawBufs > 0 ? Cfg<KIND, CTAS, NT>::kRawBufs : 1;
+            constexpr int kRawBufs = Cfg<KIND, CTAS>::kRawBufs > 0 ? Cfg<KIND, CTAS>::kRawBufs : 1;
             UnitIter ahead, cur;
             ahead.init(p, first_tile, tile_step, rank, goffs);
             cur.init(p, first_tile, tile_step, rank, goffs);
@@ -1334,7 +1315,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // to its end.
         StageIter sg;
         sg.init(p, first_tile, tile_step, rank, kStageElems, goffs, false);
-        uint32_t stage = 0, phase = 0, acc_phase = 0, acc = 0;   // acc_phase: bit a = phase of accumulator a's "empty" barrier
+        uint32_t stage = 0, phase = 0, acc_phase = 0;
         BufRing ring;   // image buffer of the current unit
         bool ok = true;
         TRACE_DECL(c_meet); TRACE_DECL(c_poll);
@@ -1378,8 +1359,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     const uint32_t nb0 = bar_cache_full + 8 * nu.buf, nb1 = (CTAS == 2 ? bar_peer_cache_full : bar_cache_full) + 8 * nu.buf;
                     if (KIND == KIND_MXF4 && ok && (sg.it & (kUnitStages - 1)) >= kUnitStages / 2 && !unit_seen)
                         unit_seen = mbar_test_wait(nb0, nu.phase) && (CTAS == 1 || mbar_test_wait(nb1, nu.phase));
-                    if (ok && sg.it == 0)
-                        ok = mbar_wait_impl<0, true>(bar_acc_empty + 16 * acc, ((acc_phase >> acc) & 1u) ^ 1u, abort_flag, p.status, wait_limit, 0x200u + acc);
+                    if (ok && sg.it == 0) ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.status, wait_limit, 0x200u);
                     if (ok) {
                         // A probe of an mbarrier takes this warp a few hundred cycles even when the phase is long
                         // complete, more than the MMA warp needs per stage.  So the slot's "full" barrier and those of
@@ -1441,10 +1421,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             ev_j++;
             named_sync(1 + stage);   // rendezvous: the MMA warp is at most one stage behind
             TRACE_ADD(c_meet, tt);
-            if (sg.it == 0) {
-                acc_phase ^= 1u << acc;
-                if (kAccs == 2) acc ^= 1u;
-            }
+            if (sg.it == 0) acc_phase ^= 1u;
             if ((sg.it & (kUnitStages - 1)) == kUnitStages - 1 || sg.it == sg.n_it - 1) ring.next(kImageBufs);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
             sg.next(p, kStageElems);
@@ -1588,7 +1565,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                         bulk_commit();
                     }
                 }
-            } else if (Cfg<KIND, CTAS, NT>::kTmaStores) {
+            } else if (Cfg<KIND, CTAS>::kTmaStores) {
                 // 128 bytes per row and round - 64 BF16 or 32 FP32 columns - go
                 // through this warp's staging rows and leave by a TMA store, which clips rows and columns past the
                 // output's edge.  With accumulation the store is the TMA's FP32 add-reduction.
@@ -1628,7 +1605,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             }
             TRACE_ADD(c_store, tt);
         }
-        if ((Cfg<KIND, CTAS, NT>::kTmaStores || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
+        if ((Cfg<KIND, CTAS>::kTmaStores || EPI == EPI_QUANT) && lane == 0) bulk_wait_all();   // every store of this warp is complete before the CTA ends
         if (warp == 4 && lane == 0) { TRACE_OUT(p, 10, c_wait); TRACE_OUT(p, 11, c_ld); TRACE_OUT(p, 12, c_store); }
     }
 
@@ -1746,7 +1723,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
         if (!make_byte_map(&tmC, p.q_rm, p.M, round_up(p.N, 32) / 2, p.q_ld_rm, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return FP4Q_ERR_CUDA;
         if (p.q_t && !make_byte_map(&tmD, p.q_t, p.N, round_up(p.M, 32) / 2, p.q_ld_t, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) return FP4Q_ERR_CUDA;
     } else if (!make_output_map(&tmC, p.C, out_rows, p.N, p.ldc, p.out_f32 != 0, p.accumulate != 0)) return FP4Q_ERR_CUDA;
-    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<KIND, CTAS, NT>::kBRows)) return FP4Q_ERR_CUDA;
+    if (!make_operand_map(&tmB, B.payload, B.rows, B.row_bytes, B.ld_bytes, Cfg<KIND, CTAS>::kBRows)) return FP4Q_ERR_CUDA;
     p.ctas = CTAS;
     p.m_tiles = (int32_t)ceil_div(p.M, BM * CTAS);
     p.n_tile_total = p.m_tiles * p.n_tiles * (p.mode == MODE_GROUPED_K ? p.n_groups : 1);
@@ -1760,7 +1737,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     static bool attr_set[kMaxDevices];   // the attribute is a property of (kernel, device): one flag per device and instantiation
     if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_block_scaled_kernel<KIND, CTAS, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<KIND, CTAS, NT>::kSmemBytes) != cudaSuccess)
+                                 Cfg<KIND, CTAS>::kSmemBytes) != cudaSuccess)
             return FP4Q_ERR_CUDA;
         attr_set[dev] = true;
     }
@@ -1772,7 +1749,7 @@ static fp4q_status launch_gemm_impl(const Operand &A, const Operand &B, GemmPara
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = Cfg<KIND, CTAS, NT>::kSmemBytes;
+    cfg.dynamicSmemBytes = Cfg<KIND, CTAS>::kSmemBytes;
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
