@@ -59,7 +59,8 @@ typedef enum { FP4Q_OUT_BF16 = 0, FP4Q_OUT_F32 = 1 } fp4q_out;
 /* Block-size study (Table 4 of the paper): quantize with 16 x 16 or 64 x 64 blocks instead of 32 x 32.
  * FP4Q_BLOCK_64: the scale matrix keeps its 32-granular shape, each block's scale written to its four entries, so the
  *   tensor is a valid operand of every GEMM entry point (the hardware's scale vectors are 32 wide).
- * FP4Q_BLOCK_16: scale is [ceil(rows/16), ld_s >= ceil(cols/16)]; such a tensor cannot be passed to the GEMMs. */
+ * FP4Q_BLOCK_16: scale is [ceil(rows/16), ld_s >= ceil(cols/16)]; such a tensor is an operand of the three
+ *   fp4q_gemm_*_b16 products only (16-element scale vectors are a different mode of the tensor cores). */
 #define FP4Q_BLOCK_16 2u
 #define FP4Q_BLOCK_64 4u
 
@@ -302,6 +303,23 @@ fp4q_status fp4q_gemm_fwd_quantized(const fp4q_tensor *X, const fp4q_tensor *W, 
 fp4q_status fp4q_gemm_dgrad_quantized(const fp4q_tensor *dY, const fp4q_tensor *W, const fp4q_tensor *dXq,
                                       fp4q_round mode, uint64_t seed, uint32_t tensor_id, const fp4q_groups *g,
                                       void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * fp4q_gemm_fwd_b16 / fp4q_gemm_dgrad_b16 / fp4q_gemm_wgrad_b16 -- the three products of Section 3 on tensors
+ * quantized in 16 x 16 blocks (the block-size study of Table 4 and the appendix "Block size"): operands are
+ * fp4q_tensor descriptors written by fp4q_quantize2d with FP4Q_BLOCK_16, i.e. the usual two payloads and a scale
+ * matrix [ceil(rows/16), ld_s >= ceil(cols/16)]; the scale of element (i, j) is scale[i/16, j/16], read transposed for
+ * the transposed payload exactly as in the 32 x 32 case.  Same outputs, accumulation, alignment rules, workspace and
+ * error behaviour as fp4q_gemm_fwd / _dgrad / _wgrad; dense form only.  Mixing block sizes in one product is not
+ * supported (both operands must be 16-block tensors; the library cannot tell, the scale matrix's shape is the caller's
+ * statement).
+ */
+fp4q_status fp4q_gemm_fwd_b16(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt,
+                              void *ws, size_t ws_bytes, void *stream);
+fp4q_status fp4q_gemm_dgrad_b16(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt,
+                                void *ws, size_t ws_bytes, void *stream);
+fp4q_status fp4q_gemm_wgrad_b16(const fp4q_tensor *dY, const fp4q_tensor *X, void *dW, int64_t ldw, fp4q_out dt,
+                                int accumulate, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * fp4q_gemm_fwd_static_workspace -- no counterpart in the paper: the dense forward product of

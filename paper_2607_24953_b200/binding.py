@@ -29,7 +29,8 @@ EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgr
            "fp4q_mxfp8_quantize1d", "fp4q_mxfp8_qk", "fp4q_workspace_bytes", "fp4q_workspace_status",
            "fp4q_status_string", "fp4q_version", "fp4q_gemm_fwd_static_workspace", "fp4q_workspace_set_wait_limit",
            "fp4q_debug_withhold_load", "fp4q_quantize1d", "fp4q_quantize1d_t", "fp4q_gemm_fwd_act1d", "fp4q_gemm_wgrad_act1d",
-           "fp4q_mxfp8_quantize1d_t", "fp4q_mxfp8_gemm", "fp4q_gemm_fwd_quantized", "fp4q_gemm_dgrad_quantized"]
+           "fp4q_mxfp8_quantize1d_t", "fp4q_mxfp8_gemm", "fp4q_gemm_fwd_quantized", "fp4q_gemm_dgrad_quantized",
+           "fp4q_gemm_fwd_b16", "fp4q_gemm_dgrad_b16", "fp4q_gemm_wgrad_b16"]
 
 
 class Fp4qError(RuntimeError):
@@ -109,6 +110,13 @@ def lib() -> ctypes.CDLL:
         L.fp4q_gemm_fwd_quantized.restype = ci
         L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
                                               ctypes.POINTER(_CTensor), ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
+        b16_args = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64, ci, vp, ctypes.c_size_t, vp]
+        L.fp4q_gemm_fwd_b16.restype = ci
+        L.fp4q_gemm_fwd_b16.argtypes = b16_args
+        L.fp4q_gemm_dgrad_b16.restype = ci
+        L.fp4q_gemm_dgrad_b16.argtypes = b16_args
+        L.fp4q_gemm_wgrad_b16.restype = ci
+        L.fp4q_gemm_wgrad_b16.argtypes = b16_args[:5] + [ci] + b16_args[5:]
         _lib = L
     return _lib
 
@@ -142,11 +150,13 @@ class QTensor:
     q_rm: torch.Tensor               # uint8 [rows, ld_rm]
     q_t: Optional[torch.Tensor]      # uint8 [cols, ld_t] or None
     scale: torch.Tensor              # uint8 [ceil(rows/32), ld_s] ([ceil(rows/16), ld_s] after BLOCK_16)
-    scale_granularity: int = 32      # 16 only for tensors quantized with BLOCK_16, which the GEMMs cannot take
+    scale_granularity: int = 32      # 16 only for tensors quantized with BLOCK_16, which only the *_b16 products take
 
-    def c_struct(self, as_quantizer_output: bool = False) -> _CTensor:
-        if self.scale_granularity != 32 and not as_quantizer_output:
-            raise ValueError("a tensor quantized in 16 x 16 blocks is not a GEMM operand (the hardware's scale vectors are 32 wide)")
+    def c_struct(self, granularity: int = 32) -> _CTensor:
+        """granularity: the scale granularity the callee expects (0 = any: the quantizer's own output)."""
+        if granularity and self.scale_granularity != granularity:
+            raise ValueError("this call takes tensors quantized in %d x %d blocks (scale matrix of that granularity); got %d"
+                             % (granularity, granularity, self.scale_granularity))
         return _CTensor(self.rows, self.cols,
                         self.q_rm.data_ptr(), self.q_rm.stride(0),
                         self.q_t.data_ptr() if self.q_t is not None else None,
@@ -178,7 +188,7 @@ def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = 
     rows, cols = x.shape
     if out is None:
         out = alloc_qtensor(rows, cols, x.device, want_t, 16 if flags & BLOCK_16 else 32)
-    cs = out.c_struct(as_quantizer_output=True)
+    cs = out.c_struct(granularity=0)
     st = lib().fp4q_quantize2d(x.data_ptr(), rows, cols, x.stride(0) if rows else cols, ctypes.byref(cs),
                                mode, seed, tensor_id, flags, _stream(stream))
     _check(st, "fp4q_quantize2d")
@@ -423,6 +433,38 @@ def fp4q_gemm_wgrad(dY: QTensor, X: QTensor, out=None, dt: int = OUT_F32, accumu
     e = 1 if row_offsets is None else row_offsets.numel() - 1
     return _gemm("fp4q_gemm_wgrad", dY, X, dY.cols * e, X.cols, out, dt, row_offsets, ws, stream,
                  accumulate=accumulate)
+
+
+def _gemm_b16(fn_name, a: QTensor, b: QTensor, out_rows, out_cols, out, dt, ws, stream, accumulate=None):
+    dev = a.q_rm.device
+    if out is None:
+        out = _out_buffer(out_rows, out_cols, dt, dev)
+        if accumulate:
+            out.zero_()
+    if ws is None:
+        ws = alloc_workspace(dev)
+    ca, cb = a.c_struct(16), b.c_struct(16)
+    args = [ctypes.byref(ca), ctypes.byref(cb), out.data_ptr(), out.stride(0) if out.numel() else out_cols, dt]
+    if accumulate is not None:
+        args.append(int(accumulate))
+    args += [ws.data_ptr(), ws.numel(), _stream(stream)]
+    _check(getattr(lib(), fn_name)(*args), fn_name)
+    return out
+
+
+def fp4q_gemm_fwd_b16(X: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, ws=None, stream=None):
+    """Y[T,N] = X^ W^^T on tensors quantized in 16 x 16 blocks (fp4q_quantize2d with BLOCK_16)."""
+    return _gemm_b16("fp4q_gemm_fwd_b16", X, W, X.rows, W.rows, out, dt, ws, stream)
+
+
+def fp4q_gemm_dgrad_b16(dY: QTensor, W: QTensor, out=None, dt: int = OUT_BF16, ws=None, stream=None):
+    """dX[T,K] = dY^ W^ on tensors quantized in 16 x 16 blocks."""
+    return _gemm_b16("fp4q_gemm_dgrad_b16", dY, W, dY.rows, W.cols, out, dt, ws, stream)
+
+
+def fp4q_gemm_wgrad_b16(dY: QTensor, X: QTensor, out=None, dt: int = OUT_F32, accumulate: bool = False, ws=None, stream=None):
+    """dW[N,K] (+)= dY^^T X^ on tensors quantized in 16 x 16 blocks."""
+    return _gemm_b16("fp4q_gemm_wgrad_b16", dY, X, dY.cols, X.cols, out, dt, ws, stream, accumulate=accumulate)
 
 
 def fp4q_mxfp8_qk(xq, xs, wq_q, wq_s, wk_q, wk_s, T: int, K: int, N: int, dt: int = OUT_BF16, ws=None,

@@ -60,6 +60,11 @@ static_assert(kUnitStagesMxf8 * kImageStageBytesMxf8 == kCacheBufBytes, "both ki
 constexpr int kUnitStagesMxf4R = 4;
 constexpr int kImageStageBytesMxf4R = 3072;
 static_assert(kUnitStagesMxf4R * kImageStageBytesMxf4R == kCacheBufBytes, "all kinds share the image buffers");
+// mxf4nvf4 with 16-element scale vectors (tensors quantized in 16 x 16 blocks): every MMA (64 contraction elements)
+// has its own image per 128 operand rows - four scale bytes per row - so a stage holds A 4 x 512 B and B 8 x 512 B
+constexpr int kUnitStagesMxf4B16 = 2;
+constexpr int kImageStageBytesMxf4B16 = 6144;
+static_assert(kUnitStagesMxf4B16 * kImageStageBytesMxf4B16 == kCacheBufBytes, "all kinds share the image buffers");
 // Epilogue staging of the pair kernel: each of the 8 epilogue warps owns 32 rows x 128 bytes, written from registers
 // (128-byte swizzle: the 16-byte pieces of 8 rows fall into different banks) and drained by a TMA store, which keeps
 // the output off the load/store unit that the MMA warp's instructions also pass through.
@@ -71,7 +76,9 @@ constexpr int kStagingWarpBytes = 32 * 128;
 // KIND_MXF4: FP4 payloads, 2D-block scales on both operands (replicated scale images).  KIND_MXF8: E4M3 payloads,
 // per-row scales.  KIND_MXF4R: FP4 payloads with per-row scale images - an operand quantized in 1D blocks (the
 // paper's activation layout) next to a 2D-block operand, whose tile scale is then expanded to its 32 rows.
-enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2 };
+// KIND_MXF4B16: FP4 payloads of tensors quantized in 16 x 16 blocks (block-size study): 16-element scale vectors
+// (kind::mxf4nvf4, scale_vec::4X, UE8M0 scales), real images built like the per-row kinds' (row_shift 4).
+enum { KIND_MXF4 = 0, KIND_MXF8 = 1, KIND_MXF4R = 2, KIND_MXF4B16 = 3 };
 __host__ __device__ constexpr bool kind_fp4(int kind) { return kind != KIND_MXF8; }
 
 // Per-row scale images are rebuilt every 4 (FP4) or 8 (MXFP8) stages from 12 KB of scale bytes, whose global-memory
@@ -105,7 +112,12 @@ struct Cfg {
 constexpr int kRasterM = 16;                 // dense products: row tiles per rasterisation group
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
-constexpr int kTmemSfBase = 256, kTmemSfStride = 32;   // per stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk)
+constexpr int kTmemSfBase = 256;
+// scale columns per ring stage: SFA at +0 (+4 per chunk), SFB at +8 (+8 per chunk); with 16-element scale vectors
+// SFA at +0 (+4 per MMA), SFB at +16 (+8 per MMA)
+template <int KIND> struct SfCols { static constexpr int kStride = KIND == KIND_MXF4B16 ? 48 : 32; };
+static_assert(kTmemSfBase + 5 * SfCols<KIND_MXF4>::kStride <= kTmemCols && kTmemSfBase + 4 * SfCols<KIND_MXF4B16>::kStride <= kTmemCols,
+              "tensor memory budget: 256 accumulator columns + one scale slot per ring stage");
 constexpr uint32_t kWaitLimit = 1u << 22;       // default number of polls after which a wait gives up (workspace word 2 overrides it)
 constexpr int kRelaxedNs = 64, kLazyNs = 256;   // back-off between polls of roles with slack
 // Developer diagnostic (off by default): -DFP4Q_TRACE makes CTA 0 add up clock64() intervals of its roles in
@@ -338,7 +350,17 @@ template <int KIND, int CTAS>
 __device__ __forceinline__ void tcgen05_mma_block_scaled(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate)
 {
-    if (kind_fp4(KIND) && CTAS == 2) {
+    if (KIND == KIND_MXF4B16 && CTAS == 2) {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
+    } else if (KIND == KIND_MXF4B16) {
+        asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                     " tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}"
+                     ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+                     : "memory");
+    } else if (kind_fp4(KIND) && CTAS == 2) {
         asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                      " tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n}"
                      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
@@ -617,53 +639,6 @@ __device__ __forceinline__ void ldg_v4(const uint8_t *ptr, uint32_t *w)
     asm volatile("ld.global.nc.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(ptr));
 }
 
-// Builds the scale images of one unit (32 contraction blocks from k0: 8 MXFP8 stages, or 4 FP4 stages of two chunks)
-// for per-row scales.  Lane l takes operand rows l, l+32, ... (4 of A, 8 of B); the 32 scale bytes of a row for the
-// whole unit are contiguous in the scale matrix, so the common case is two 16-byte loads per row, all 24 issued
-// before any use.  An operand with 2D-block scales (row_shift 5) reads its tile's scale row instead (every lane the
-// same bytes); if that view is transposed (consecutive blocks stride_kb apart) each lane fetches one block's byte
-// and the 32 bytes are regrouped through `scratch` (12 x 32 bytes).
-// Two steps, so that the loads are in flight while the builder waits for the image buffer to be free.
-__device__ __forceinline__ void load_row_scales(const GemmParams &p, const Tile &t, int k0, uint8_t *scratch, int lane, uint32_t (&w)[12][8])
-{
-    const bool a_tr = p.sfa.row_shift != 0 && p.sfa.stride_kb != 1, b_tr = p.sfb.row_shift != 0 && p.sfb.stride_kb != 1;
-    if (a_tr || b_tr) {
-#pragma unroll
-        for (int q = 0; q < 12; q++) {
-            if (q < 4 ? a_tr : b_tr) {
-                const ScaleView &v = q < 4 ? p.sfa : p.sfb;
-                const int row = (q < 4 ? t.a_row0 + 32 * q : t.b_row0 + 32 * (q - 4)) >> v.row_shift;
-                const int kb0 = ((q < 4 ? t.a_k0 : t.b_k0) + k0) >> 5;
-                uint32_t b;
-                load_scale(v, row, kb0 + lane, b);
-                scratch[q * 32 + lane] = (uint8_t)b;
-            }
-        }
-        __syncwarp();
-    }
-#pragma unroll
-    for (int q = 0; q < 12; q++) {
-        const ScaleView &v = q < 4 ? p.sfa : p.sfb;
-        if (q < 4 ? a_tr : b_tr) {
-            const uint4 lo = reinterpret_cast<const uint4 *>(scratch + q * 32)[0], hi = reinterpret_cast<const uint4 *>(scratch + q * 32)[1];
-            w[q][0] = lo.x; w[q][1] = lo.y; w[q][2] = lo.z; w[q][3] = lo.w;
-            w[q][4] = hi.x; w[q][5] = hi.y; w[q][6] = hi.z; w[q][7] = hi.w;
-            continue;
-        }
-        const int row = (q < 4 ? t.a_row0 + lane + 32 * q : t.b_row0 + lane + 32 * (q - 4)) >> v.row_shift;
-        const int kb0 = ((q < 4 ? t.a_k0 : t.b_k0) + k0) >> 5;
-        const uint8_t *ptr = v.ptr + (int64_t)row * v.stride_row + kb0;
-        if (row < v.n_row && kb0 + 32 <= v.n_kb && v.stride_kb == 1 && (reinterpret_cast<uintptr_t>(ptr) & 15) == 0) {
-            ldg_v4(ptr, w[q]);
-            ldg_v4(ptr + 16, w[q] + 4);
-        } else {
-#pragma unroll
-            for (int st = 0; st < 8; st++) load_scale_word(v, row, kb0 + 4 * st, w[q][st]);
-        }
-    }
-    if (a_tr || b_tr) __syncwarp();   // scratch is rewritten for the next unit
-}
-
 template <int KIND>
 __device__ __forceinline__ void store_row_scale_images(const uint32_t (&w)[12][8], int n_stages, uint8_t *images, int lane)
 {
@@ -675,6 +650,21 @@ __device__ __forceinline__ void store_row_scale_images(const uint32_t (&w)[12][8
                 img[lane] = make_uint4(w[0][st], w[1][st], w[2][st], w[3][st]);           // A
                 img[32 + lane] = make_uint4(w[4][st], w[5][st], w[6][st], w[7][st]);      // B rows 0..127
                 img[64 + lane] = make_uint4(w[8][st], w[9][st], w[10][st], w[11][st]);    // B rows 128..255
+            }
+        }
+    } else if (KIND == KIND_MXF4B16) {
+        // word j of a row = the four scale bytes of MMA j of the unit (stage j / 4, MMA j % 4)
+#pragma unroll
+        for (int st = 0; st < 2; st++) {
+            if (st < n_stages) {
+                uint4 *img = reinterpret_cast<uint4 *>(images + st * kImageStageBytesMxf4B16);
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    const int j = 4 * st + i;
+                    img[32 * i + lane] = make_uint4(w[0][j], w[1][j], w[2][j], w[3][j]);                  // A, MMA i
+                    img[128 + 64 * i + lane] = make_uint4(w[4][j], w[5][j], w[6][j], w[7][j]);            // B rows 0..127
+                    img[160 + 64 * i + lane] = make_uint4(w[8][j], w[9][j], w[10][j], w[11][j]);          // B rows 128..255
+                }
             }
         }
     } else {
@@ -851,8 +841,11 @@ __device__ __forceinline__ void cp_async(uint32_t dst, const void *src, int byte
 // q < 4: A rows 32q.., q >= 4: B rows 32(q-4)..) holds 32 bytes per lane, the scale bytes of the lane's operand row.
 // A 2D-block operand (row_shift 5) needs only 32 bytes per row tile: they are packed at the start of the operand's
 // first slot; if its view is transposed (blocks stride_kb apart, row tiles contiguous) lane l fetches block l's
-// bytes for the operand's 4 or 8 row tiles into the first 8 bytes of its entry of that slot.  Bytes beyond the tensor arrive as zero.  Every lane commits
-// exactly one cp.async group per call.
+// bytes for the operand's 4 or 8 row tiles into the first 8 bytes of its entry of that slot.  With 16 x 16 blocks
+// (row_shift 4, KB_SHIFT 4: a block is 16 contraction elements and a row tile 16 rows) the unit still has 32 blocks but
+// the operand has 8 or 16 row tiles.  Bytes beyond the tensor arrive as zero.  Every lane commits exactly one
+// cp.async group per call.
+template <int KB_SHIFT>
 __device__ __forceinline__ void issue_raw_scales(const GemmParams &p, const Tile &t, int k0, uint8_t *raw, int lane)
 {
 #pragma unroll
@@ -860,14 +853,15 @@ __device__ __forceinline__ void issue_raw_scales(const GemmParams &p, const Tile
         const ScaleView &v = op == 0 ? p.sfa : p.sfb;
         const int nq = op == 0 ? 4 : 8, q0 = op == 0 ? 0 : 4;
         const int row0 = op == 0 ? t.a_row0 : t.b_row0;
-        const int kb0 = ((op == 0 ? t.a_k0 : t.b_k0) + k0) >> 5;
+        const int kb0 = ((op == 0 ? t.a_k0 : t.b_k0) + k0) >> KB_SHIFT;
+        const int n_tiles = v.row_shift != 0 ? nq << (5 - v.row_shift) : 0;   // row tiles of a 2D-block operand
         if (v.row_shift != 0 && v.stride_kb != 1) {
-            const int rt0 = row0 >> 5, kb = kb0 + lane, nbytes = nq;   // 4 or 8 row tiles, one byte each
+            const int rt0 = row0 >> v.row_shift, kb = kb0 + lane, nbytes = n_tiles;   // 4 .. 16 row tiles, one byte each
             uint8_t *dst = raw + q0 * 1024 + lane * 32;
             const uint8_t *src = v.ptr + (int64_t)kb * v.stride_kb + rt0;
             const int valid = kb < v.n_kb ? max(0, min(nbytes, v.n_row - rt0)) : 0;
             if (v.stride_row == 1 && (reinterpret_cast<uintptr_t>(src) & (nbytes - 1)) == 0) {
-                cp_async(smem_u32(dst), valid > 0 ? src : v.ptr - (reinterpret_cast<uintptr_t>(v.ptr) & 7), nbytes, valid);
+                cp_async(smem_u32(dst), valid > 0 ? src : v.ptr - (reinterpret_cast<uintptr_t>(v.ptr) & 15), nbytes, valid);
             } else {
                 for (int r = 0; r < nbytes; r++) {
                     uint32_t b;
@@ -878,10 +872,10 @@ __device__ __forceinline__ void issue_raw_scales(const GemmParams &p, const Tile
             continue;
         }
         if (v.row_shift != 0) {
-            // 2D-block operand, blocks contiguous: the 32 bytes of each of the operand's row tiles once (lanes
-            // 0 .. 2 nq - 1 copy 16 bytes each), packed at the start of the operand's first slot
-            if (lane < 2 * nq) {
-                const int rt = (row0 >> 5) + (lane >> 1), kb = kb0 + 16 * (lane & 1);
+            // 2D-block operand, blocks contiguous: the 32 bytes of each of the operand's row tiles once (two lanes
+            // per row tile copy 16 bytes each), packed at the start of the operand's first slot
+            if (lane < 2 * n_tiles) {
+                const int rt = (row0 >> v.row_shift) + (lane >> 1), kb = kb0 + 16 * (lane & 1);
                 uint8_t *dst = raw + q0 * 1024 + lane * 16;
                 const uint8_t *src = v.ptr + (int64_t)rt * v.stride_row + kb;
                 if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
@@ -933,6 +927,24 @@ __device__ __forceinline__ void read_raw_scales(const GemmParams &p, const uint8
         if (v.row_shift != 0 && v.stride_kb != 1) {
             // lane l holds block l's bytes [row tile 0..]: words of four consecutive lanes, transposed as 4x4 bytes,
             // are the four row tiles' words of one chunk
+            if (v.row_shift == 4) {
+                // 16-row tiles: 8 (A) or 16 (B) bytes per lane; operand rows l + 32 q of image row l lie in row tile
+                // 2 q + (l >> 4), so the two halves of the warp pick different tiles of each transposed word
+                const uint4 mine4 = *reinterpret_cast<const uint4 *>(raw + q0 * 1024 + lane * 32);
+                const bool hi = lane >= 16;
+#pragma unroll
+                for (int h = 0; h < (op == 0 ? 2 : 4); h++) {
+                    const uint32_t m = h == 0 ? mine4.x : h == 1 ? mine4.y : h == 2 ? mine4.z : mine4.w;
+#pragma unroll
+                    for (int j = 0; j < 8; j++) {
+                        const uint4 tr = transpose4x4_bytes(__shfl_sync(0xFFFFFFFFu, m, 4 * j), __shfl_sync(0xFFFFFFFFu, m, 4 * j + 1),
+                                                            __shfl_sync(0xFFFFFFFFu, m, 4 * j + 2), __shfl_sync(0xFFFFFFFFu, m, 4 * j + 3));
+                        w[q0 + 2 * h][j] = hi ? tr.y : tr.x;
+                        w[q0 + 2 * h + 1][j] = hi ? tr.w : tr.z;
+                    }
+                }
+                continue;
+            }
             const uint2 mine = *reinterpret_cast<const uint2 *>(raw + q0 * 1024 + lane * 32);
 #pragma unroll
             for (int h = 0; h < (op == 0 ? 1 : 2); h++) {
@@ -948,7 +960,8 @@ __device__ __forceinline__ void read_raw_scales(const GemmParams &p, const uint8
         }
 #pragma unroll
         for (int q = 0; q < nq; q++) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(v.row_shift != 0 ? raw + q0 * 1024 + q * 32 : raw + (q0 + q) * 1024 + lane * 32);
+            const int tile = v.row_shift == 4 ? 2 * q + (lane >> 4) : q;   // row tile of operand row lane + 32 q
+            const uint4 *src = reinterpret_cast<const uint4 *>(v.row_shift != 0 ? raw + q0 * 1024 + tile * 32 : raw + (q0 + q) * 1024 + lane * 32);
             const uint4 lo = src[0], hi = src[1];
             w[q0 + q][0] = lo.x; w[q0 + q][1] = lo.y; w[q0 + q][2] = lo.z; w[q0 + q][3] = lo.w;
             w[q0 + q][4] = hi.x; w[q0 + q][5] = hi.y; w[q0 + q][6] = hi.z; w[q0 + q][7] = hi.w;
@@ -969,7 +982,9 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     constexpr int kElemsPerByte = kind_fp4(KIND) ? 2 : 1;
     constexpr int kStages = Cfg<KIND, CTAS>::kStages;
     constexpr int kBStageBytes = Cfg<KIND, CTAS>::kBStageBytes;
-    constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8 : kUnitStagesMxf4R;   // stages whose scale images are built together
+    constexpr int kUnitStages = KIND == KIND_MXF4 ? kUnitStagesMxf4 : KIND == KIND_MXF8 ? kUnitStagesMxf8
+                                : KIND == KIND_MXF4R ? kUnitStagesMxf4R : kUnitStagesMxf4B16;   // stages whose scale images are built together
+    constexpr int kKbShift = KIND == KIND_MXF4B16 ? 4 : 5;    // log2 of the scale vector's length (contraction elements per scale byte)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -1145,7 +1160,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
                 if (issuer) {
-                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * kTmemSfStride;
+                    const uint32_t sf_tmem = tmem_base + kTmemSfBase + stage * SfCols<KIND>::kStride;
                     if (KIND == KIND_MXF4) {
                         const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytes);
 #pragma unroll
@@ -1153,6 +1168,14 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * c, smem_desc_scale_image_rep(img + 128 * c));
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 8 + 8 * c, smem_desc_scale_image_rep(img + 256 + 256 * c));
                             tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 12 + 8 * c, smem_desc_scale_image_rep(img + 384 + 256 * c));
+                        }
+                    } else if (KIND == KIND_MXF4B16) {
+                        const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4B16);
+#pragma unroll
+                        for (int i = 0; i < 4; i++) {
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 4 * i, smem_desc_scale_image(img + 512 * i));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 16 + 8 * i, smem_desc_scale_image(img + 2048 + 1024 * i));
+                            tcgen05_cp_32x128b_warpx4<CTAS>(sf_tmem + 20 + 8 * i, smem_desc_scale_image(img + 2560 + 1024 * i));
                         }
                     } else if (KIND == KIND_MXF4R) {
                         const uint32_t img = smem_u32(smem_images + ring.buf * kCacheBufBytes + (it & (kUnitStages - 1)) * kImageStageBytesMxf4R);
@@ -1175,6 +1198,11 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 #pragma unroll
                     for (int i = 0; i < 4; i++) {
                         if (i < n_mma) {
+                            if (KIND == KIND_MXF4B16) {   // one 32-bit scale column entry per row and MMA: all four bytes are used
+                                tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i, instr_desc<KIND, CTAS>(0u, 0u),
+                                                                     sf_tmem + 4 * i, sf_tmem + 16 + 8 * i, (it > 0 || i > 0) ? 1u : 0u);
+                                continue;
+                            }
                             const int chunk = kind_fp4(KIND) ? (i >> 1) : 0;
                             const uint32_t sf_id = kind_fp4(KIND) ? 2u * (i & 1) : (uint32_t)i;
                             tcgen05_mma_block_scaled<KIND, CTAS>(tmem_base, adesc + 2 * i, bdesc + 2 * i,
@@ -1228,7 +1256,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             uint32_t raw_fill = 0, raw_read = 0;
             for (int i = 0; i < kRawBufs; i++) {
                 if (ahead.valid(p)) {
-                    issue_raw_scales(p, ahead.t, ahead.k0, smem_raw_scales + raw_fill * kCacheBufBytes, lane);
+                    issue_raw_scales<kKbShift>(p, ahead.t, ahead.k0, smem_raw_scales + raw_fill * kCacheBufBytes, lane);
                     ahead.next(p, kUnitStages * kStageElems);
                 } else {
                     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -1255,7 +1283,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 cur.next(p, kUnitStages * kStageElems);
                 // the raw buffer just read is free: fetch the unit kRawBufs ahead into it
                 if (ahead.valid(p)) {
-                    issue_raw_scales(p, ahead.t, ahead.k0, smem_raw_scales + raw_read * kCacheBufBytes, lane);
+                    issue_raw_scales<kKbShift>(p, ahead.t, ahead.k0, smem_raw_scales + raw_read * kCacheBufBytes, lane);
                     ahead.next(p, kUnitStages * kStageElems);
                 } else {
                     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -2093,6 +2121,69 @@ extern "C" fp4q_status fp4q_gemm_wgrad_act1d(const fp4q_tensor *dY, const uint8_
     p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = accumulate ? 1 : 0;
     dense_tiles(p);
     return launch_gemm<KIND_MXF4R>(A, B, p, ws, ws_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Products on tensors quantized in 16 x 16 blocks (block-size study): same payloads, scale matrix
+// [ceil(rows/16), ceil(cols/16)], 16-element scale vectors in the MMA.  Dense only.
+namespace fp4q {
+
+static Operand operand_rm16(const fp4q_tensor *t)
+{
+    Operand o = operand_rm(t);
+    o.sf = ScaleView{t->scale, t->ld_s, 1, (int32_t)ceil_div(t->rows, 16), (int32_t)ceil_div(t->cols, 16), 4};
+    return o;
+}
+static Operand operand_t16(const fp4q_tensor *t)
+{
+    Operand o = operand_t(t);
+    o.sf = ScaleView{t->scale, 1, t->ld_s, (int32_t)ceil_div(t->cols, 16), (int32_t)ceil_div(t->rows, 16), 4};
+    return o;
+}
+
+// which: 0 forward (A = a.q_rm [M,K], B = b.q_rm [N,K]), 1 input gradient (A = a.q_rm [M,K'], B = b.q_t), 2 weight
+// gradient (A = a.q_t, B = b.q_t)
+static fp4q_status gemm_b16(int which, const fp4q_tensor *a, const fp4q_tensor *b, void *C, int64_t ldc, fp4q_out dt, int accumulate,
+                            void *ws, size_t ws_bytes, void *stream)
+{
+    if (!tensor_ok(a) || !tensor_ok(b)) return a && b ? FP4Q_ERR_SHAPE : FP4Q_ERR_NULL;
+    if (dt != FP4Q_OUT_BF16 && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    if (accumulate && dt != FP4Q_OUT_F32) return FP4Q_ERR_UNSUPPORTED;
+    int64_t M, N, K;
+    if (which == 0) { if (a->cols != b->cols) return FP4Q_ERR_SHAPE; M = a->rows; N = b->rows; K = a->cols; }
+    else if (which == 1) { if (a->cols != b->rows) return FP4Q_ERR_SHAPE; M = a->rows; N = b->cols; K = a->cols; }
+    else { if (a->rows != b->rows) return FP4Q_ERR_SHAPE; M = a->cols; N = b->cols; K = a->rows; }
+    if (M > kMaxDim || N > kMaxDim || K > kMaxDim) return FP4Q_ERR_UNSUPPORTED;
+    if (M == 0 || N == 0) return FP4Q_OK;
+    const uint8_t *pa = which == 2 ? a->q_t : a->q_rm, *pb = which == 0 ? b->q_rm : b->q_t;
+    if (!C || !pa || !pb || !a->scale || !b->scale) return FP4Q_ERR_NULL;
+    if (ldc < N) return FP4Q_ERR_SHAPE;
+    GemmParams p = {};
+    p.C = C; p.ldc = ldc; p.M = (int32_t)M; p.N = (int32_t)N; p.K = (int32_t)K;
+    p.out_f32 = dt == FP4Q_OUT_F32; p.accumulate = accumulate ? 1 : 0;
+    dense_tiles(p);
+    return launch_gemm<KIND_MXF4B16>(which == 2 ? operand_t16(a) : operand_rm16(a), which == 0 ? operand_rm16(b) : operand_t16(b), p, ws,
+                                     ws_bytes, stream);
+}
+
+}  // namespace fp4q
+
+extern "C" fp4q_status fp4q_gemm_fwd_b16(const fp4q_tensor *X, const fp4q_tensor *W, void *Y, int64_t ldy, fp4q_out dt, void *ws,
+                                         size_t ws_bytes, void *stream)
+{
+    return gemm_b16(0, X, W, Y, ldy, dt, 0, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_dgrad_b16(const fp4q_tensor *dY, const fp4q_tensor *W, void *dX, int64_t ldx, fp4q_out dt, void *ws,
+                                           size_t ws_bytes, void *stream)
+{
+    return gemm_b16(1, dY, W, dX, ldx, dt, 0, ws, ws_bytes, stream);
+}
+
+extern "C" fp4q_status fp4q_gemm_wgrad_b16(const fp4q_tensor *dY, const fp4q_tensor *X, void *dW, int64_t ldw, fp4q_out dt,
+                                           int accumulate, void *ws, size_t ws_bytes, void *stream)
+{
+    return gemm_b16(2, dY, X, dW, ldw, dt, accumulate, ws, ws_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------------------
