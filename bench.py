@@ -134,6 +134,35 @@ def aggregate_throughput(units_per_rank, world, ms):
     return world * units_per_rank / (ms * 1e-3)
 
 
+def launcher_command(n_ranks, argv, port=None):
+    """The command that starts n_ranks copies of this script, one per GPU (torch.distributed.run on this node)."""
+    port = port or (29500 + os.getpid() % 2000)
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_ranks),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def relaunch_as_ranks(args, argv):
+    """`--gpus N` with N > 1 outside a torchrun launch: start the N ranks here and hand their exit code back."""
+    return subprocess.call(launcher_command(args.gpus, argv))
+
+
+def run_rank_selftest(args):
+    """Host-side logic of the N > 1 path on CPU ranks (gloo): rendezvous, max over ranks, aggregation, one JSON line
+    from rank 0.  Used by the tests; touches no GPU."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = max_over_ranks([10.0 + rank], dist if world > 1 else None, "cpu")[0]
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "ms_per_step": ms,
+                          "value": aggregate_throughput(1000.0, world, ms), "scaling": "weak"}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------------------------------ workload
 
 def build_dense_workload(cfg, device, torch, workloads):
@@ -159,6 +188,10 @@ def run_gpu(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit("bench.py: --gpus %d but the launch has %d rank(s)" % (args.gpus, world))
+    if torch.cuda.device_count() < world:
+        raise SystemExit("bench.py: %d ranks need %d GPUs, %d visible" % (world, world, torch.cuda.device_count()))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
@@ -196,9 +229,14 @@ def run_gpu(args):
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
-    def phase_quantize():
+    def phase_quantize_per_tensor():
         for x, q, tid in quant_jobs:
             binding.fp4q_quantize2d(x, q, mode=SR, seed=seed, tensor_id=tid)
+
+    def phase_quantize():
+        # all 18 operands by one call of the library's multi-tensor entry point (chained launches in one stream)
+        binding.fp4q_quantize2d_multi([x for x, _, _ in quant_jobs], [q for _, q, _ in quant_jobs], mode=SR, seed=seed,
+                                      tensor_ids=[tid for _, _, tid in quant_jobs])
 
     def phase_fwd():
         for i, o in enumerate(ops):
@@ -225,7 +263,8 @@ def run_gpu(args):
         for st in side:
             cur.wait_stream(st)
 
-    phases = [phase_quantize, phase_fwd, phase_dgrad, phase_wgrad]
+    quantize_variant = "two-streams" if args.two_stream_quantize else "per-tensor" if args.per_tensor_quantize else "multi"
+    phases = [phase_quantize_per_tensor if quantize_variant != "multi" else phase_quantize, phase_fwd, phase_dgrad, phase_wgrad]
 
     def step(marks=None):
         for i, ph in enumerate(phases):
@@ -256,7 +295,7 @@ def run_gpu(args):
         # from Python: each phase is captured once into a CUDA graph (same kernels, same arguments, same order) and
         # the timed steps replay the graphs.
         graphs = []
-        if not args.serial_quantize:
+        if quantize_variant == "two-streams":
             phases[0] = phase_quantize_two_streams
         for ph in list(phases):
             g = torch.cuda.CUDAGraph()
@@ -402,7 +441,7 @@ def run_gpu(args):
 
     extras = {}
     if not args.no_extras:
-        extras = run_extras(torch, binding, workloads, dev, ws)
+        extras = run_extras(torch, binding, workloads, dev, ws, measured_peaks())
         if per_operand is not None:
             extras["per_operand"] = per_operand
 
@@ -436,12 +475,14 @@ def run_gpu(args):
                          "peak_source": peaks["source"] + " copy bandwidth",
                          "bytes_per_launch": quant_bytes / len(quant_jobs), "ms_per_launch": q_ms / len(quant_jobs),
                          "time_share_of_step": q_ms / ms_per_step}
-    if not args.no_graphs and not args.serial_quantize:
-        # the sweep on its own (no GEMMs between repetitions, so at cooler clocks than inside the step), as captured
-        # for the step and with its launches in one stream, one after the other
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            phase_quantize()
+    if not args.no_graphs:
+        # the sweep on its own (no GEMMs between repetitions, so at cooler clocks than inside the step): the library's
+        # multi-tensor call, one plain launch per tensor in one stream, and plain launches alternating between two streams
+        def captured(fn):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            return g
 
         def sweep_rate(replay):
             replay()
@@ -454,13 +495,26 @@ def run_gpu(args):
             torch.cuda.synchronize()
             return quant_bytes / (a.elapsed_time(b) / 10 * 1e-3) / 1e9
 
-        roofline_quantize["sweep_alone_gbs"] = {"two_streams": sweep_rate(phases[0]), "one_stream": sweep_rate(g.replay)}
-        roofline_quantize["note"] = ("launches of independent operands overlap (two streams in the graph), so ms_per_launch is "
-                                     "the phase time divided by the launch count; sweep_alone_gbs compares the two captures "
-                                     "of the sweep run on their own")
+        roofline_quantize["sweep_alone_gbs"] = {"multi_tensor_call": sweep_rate(captured(phase_quantize).replay),
+                                                "per_tensor_one_stream": sweep_rate(captured(phase_quantize_per_tensor).replay),
+                                                "per_tensor_two_streams": sweep_rate(captured(phase_quantize_two_streams).replay)}
+        roofline_quantize["note"] = ("the timed step quantizes its 18 operands with the '%s' variant; sweep_alone_gbs compares "
+                                     "the three variants of the sweep run on their own; launches of independent operands overlap, "
+                                     "so ms_per_launch is the phase time divided by the launch count" % quantize_variant)
     fill_traffic(roofline, roofline_quantize)
 
     cpu = cpu_baseline_quantize(workloads, cfg, seconds=args.cpu_seconds)
+    inputs_sha256 = None
+    if not args.no_hash:
+        import hashlib
+        names = ["W_" + o["name"] for o in ops] + ["X_" + k for k in xs] + ["dY_" + o["name"] for o in ops]
+        digest_all, per = hashlib.sha256(), {}
+        for (x, _, _), nm in zip(quant_jobs, names):
+            h = hashlib.sha256(workloads.bf16_bits(x).tobytes()).hexdigest()
+            per[nm] = h[:16]
+            digest_all.update(bytes.fromhex(h))
+        inputs_sha256 = {"all": digest_all.hexdigest(), "per_tensor_first16": per,
+                         "note": "SHA-256 of each BF16 operand's bytes (row-major); 'all' hashes the 18 digests in sweep order"}
 
     line = {
         "metric": METRIC, "value": quant_gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -472,12 +526,15 @@ def run_gpu(args):
                    "parallelism": "replicas only (x%d)" % world,
                    "launch": "per-launch calls from Python" if args.no_graphs else
                              "one CUDA graph per phase (quantize, fwd, dgrad, wgrad), replayed" +
-                             ("" if args.serial_quantize else "; the quantize sweep's independent launches alternate between two streams"), "l2": "inputs larger than L2 (%.2f GB of BF16 operands per step)" %
+                             {"multi": "; the quantize sweep is one fp4q_quantize2d_multi call (18 chained launches in one stream)",
+                              "per-tensor": "; one plain quantize launch per tensor",
+                              "two-streams": "; the quantize sweep's per-tensor launches alternate between two streams"}[quantize_variant], "l2": "inputs larger than L2 (%.2f GB of BF16 operands per step)" %
                    (quant_elems * 2 / 1e9), "quantize_bytes_per_step": quant_bytes, "gemm_flops_per_step": 3 * gemm_flops},
         "gemm_tflops": gemm_tflops,
         "phase_ms": {"quantize": q_ms, "fwd": f_ms, "dgrad": d_ms, "wgrad": w_ms},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "roofline": roofline, "roofline_quantize": roofline_quantize, "cpu_baseline": cpu, "extras": extras,
+        "roofline": roofline, "roofline_quantize": roofline_quantize, "cpu_baseline": cpu, "inputs_sha256": inputs_sha256,
+        "extras": extras,
     }
     print(json.dumps(line))
     if dist is not None:
@@ -501,9 +558,16 @@ def fill_traffic(roofline, roofline_quantize):
         pass
 
 
-def run_extras(torch, binding, workloads, dev, ws):
+def bound_of(flops, alg_bytes, tensor_tflops, hbm_gbs):
+    """Roofline of one product: the slower of its flops at the tensor peak and its algorithmic bytes at the HBM rate."""
+    t_tensor, t_hbm = flops / (tensor_tflops * 1e12), alg_bytes / (hbm_gbs * 1e9)
+    return {"bound": "tensor" if t_tensor >= t_hbm else "hbm", "ms": max(t_tensor, t_hbm) * 1e3}
+
+
+def run_extras(torch, binding, workloads, dev, ws, peaks):
     """MXFP8 query/key projections at 7B shapes and the grouped MoE expert layer, timed on their own."""
     out = {}
+    fp4_peak, fp8_peak, hbm = peaks["bf16_tflops"] * FP4_OVER_BF16, peaks["bf16_tflops"] * FP8_OVER_BF16, peaks["hbm_gbs"]
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
     def timed(fn, iters=5):
@@ -528,9 +592,14 @@ def run_extras(torch, binding, workloads, dev, ws):
     wkq, wks = binding.fp4q_mxfp8_quantize1d(Wk)
     ms_q = timed(lambda: binding.fp4q_mxfp8_quantize1d(X))
     ms_g = timed(lambda: binding.fp4q_mxfp8_qk(xq, xs, wqq, wqs, wkq, wks, T, H, H, ws=ws))
+    qk_tf = 2 * 2.0 * T * H * H / (ms_g * 1e-3) / 1e12
     out["mxfp8_qk"] = {"workload": "Q and K projections, %d tokens, %dx%d each" % (T, H, H),
                        "quantize_gbs": T * H * (3.0 + 1 / 32) / (ms_q * 1e-3) / 1e9,
-                       "gemm_tflops": 2 * 2.0 * T * H * H / (ms_g * 1e-3) / 1e12, "gemm_ms": ms_g}
+                       "gemm_tflops": qk_tf, "gemm_ms": ms_g,
+                       "roofline": {"kernel": "gemm_block_scaled_kernel<mxf8f6f4>", "bound": "tensor", "achieved": qk_tf, "peak": fp8_peak,
+                                    "unit": "TFLOP/s", "frac": qk_tf / fp8_peak, "frac_of_nominal_4500": qk_tf / 4500.0,
+                                    "peak_source": "%s bf16 burst %.1f TFLOP/s x %.0f (nominal FP8:BF16 ratio)" %
+                                                   (peaks["source"], peaks["bf16_tflops"], FP8_OVER_BF16)}}
     # backward of the same projections: operands re-quantized along the new contraction axis
     dYq = workloads.gradients_rowscaled(T, H, cfg.data_seed + 2, dev)
     ms_qt = timed(lambda: binding.fp4q_mxfp8_quantize1d_t(X))
@@ -558,6 +627,23 @@ def run_extras(torch, binding, workloads, dev, ws):
         "workload": "Y = X W^T, %d x %d x %d, output as 2D-block FP4 (stochastic rounding)" % (T, H, H),
         "fused_ms": ms_f, "product_ms": ms_p, "separate_quantize_ms": ms_s,
         "fused_tflops": 2.0 * T * H * H / (ms_f * 1e-3) / 1e12, "speedup_vs_unfused": (ms_p + ms_s) / ms_f}
+    # --- block-size study (Table 4): quantize and forward product at block edges 16 / 32 / 64 on the same tensors
+    bs = {}
+    y32 = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+    for b, flag in ((16, binding.BLOCK_16), (32, 0), (64, binding.BLOCK_64)):
+        qxb, qwb = binding.fp4q_quantize2d(X, flags=flag), binding.fp4q_quantize2d(Wq, flags=flag)
+        ms_qb = timed(lambda: binding.fp4q_quantize2d(X, out=qxb, mode=SR, seed=1, tensor_id=2, flags=flag))
+        gemm = binding.fp4q_gemm_fwd_b16 if b == 16 else binding.fp4q_gemm_fwd
+        ms_gb = timed(lambda: gemm(qxb, qwb, out=y32, ws=ws))
+        bs[str(b)] = {"quantize_gbs": T * H * (3.0 + 1.0 / (b * b if b != 64 else 1024)) / (ms_qb * 1e-3) / 1e9,
+                      "fwd_tflops": 2.0 * T * H * H / (ms_gb * 1e-3) / 1e12, "fwd_ms": ms_gb}
+        del qxb, qwb
+    for b in bs:
+        bs[b]["fwd_relative_to_32"] = bs["32"]["fwd_ms"] / bs[b]["fwd_ms"]
+    bs["paper_table4_relative_throughput"] = {"8": 0.85, "16": 0.92, "32": 1.0, "64": 1.05,
+                                              "note": "the paper's idealised trend column, for context (block edge 8 is not built)"}
+    out["block_sizes"] = {"workload": "X %d x %d, W %d x %d, forward product" % (T, H, H, H), **bs}
+    del y32
     # --- the paper's mixed layout: activations in 1D blocks (two encodings of X), weights and gradients in 2D blocks
     dY4 = binding.fp4q_quantize2d(workloads.gradients_rowscaled(T, H, cfg.data_seed + 2, dev), mode=SR, seed=1, tensor_id=3)
     x1q, x1s = binding.fp4q_quantize1d(X)
@@ -601,9 +687,16 @@ def run_extras(torch, binding, workloads, dev, ws):
             ms = [timed(lambda: binding.fp4q_gemm_fwd(qx, qw, out=y, row_offsets=d_offs, ws=ws, row_alignment=pad)),
                   timed(lambda: binding.fp4q_gemm_dgrad(qdy, qw, out=dx, row_offsets=d_offs, ws=ws, row_alignment=pad)),
                   timed(lambda: binding.fp4q_gemm_wgrad(qdy, qx, out=dw, row_offsets=d_offs, ws=ws))]
+            # each product against its own bound: operand payloads + scales read once, output written once
+            pay = lambda r, c: r * c * (0.5 + 1.0 / 1024)
+            alg = [pay(Tp, k) + pay(E * n, k) + Tp * n * 2.0, pay(Tp, n) + pay(E * n, k) + Tp * k * 2.0,
+                   pay(Tp, n) + pay(Tp, k) + E * n * k * 4.0]
+            bounds = [bound_of(flops, a, fp4_peak, hbm) for a in alg]
             res[name] = {"fwd_tflops": flops / (ms[0] * 1e-3) / 1e12, "dgrad_tflops": flops / (ms[1] * 1e-3) / 1e12,
                          "wgrad_tflops": flops / (ms[2] * 1e-3) / 1e12, "ms": ms,
-                         "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9}
+                         "wgrad_output_gbs": E * n * k * 4 / (ms[2] * 1e-3) / 1e9,
+                         "bound": {nm: {"kind": b["bound"], "bound_ms": b["ms"], "frac": b["ms"] / m}
+                                   for nm, b, m in zip(("fwd", "dgrad", "wgrad"), bounds, ms)}}
             if pad == 256:   # forward product with the output quantization in the epilogue, against product + quantize
                 qy = binding.alloc_qtensor(Tp, n, dev)
                 ms_fq = timed(lambda: binding.fp4q_gemm_fwd_quantized(qx, qw, out=qy, mode=1, seed=1, tensor_id=9, ws=ws, row_offsets=d_offs))
@@ -615,6 +708,8 @@ def run_extras(torch, binding, workloads, dev, ws):
             tot_flops += 3 * flops
             del Xm, dYm, Wm, qx, qw, qdy, y, dx, dw
         res["all_tflops"] = tot_flops / (tot_ms * 1e-3) / 1e12
+        res["bound_note"] = ("per product: bound_ms = max(flops / (measured BF16 burst x 4), algorithmic bytes / measured copy "
+                             "bandwidth); frac = bound_ms / measured ms")
         out[key] = res
     if binding.fp4q_workspace_status(ws) != 0:
         out["status"] = "device-side timeout reported"
@@ -648,8 +743,20 @@ def cpu_baseline_quantize(workloads, cfg, seconds=12.0):
     wd = oracle.dequantize2d(qw[0], qw[2], 512, cols)
     oracle.gemm_fwd(xd, wd)
     g_dt = max(time.perf_counter() - t1, 1e-9)
+    # the tiny linear layer (W 256x256, X and dY 128x256) in full: three quantizations and the three products
+    tiny = {k: workloads.bf16_bits(v) for k, v in workloads.tiny_layer("cpu").items()}
+    t2 = time.perf_counter()
+    tq = {k: oracle.quantize2d(v, oracle.MODE_STOCHASTIC, seed=0, tensor_id=i) for i, (k, v) in enumerate(tiny.items())}
+    t3 = time.perf_counter()
+    td = {k: oracle.dequantize2d(q[0], q[2], tiny[k].shape[0], tiny[k].shape[1]) for k, q in tq.items()}
+    oracle.gemm_fwd(td["X"], td["W"]); oracle.gemm_dgrad(td["dY"], td["W"]); oracle.gemm_wgrad(td["dY"], td["X"])
+    t4 = time.perf_counter()
+    tiny_elems = sum(v.size for v in tiny.values())
+    tiny_full = {"quantize_gbs": tiny_elems * BYTES_PER_ELEMENT / max(t3 - t2, 1e-9) / 1e9,
+                 "gemm_gflops": 3 * 2.0 * 128 * 256 * 256 / max(t4 - t3, 1e-9) / 1e9,
+                 "sample": "the tiny linear layer in full: 3 quantizations, then dequantize + the 3 float64 products"}
     return {"value": rows * cols * BYTES_PER_ELEMENT / dt / 1e9, "unit": "GB/s", "cores": oracle.num_threads(),
-            "kind": "oracle", "seconds": dt,
+            "kind": "oracle", "seconds": dt, "tiny_layer_full": tiny_full,
             "gemm": {"value": 2.0 * g_rows * 512 * cols / g_dt / 1e9, "unit": "GFLOP/s",
                      "sample": "forward product oracle (dequantize + float64 matmul) on %d x 512 x %d" % (g_rows, cols)},
             "sample": "quantize+dual-pack (stochastic) of a %dx%d row slab of the %dx%d down-projection activation" %
@@ -672,23 +779,26 @@ def run_reference(args):
     n_tok, n_out, k = 32, 512, cfg.hidden
 
     def step():
+        """Returns (seconds in the quantizer, seconds in dequantize + the three products)."""
+        t0 = time.perf_counter()
         qs = [oracle.quantize2d(t, oracle.MODE_STOCHASTIC, seed=cfg.philox_seed, tensor_id=i) for i, t in enumerate(tensors)]
+        t1 = time.perf_counter()
         wd = oracle.dequantize2d(qs[0][0], qs[0][2], rows, cfg.hidden)
         xd = oracle.dequantize2d(qs[2][0], qs[2][2], rows, cfg.hidden)
-        t0 = time.perf_counter()
         oracle.gemm_fwd(xd[:n_tok], wd[:n_out])
         oracle.gemm_dgrad(xd[:n_tok, :rows], wd)
         oracle.gemm_wgrad(xd[:n_tok, :rows], xd[:n_tok])
-        return time.perf_counter() - t0
+        return t1 - t0, time.perf_counter() - t1
 
     for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
-    gemm_s = 0.0
+    quant_s = gemm_s = 0.0
     for _ in range(args.steps):
-        gemm_s += step()
+        q_s, g_s = step()
+        quant_s += q_s
+        gemm_s += g_s
     total = time.perf_counter() - t0
-    quant_s = total - gemm_s
     value = args.steps * elems * BYTES_PER_ELEMENT / quant_s / 1e9
     gemm_flops = 2.0 * n_tok * (n_out * k + rows * cfg.hidden + rows * cfg.hidden)
     sample = ("per step: oracle quantize+dual-pack (stochastic) of %d-row slabs of a weight, the down-projection "
@@ -780,8 +890,11 @@ def main():
     ap.add_argument("--workload", default="7b", choices=["7b", "1b", "tiny"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-hash", action="store_true", help="skip the SHA-256 of the input buffers")
     ap.add_argument("--no-graphs", action="store_true", help="issue every launch from Python instead of replaying CUDA graphs")
-    ap.add_argument("--serial-quantize", action="store_true", help="capture the quantize sweep on one stream (no overlap between operands)")
+    ap.add_argument("--per-tensor-quantize", action="store_true", help="one fp4q_quantize2d launch per operand instead of the multi-tensor launch")
+    ap.add_argument("--two-stream-quantize", action="store_true", help="per-operand launches alternating between two streams inside the graph")
+    ap.add_argument("--rank-selftest", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "quantize1d", "quantize1d_t",
                                                         "gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm"],
@@ -790,7 +903,14 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--mode", type=int, default=1, help="quantize rounding mode: 0 nearest, 1 stochastic")
     args = ap.parse_args()
-    if args.kernel:
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.kernel:
+        # not under torchrun: start one rank per GPU (replicas; rank 0 prints the line with n_gpus = N)
+        raise SystemExit(relaunch_as_ranks(args, sys.argv[1:]))
+    if args.rank_selftest:
+        run_rank_selftest(args)
+    elif args.kernel:
         run_kernel(args)
     elif args.impl == "reference":
         run_reference(args)

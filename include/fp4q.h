@@ -123,6 +123,28 @@ fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int6
                             const fp4q_tensor *out, fp4q_round mode, uint64_t seed,
                             uint32_t tensor_id, uint32_t flags, void *stream);
 
+/*
+ * fp4q_quantize2d_multi -- fp4q_quantize2d applied to several independent tensors by one call (same arithmetic, same
+ * bytes as one call per tensor; the rounding stream of tensor j is keyed on jobs[j].tensor_id).  The operands of a
+ * layer do not depend on one another and many of them are small (a 4096 x 4096 weight is a few waves of CTAs), so the
+ * call enqueues one kernel per tensor on `stream` with each kernel after the first configured as the programmatic
+ * dependent of its predecessor: it starts beside the predecessor's last wave instead of after it and completes after
+ * it, and whatever is enqueued after the call sees all tensors.  `jobs` is a HOST array of n_jobs descriptors, read
+ * during the call; the pointers inside are device pointers as for fp4q_quantize2d.  32 x 32 blocks only (flags: 0 or
+ * FP4Q_INDEX_TRANSPOSED).  The tensors must not overlap one another's outputs.  Every job is validated before anything
+ * is enqueued; empty tensors are skipped.
+ */
+typedef struct {
+    const void *x_bf16;
+    int64_t rows, cols, ld_x;
+    const fp4q_tensor *out;
+    uint32_t tensor_id;
+    uint32_t flags;
+} fp4q_quantize_job;
+
+fp4q_status fp4q_quantize2d_multi(const fp4q_quantize_job *jobs, int32_t n_jobs, fp4q_round mode, uint64_t seed,
+                                  void *stream);
+
 /* GEMM workspace: fp4q_workspace_bytes() bytes of device memory, 256-byte aligned, zeroed once by
  * the caller before first use (the kernels restore what they use).  Holds the device status word.
  * Calls that share a workspace must not overlap on the GPU. */

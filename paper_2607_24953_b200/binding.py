@@ -30,7 +30,7 @@ EXPORTS = ["fp4q_quantize2d", "fp4q_gemm_fwd", "fp4q_gemm_dgrad", "fp4q_gemm_wgr
            "fp4q_status_string", "fp4q_version", "fp4q_gemm_fwd_static_workspace", "fp4q_workspace_set_wait_limit",
            "fp4q_debug_withhold_load", "fp4q_quantize1d", "fp4q_quantize1d_t", "fp4q_gemm_fwd_act1d", "fp4q_gemm_wgrad_act1d",
            "fp4q_mxfp8_quantize1d_t", "fp4q_mxfp8_gemm", "fp4q_gemm_fwd_quantized", "fp4q_gemm_dgrad_quantized",
-           "fp4q_gemm_fwd_b16", "fp4q_gemm_dgrad_b16", "fp4q_gemm_wgrad_b16"]
+           "fp4q_gemm_fwd_b16", "fp4q_gemm_dgrad_b16", "fp4q_gemm_wgrad_b16", "fp4q_quantize2d_multi"]
 
 
 class Fp4qError(RuntimeError):
@@ -44,6 +44,11 @@ class _CTensor(ctypes.Structure):
                 ("q_rm", ctypes.c_void_p), ("ld_rm", ctypes.c_int64),
                 ("q_t", ctypes.c_void_p), ("ld_t", ctypes.c_int64),
                 ("scale", ctypes.c_void_p), ("ld_s", ctypes.c_int64)]
+
+
+class _CQuantJob(ctypes.Structure):
+    _fields_ = [("x_bf16", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("ld_x", ctypes.c_int64),
+                ("out", ctypes.POINTER(_CTensor)), ("tensor_id", ctypes.c_uint32), ("flags", ctypes.c_uint32)]
 
 
 class _CGroups(ctypes.Structure):
@@ -110,6 +115,8 @@ def lib() -> ctypes.CDLL:
         L.fp4q_gemm_fwd_quantized.restype = ci
         L.fp4q_gemm_fwd_quantized.argtypes = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor),
                                               ctypes.POINTER(_CTensor), ci, u64, u32, vp, vp, ctypes.c_size_t, vp]
+        L.fp4q_quantize2d_multi.restype = ci
+        L.fp4q_quantize2d_multi.argtypes = [ctypes.POINTER(_CQuantJob), ctypes.c_int32, ci, u64, vp]
         b16_args = [ctypes.POINTER(_CTensor), ctypes.POINTER(_CTensor), vp, i64, ci, vp, ctypes.c_size_t, vp]
         L.fp4q_gemm_fwd_b16.restype = ci
         L.fp4q_gemm_fwd_b16.argtypes = b16_args
@@ -193,6 +200,27 @@ def fp4q_quantize2d(x: torch.Tensor, out: Optional[QTensor] = None, mode: int = 
                                mode, seed, tensor_id, flags, _stream(stream))
     _check(st, "fp4q_quantize2d")
     return out
+
+
+def fp4q_quantize2d_multi(xs, outs=None, mode: int = ROUND_NEAREST, seed: int = 0, tensor_ids=None, flags: int = 0,
+                          want_t: bool = True, stream=None):
+    """fp4q_quantize2d of several independent BF16 tensors by one call (chained launches in one stream).  xs: list of 2-D BF16 device tensors; outs: matching
+    list of QTensor (allocated when None); tensor_ids: one rounding-stream id per tensor (default 0, 1, ...)."""
+    n = len(xs)
+    if outs is None:
+        outs = [alloc_qtensor(x.shape[0], x.shape[1], x.device, want_t) for x in xs]
+    if tensor_ids is None:
+        tensor_ids = list(range(n))
+    structs = [o.c_struct() for o in outs]                    # kept alive until the call returns
+    jobs = (_CQuantJob * max(n, 1))()
+    for j, x in enumerate(xs):
+        _dev(x, "xs[%d]" % j)
+        if x.dtype != torch.bfloat16 or x.dim() != 2 or (x.numel() and x.stride(1) != 1):
+            raise ValueError("every input must be a 2-D BF16 tensor with contiguous rows")
+        jobs[j] = _CQuantJob(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0) if x.shape[0] else x.shape[1],
+                             ctypes.pointer(structs[j]), int(tensor_ids[j]), flags)
+    _check(lib().fp4q_quantize2d_multi(jobs, n, mode, seed, _stream(stream)), "fp4q_quantize2d_multi")
+    return outs
 
 
 def fp4q_mxfp8_quantize1d(x: torch.Tensor, stream=None):

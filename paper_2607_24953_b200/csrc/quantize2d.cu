@@ -331,20 +331,30 @@ __global__ void __launch_bounds__(128, FP4Q_QUANT_MIN_BLOCKS) quantize2d_kernel(
     __shared__ uint4 qt_stage[128 * 4];   // 128 transposed rows x 64 B (four 16-byte chunks, XOR-swizzled)
     __shared__ uint4 rnd_stage[MODE == FP4Q_ROUND_STOCHASTIC ? 8 * 128 : 1];   // per thread: 8 rows x 16 random bytes
     __shared__ uint32_t xchg[BLK == 64 ? 16 : 1];   // 64x64 blocks: maxima of the four warps' two half blocks
+    // Programmatic dependent launch (used by fp4q_quantize2d_multi to chain the launches of independent tensors in
+    // one stream): a launch configured as this one's dependent may start filling SMs as soon as every CTA of this
+    // grid is resident, i.e. beside this grid's last wave.  Without such a configuration both instructions do nothing.
+    asm volatile("griddepcontrol.launch_dependents;");
     const int64_t bx = (int64_t)blockIdx.x % p.grid_x, by = (int64_t)blockIdx.x / p.grid_x;
     const bool full = p.x_vec_ok == 2 && p.rng_aligned && (by + 1) * 128 <= p.rows && (bx + 1) * 128 <= p.cols;
     if (full) quantize_tile<MODE, true, BLK>(p, qt_stage, rnd_stage, xchg);
     else quantize_tile<MODE, false, BLK>(p, qt_stage, rnd_stage, xchg);
+    // A dependent grid does not read what its predecessor wrote (different tensors), so it never waited for it; it
+    // waits here, after its own stores, so that the grids of a chain still COMPLETE in launch order and whatever is
+    // enqueued after the chain sees every tensor of it.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace fp4q
 
 using namespace fp4q;
 
-extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
-                                       const fp4q_tensor *out, fp4q_round mode, uint64_t seed,
-                                       uint32_t tensor_id, uint32_t flags, void *stream)
+// Argument checks and kernel parameters of one tensor.  *n_cta = 0 for an empty tensor (nothing to launch).
+static fp4q_status prepare_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x, const fp4q_tensor *out,
+                                      fp4q_round mode, uint64_t seed, uint32_t tensor_id, uint32_t flags, Quant2dParams &p,
+                                      int64_t *n_cta)
 {
+    *n_cta = 0;
     if (rows < 0 || cols < 0) return FP4Q_ERR_SHAPE;
     if (mode != FP4Q_ROUND_NEAREST && mode != FP4Q_ROUND_STOCHASTIC) return FP4Q_ERR_UNSUPPORTED;
     if (flags & ~(FP4Q_INDEX_TRANSPOSED | FP4Q_BLOCK_16 | FP4Q_BLOCK_64)) return FP4Q_ERR_UNSUPPORTED;
@@ -359,7 +369,6 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
     if (!aligned(x_bf16, 2) || !aligned(out->q_rm, 16) || out->ld_rm % 16 != 0) return FP4Q_ERR_ALIGN;
     if (out->q_t && (!aligned(out->q_t, 16) || out->ld_t % 16 != 0)) return FP4Q_ERR_ALIGN;
 
-    Quant2dParams p;
     p.x = static_cast<const uint16_t *>(x_bf16);
     p.rows = rows; p.cols = cols; p.ld_x = ld_x;
     p.q_rm = out->q_rm; p.ld_rm = out->ld_rm;
@@ -371,9 +380,19 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
     p.x_vec_ok = (aligned(x_bf16, 32) && ld_x % 16 == 0) ? 2 : (aligned(x_bf16, 16) && ld_x % 8 == 0) ? 1 : 0;
     p.rng_aligned = cols % 16 == 0 && !(flags & FP4Q_INDEX_TRANSPOSED);
     philox_round_keys(seed, p.keys);
+    *n_cta = p.grid_x * ceil_div(rows, 128);
+    if (*n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
+    return FP4Q_OK;
+}
 
-    const int64_t n_cta = p.grid_x * ceil_div(rows, 128);
-    if (n_cta > 0x7FFFFFFF) return FP4Q_ERR_UNSUPPORTED;
+extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t cols, int64_t ld_x,
+                                       const fp4q_tensor *out, fp4q_round mode, uint64_t seed,
+                                       uint32_t tensor_id, uint32_t flags, void *stream)
+{
+    Quant2dParams p;
+    int64_t n_cta;
+    if (fp4q_status st = prepare_quantize2d(x_bf16, rows, cols, ld_x, out, mode, seed, tensor_id, flags, p, &n_cta)) return st;
+    if (n_cta == 0) return FP4Q_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool sr = mode == FP4Q_ROUND_STOCHASTIC;
     if (flags & FP4Q_BLOCK_16) {
@@ -388,4 +407,46 @@ extern "C" fp4q_status fp4q_quantize2d(const void *x_bf16, int64_t rows, int64_t
         quantize2d_kernel<FP4Q_ROUND_NEAREST><<<(unsigned)n_cta, 128, 0, s>>>(p);
     }
     return cudaGetLastError() == cudaSuccess ? FP4Q_OK : FP4Q_ERR_CUDA;
+}
+
+extern "C" fp4q_status fp4q_quantize2d_multi(const fp4q_quantize_job *jobs, int32_t n_jobs, fp4q_round mode, uint64_t seed,
+                                             void *stream)
+{
+    if (n_jobs < 0) return FP4Q_ERR_SHAPE;
+    if (n_jobs > 0 && !jobs) return FP4Q_ERR_NULL;
+    // every job is checked before the first launch: an argument error leaves the stream untouched
+    for (int32_t j = 0; j < n_jobs; j++) {
+        if (jobs[j].flags & (FP4Q_BLOCK_16 | FP4Q_BLOCK_64)) return FP4Q_ERR_UNSUPPORTED;   // 32 x 32 blocks only
+        Quant2dParams p;
+        int64_t n_cta;
+        if (fp4q_status st = prepare_quantize2d(jobs[j].x_bf16, jobs[j].rows, jobs[j].cols, jobs[j].ld_x, jobs[j].out, mode, seed,
+                                                jobs[j].tensor_id, jobs[j].flags, p, &n_cta))
+            return st;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // One launch of the one-tensor kernel per tensor, each after the first configured as the programmatic dependent of
+    // the one before it: the tensors are independent, so a launch may begin beside its predecessor's last wave instead
+    // of after it (what two streams would give, in one stream).
+    bool first = true;
+    for (int32_t j = 0; j < n_jobs; j++) {
+        Quant2dParams p;
+        int64_t n_cta;
+        prepare_quantize2d(jobs[j].x_bf16, jobs[j].rows, jobs[j].cols, jobs[j].ld_x, jobs[j].out, mode, seed, jobs[j].tensor_id,
+                           jobs[j].flags, p, &n_cta);
+        if (n_cta == 0) continue;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)n_cta);
+        cfg.blockDim = dim3(128);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = first ? 0 : 1;
+        const cudaError_t e = mode == FP4Q_ROUND_STOCHASTIC ? cudaLaunchKernelEx(&cfg, quantize2d_kernel<FP4Q_ROUND_STOCHASTIC, 32>, p)
+                                                            : cudaLaunchKernelEx(&cfg, quantize2d_kernel<FP4Q_ROUND_NEAREST, 32>, p);
+        if (e != cudaSuccess) return FP4Q_ERR_CUDA;
+        first = false;
+    }
+    return FP4Q_OK;
 }

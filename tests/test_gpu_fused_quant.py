@@ -55,7 +55,7 @@ def test_exact_operands_match_the_oracle_bit_for_bit(T, mode):
     compare_logical(yq, o_rm, o_t, o_s, T, N)
 
 
-@pytest.mark.parametrize("T,N,K", [(128, 256, 256), (300, 272, 1000), (1000, 1040, 320), (33, 16, 64)])
+@pytest.mark.parametrize("T,N,K", [(128, 256, 256), (300, 272, 1008), (1000, 1040, 320), (33, 16, 64)])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_fused_equals_product_then_quantize(T, N, K, mode):
     X = workloads.activations_student_t(T, K, 700, "cuda")
@@ -72,7 +72,7 @@ def test_fused_equals_product_then_quantize(T, N, K, mode):
     compare_logical(fused, c_rm, c_t, c_s, T, N)
 
 
-@pytest.mark.parametrize("T,N,K", [(300, 272, 1000), (1000, 1040, 320)])
+@pytest.mark.parametrize("T,N,K", [(300, 272, 1008), (1000, 1040, 320)])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_general_operands_against_the_oracle_in_two_steps(T, N, K, mode):
     """General operands (FP32 accumulation order differs from the oracle's): the BF16 product is within the GEMM

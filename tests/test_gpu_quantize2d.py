@@ -163,3 +163,59 @@ def _oracle_window(rows_bits, total_rows, cols, I, J, seed, tid):
                                  I, I + 2, J, J + 3, q_rm.ctypes.data, 48, q_t.ctypes.data, 32, s.ctypes.data, 3)
     assert rc == 0
     return q_rm, q_t, s
+
+
+def test_multi_tensor_call_equals_one_call_per_tensor():
+    # several tensors in one call (mixed sizes, ragged edges, an empty one, an unaligned view): the bytes are those
+    # of fp4q_quantize2d called once per tensor, hence the oracle's
+    g = torch.Generator(device="cuda").manual_seed(12)
+    shapes = [(256, 256), (100, 200), (0, 64), (384, 1024), (1, 1), (130, 72), (512, 128)]
+    xs = [torch.randn(r, c, generator=g, device="cuda").to(torch.bfloat16) for r, c in shapes]
+    big = torch.randn(260, 300, generator=g, device="cuda").to(torch.bfloat16)
+    xs.append(big[3:200, 5:133])                                  # odd offset, pitch 300
+    for mode in MODES:
+        ids = [7 + 3 * j for j in range(len(xs))]
+        outs = binding.fp4q_quantize2d_multi(xs, mode=mode, seed=21, tensor_ids=ids)
+        torch.cuda.synchronize()
+        for x, q, tid in zip(xs, outs, ids):
+            if x.numel() == 0:
+                continue
+            one = gpu_quantize(x, mode, seed=21, tensor_id=tid)
+            assert all(np.array_equal(a, b) for a, b in zip(logical(q), logical(one)))
+        # and directly against the oracle for two of them
+        for j in (1, 5):
+            o_rm, o_t, o_s = oracle.quantize2d(workloads.bf16_bits(xs[j]), mode, 21, ids[j])
+            g_rm, g_t, g_s = logical(outs[j])
+            r, c = shapes[j]
+            assert np.array_equal(g_s, o_s) and np.array_equal(g_rm[:, :(c + 1) // 2], o_rm) and np.array_equal(g_t[:, :(r + 1) // 2], o_t)
+
+
+def test_multi_tensor_call_with_many_tensors():
+    g = torch.Generator(device="cuda").manual_seed(13)
+    xs = [torch.randn(64 + 32 * (j % 3), 96, generator=g, device="cuda").to(torch.bfloat16) for j in range(70)]
+    outs = binding.fp4q_quantize2d_multi(xs, mode=binding.ROUND_STOCHASTIC, seed=5)
+    torch.cuda.synchronize()
+    for j in (0, 31, 32, 33, 69):
+        one = gpu_quantize(xs[j], binding.ROUND_STOCHASTIC, seed=5, tensor_id=j)
+        assert all(np.array_equal(a, b) for a, b in zip(logical(outs[j]), logical(one)))
+
+
+def test_ragged_outputs_do_not_write_outside_their_extent():
+    # the quantizers use plain stores: guard bytes before and after every output buffer must survive
+    for rows, cols in [(33, 31), (100, 200), (129, 257), (1, 1)]:
+        x = torch.randn(rows, cols, device="cuda").to(torch.bfloat16)
+        q = binding.alloc_qtensor(rows, cols, "cuda")
+        guard = 256
+        bufs = {}
+        for name in ("q_rm", "q_t", "scale"):
+            t = getattr(q, name)
+            flat = torch.full((guard + t.numel() + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+            bufs[name] = flat
+            setattr(q, name, flat[guard:guard + t.numel()].view(t.shape))
+        binding.fp4q_quantize2d(x, out=q, mode=binding.ROUND_STOCHASTIC, seed=3, tensor_id=1)
+        torch.cuda.synchronize()
+        for name, flat in bufs.items():
+            assert bool((flat[:guard] == 0xA5).all()) and bool((flat[-guard:] == 0xA5).all()), (name, rows, cols)
+        o_rm, o_t, o_s = oracle.quantize2d(workloads.bf16_bits(x), oracle.MODE_STOCHASTIC, 3, 1)
+        assert np.array_equal(q.scale.cpu().numpy()[:, :o_s.shape[1]], o_s)
+        assert np.array_equal(q.q_rm.cpu().numpy()[:, :o_rm.shape[1]], o_rm) and np.array_equal(q.q_t.cpu().numpy()[:, :o_t.shape[1]], o_t)

@@ -1,6 +1,6 @@
 """The N>1 path of the benchmark is 'replicas only': ranks run the same step on their own GPU and rank 0
 reports units of all ranks over the slowest rank's time.  The reduction is exercised here with two gloo
-ranks on the CPU."""
+ranks on the CPU, once in-process and once through the launcher that `bench.py --gpus N` itself uses."""
 import os
 import sys
 
@@ -45,3 +45,27 @@ def test_single_process_passthrough():
     import bench
     assert bench.max_over_ranks([1.5, 2.5], None) == [1.5, 2.5]
     assert bench.aggregate_throughput(10.0, 1, 1000.0) == 10.0
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` outside a torchrun launch re-executes itself as two ranks; here with the host-side
+    self-test (gloo on CPU) in place of the GPU step: rank 0 prints one line with n_gpus = 2, the slowest rank's time
+    and the units of both ranks."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-selftest"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-1000:] + r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                  # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 11.0
+    assert abs(lines[0]["value"] - 2 * 1000.0 / 11e-3) < 1e-6
+
+
+def test_launcher_command_shape():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "2"], port=29999)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd and cmd[cmd.index("--nproc-per-node") + 1] == "4"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "4", "--steps", "2"]
