@@ -227,8 +227,8 @@ fp4q_status fp4q_mxfp8_qk(const uint8_t *xq, int64_t ld_xq, const uint8_t *xs, i
                           void *ws, size_t ws_bytes, void *stream);
 
 /*
- * fp4q_quantize1d -- 1D-block FP4 quantization, the layout the paper keeps for activations (Section 3.1, "We retain a
- * 1D layout for activations"; appendix "Quantization Placement"): one UE8M0 scale per 32 consecutive elements of a
+ * fp4q_quantize1d -- 1D-block FP4 quantization, the layout the paper keeps for activations (Section 3,
+ * "Application to linear layers"; appendix "Quantization Placement"): one UE8M0 scale per 32 consecutive elements of a
  * row of x[rows, cols], otherwise the arithmetic of fp4q_quantize2d (truncation-free scale with bound 6, E2M1 codes,
  * nearest-even or stochastic rounding with the random byte of element index i*cols + j, non-finite inputs as there).
  * q [rows, ld_q] packed two codes per byte (low nibble = even column; ld_q >= ceil32(cols)/2, multiple of 16, q

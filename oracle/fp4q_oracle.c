@@ -378,8 +378,8 @@ void orc_dequantize2d_block(const uint8_t *q_rm, int64_t ld_rm, const uint8_t *s
 /* ------------------------------------------------------- 1D (1 x 32) FP4 blocks */
 
 /*
- * The activation layout the paper keeps (Section 3.1, "We retain a 1D layout for activations"; appendix
- * "Quantization Placement", paragraph Activations): one scale per 32 consecutive elements of a row, everything
+ * The activation layout the paper keeps (Section 3, "Application to linear layers": activations stay in 1D
+ * blocks; appendix "Quantization Placement", paragraph Activations): one scale per 32 consecutive elements of a row, everything
  * else as in the 2D scheme - truncation-free power-of-two scale, E2M1 codes, nearest-even or stochastic rounding
  * with the random byte of the element's row-major index i*cols + j (j*rows + i with the transposed-index flag).
  * q[rows, ld_q] packed two codes per byte (low nibble = even column), scale[rows, ld_s], ld_s >= ceil(cols/32).

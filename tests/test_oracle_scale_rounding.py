@@ -54,7 +54,7 @@ def test_scale_special_cases():
 
 
 def test_truncation_free_no_value_exceeds_qp():
-    # "all values fall within the representable range" (Section 3.1): M/S <= Qp for every M, and the
+    # Section 3.1: with the truncation-free scale nothing clips: M/S <= Qp for every M, and the
     # scale is the smallest such power of two unless clamped at 2^-127.
     for bits in ALL_POSITIVE_FINITE_BF16:
         M = bf16_fraction(bits)
