@@ -223,6 +223,12 @@ def run_gpu(args):
     dw_buf = torch.empty((max(o["N"] * o["K"] for o in ops),), dtype=torch.float32, device=dev)
     ws = binding.alloc_workspace(dev)
     gemm_flops = sum(2.0 * T * o["N"] * o["K"] for o in ops)
+    # algorithmic bytes of the 21 GEMM launches: both operands' payloads and scales read once, the output written once
+    # (forward and dgrad in BF16, wgrad in FP32)
+    pay = lambda r, c: r * c * (0.5 + 1.0 / 1024)
+    gemm_alg_bytes = sum(pay(T, o["K"]) + pay(o["N"], o["K"]) + 2.0 * T * o["N"] +        # forward
+                         pay(T, o["N"]) + pay(o["N"], o["K"]) + 2.0 * T * o["K"] +        # dgrad
+                         pay(T, o["N"]) + pay(T, o["K"]) + 4.0 * o["N"] * o["K"] for o in ops)
 
     def outputs(o):
         return (y_buf[:, :o["N"]], dx_buf[:, :o["K"]], dw_buf[:o["N"] * o["K"]].view(o["N"], o["K"]))
@@ -468,6 +474,7 @@ def run_gpu(args):
                 "frac_of_sustained_peak": achieved_tf / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16),
                 "frac_of_nominal_9pf": achieved_tf / 9000.0,
                 "flops_per_launch": 3 * gemm_flops / (3 * len(ops)), "ms_per_launch": gemm_ms_per_launch,
+                "algorithmic_bytes_per_launch": gemm_alg_bytes / (3 * len(ops)),
                 "time_share_of_step": (f_ms + d_ms + w_ms) / ms_per_step}
     q_gbs_1 = quant_bytes / (q_ms * 1e-3) / 1e9
     roofline_quantize = {"kernel": "quantize2d_kernel<stochastic>", "bound": "hbm", "achieved": q_gbs_1,
@@ -550,8 +557,8 @@ def fill_traffic(roofline, roofline_quantize):
         with open(path) as f:
             t = json.load(f)
         # captured on a smaller case and scaled by the units processed (traffic grows in proportion)
-        if "gemm_bytes_per_flop" in t:
-            roofline["traffic"] = t["gemm_bytes_per_flop"] * roofline["flops_per_launch"]
+        if "gemm_dram_over_algorithmic" in t:   # measured on one full-size launch (7B gate/up shape)
+            roofline["traffic"] = t["gemm_dram_over_algorithmic"] * roofline["algorithmic_bytes_per_launch"]
         if "quantize_dram_bytes_per_algorithmic_byte" in t:
             roofline_quantize["traffic"] = t["quantize_dram_bytes_per_algorithmic_byte"] * roofline_quantize["bytes_per_launch"]
     except Exception:
@@ -858,7 +865,12 @@ def run_kernel(args):
         qx = binding.fp4q_quantize2d(workloads.activations_student_t(T, K, 1, dev), mode=1, seed=3, tensor_id=1)
         qw = binding.fp4q_quantize2d(workloads.weights(N, K, 2, dev), mode=1, seed=3, tensor_id=0)
         qdy = binding.fp4q_quantize2d(workloads.gradients_rowscaled(T, N, 3, dev), mode=1, seed=3, tensor_id=2)
-        if args.kernel == "gemm_fwd":
+        if args.kernel == "gemm_fwd_b16":
+            qx16 = binding.fp4q_quantize2d(workloads.activations_student_t(T, K, 1, dev), flags=binding.BLOCK_16)
+            qw16 = binding.fp4q_quantize2d(workloads.weights(N, K, 2, dev), flags=binding.BLOCK_16)
+            out = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+            fn = lambda: binding.fp4q_gemm_fwd_b16(qx16, qw16, out=out, ws=ws)
+        elif args.kernel == "gemm_fwd":
             out = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
             fn = lambda: binding.fp4q_gemm_fwd(qx, qw, out=out, ws=ws)
         elif args.kernel == "gemm_dgrad":
@@ -897,7 +909,7 @@ def main():
     ap.add_argument("--rank-selftest", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--kernel", default=None, choices=["quantize", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "quantize1d", "quantize1d_t",
-                                                        "gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm"],
+                                                        "gemm_fwd_act1d", "gemm_wgrad_act1d", "mxfp8_gemm", "gemm_fwd_b16"],
                     help="run one kernel on --shape a few times (for profiler captures) instead of the benchmark")
     ap.add_argument("--shape", default="16384x4096", help="RxC for quantize, TxNxK for the GEMMs")
     ap.add_argument("--iters", type=int, default=3)
