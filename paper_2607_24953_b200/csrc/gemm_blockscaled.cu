@@ -97,6 +97,11 @@ struct Cfg {
     // contractions - plain stores of the 64 KB tile filled the SM's path to L2 and the TMA loads issued meanwhile
     // took 6500-8000 cycles instead of 3000; the staging costs that kernel its fourth ring stage.
     static constexpr bool kTmaStores = CTAS == 2 || !kRowImages;
+    // One-CTA kernel of the 2D kind (grouped products): its 48 KB stages keep the TMA unit busy ~740 of every ~800 cycles,
+    // so a producer that also polls (a poll queues behind the loads the same warp has just issued) leaves gaps.  There
+    // the producer is split: warp 2 waits for free slots and arms their barriers, warp 0 only issues loads; the MMA warp
+    // waits on its barriers itself (measured: MoE expert layer 1.95 -> 2.07 PFLOP/s; no gain for the pair kernel).
+    static constexpr bool kSplitProducer = KIND == KIND_MXF4 && CTAS == 1;
     static constexpr int kStages = (CTAS == 2 ? 5 : (kTmaStores ? 3 : 4)) - (kRowImages ? 1 : 0);
     static constexpr int kSmemCache = kCompactBytes + (kImageBufs + kRawBufs) * kCacheBufBytes;
     static constexpr int kBRows = CTAS == 2 ? 128 : 256;
@@ -1085,6 +1090,18 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         TRACE_DECL(c_empty); TRACE_DECL(c_issue); TRACE_DECL(c_rounds);
         TRACE_T0(tt);
         int ev_j = 0;
+        while (Cfg<KIND, CTAS>::kSplitProducer && pr.valid(p)) {
+            asm volatile("bar.sync %0, 64;" ::"r"(8 + stage) : "memory");   // the poller (warp 2) has seen the slot free and armed its barrier
+            if (issuer && !(withhold_load != 0u && (uint32_t)ev_j + 1u == withhold_load)) {
+                const Tile &t = pr.t;
+                const int xa = (t.a_k0 + pr.it * kStageElems) / kElemsPerByte, xb = (t.b_k0 + pr.it * kStageElems) / kElemsPerByte;
+                tma_load_2d(smem_u32(smem_a + stage * kAStageBytes), &tmA, xa, t.a_row0, bar_full + 8 * stage);
+                tma_load_2d(smem_u32(smem_b + stage * kBStageBytes), &tmB, xb, t.b_load_row0, bar_full + 8 * stage);
+            }
+            ev_j++;
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            pr.next(p, kStageElems);
+        }
         while (ok && pr.valid(p)) {
             int n_free = 0;
 #ifdef FP4Q_TRACE
@@ -1142,7 +1159,8 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         // warp never reads shared memory inside the loop: a shared-memory access of this warp queues behind its own
         // pending MMAs and stalls the tensor pipe for ~200 cycles per poll.  A watcher warp polls the stage's "full"
         // barrier (and, for 2D scales, the accumulator's "empty" barrier) and hands over through a named barrier.
-        uint32_t stage = 0;
+        uint32_t stage = 0, full_phase = 0, acc_empty_phase = 0;
+        bool mma_ok = true;   // split producer only: this warp's own waits have not run out
         BufRing ring;   // image buffer of the current unit
         const bool issuer = elect_one();
         int ev_j = 0;
@@ -1155,7 +1173,19 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             if (n_it == 0) continue;
             TRACE_ADD(c_acc, tt);
             for (int it = 0; it < n_it; it++) {
-                named_sync(1 + stage);   // the watcher has seen the operands and both scale images of this stage
+                if (Cfg<KIND, CTAS>::kSplitProducer) {
+                    // no watcher: the elected lane waits for the accumulator, the unit's scale images and the operands itself
+                    if (lane == 0 && mma_ok) {
+                        if (it == 0) mma_ok = mbar_wait_impl<0, true>(bar_acc_empty, acc_empty_phase ^ 1u, abort_flag, p.status, wait_limit, 0x200u);
+                        if (mma_ok && (it & (kUnitStages - 1)) == 0)
+                            mma_ok = mbar_wait_impl<0, true>(bar_cache_full + 8 * ring.buf, ring.phase, abort_flag, p.status, wait_limit, 0x510u + ring.buf);
+                        if (mma_ok) mma_ok = mbar_wait_impl<0, true>(bar_full + 8 * stage, full_phase, abort_flag, p.status, wait_limit, 0x300u + stage);
+                    }
+                    if (it == 0) acc_empty_phase ^= 1u;
+                    __syncwarp();
+                } else {
+                    named_sync(1 + stage);   // the watcher has seen the operands and both scale images of this stage
+                }
                 tcgen05_fence_after();
                 TRACE_ADD(c_sync, tt);
                 if (lane == 0) TRACE_EV(2, ev_j);
@@ -1219,7 +1249,7 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 TRACE_ADD(c_issue, tt);
                 if (lane == 0) TRACE_EV(3, ev_j);
                 ev_j++;
-                if (++stage == kStages) stage = 0;
+                if (++stage == kStages) { stage = 0; full_phase ^= 1u; }
             }
         }
         if (leader && *abort_flag) {
@@ -1351,7 +1381,21 @@ gemm_block_scaled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         int ev_j = 0;
         bool unit_seen = false;   // lane 0: the next unit's scale images have been seen complete
         uint32_t ahead = 0;   // stages after the current one whose "full" barrier is already known to be complete
-        while (leader && sg.valid(p)) {
+        if (Cfg<KIND, CTAS>::kSplitProducer) {
+            // poller half of the split producer: waits for each slot to be free, arms its barrier for the stage's bytes and
+            // releases the issuing warp; after a timeout it keeps releasing, so that warp 0 always reaches its end
+            while (sg.valid(p)) {
+                if (lane == 0) {
+                    if (ok) ok = mbar_wait_impl<0, true>(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status, wait_limit, 0x100u + stage);
+                    mbar_arrive_expect_tx(bar_full + 8 * stage, kAStageBytes + kBStageBytes);
+                }
+                __syncwarp();
+                asm volatile("bar.sync %0, 64;" ::"r"(8 + stage) : "memory");
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                sg.next(p, kStageElems);
+            }
+        }
+        while (!Cfg<KIND, CTAS>::kSplitProducer && leader && sg.valid(p)) {
             if (lane == 0) TRACE_EV(4, ev_j);
             if (ahead > 0) {
                 ahead--;
